@@ -1,0 +1,189 @@
+/*
+ * eqat.h - C ABI of the B200 (sm_100a) library for the group-wise low-bit
+ * quantised linear layer of EfficientQAT (arXiv 2407.11062).
+ *
+ * The layer is the one both training phases of the paper run through:
+ *   Block-AP (Sec. 3.2): the weight is fake-quantised in the graph,
+ *       W_int = clamp(round(W / s) + z, 0, 2^N - 1)          (Eq. 1)
+ *       W_hat = (W_int - z) * s                              (Eq. 2)
+ *     and W, s, z receive straight-through gradients (appendix "Gradient of
+ *     Trainable Parameters in Block-AP", Eqs. 3-5).
+ *   E2E-QP (Sec. 3.3): W_int is frozen and stored in N bits, only Eq. 2 runs,
+ *     and the step size s is trained with d w_hat / d s = w_q - z.
+ *
+ * Conventions shared by every entry point
+ *   - W is [out_features, in_features] row-major, as in Y = X * W^T.  A
+ *     quantisation group is `group` consecutive elements along in_features
+ *     inside one row; s and z are [out_features, in_features / group]
+ *     row-major.  X is [tokens, in_features], Y and dY are [tokens,
+ *     out_features], all row-major and dense (no padding, no strides).
+ *   - bf16 / fp16 values are passed as their 16-bit patterns.
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller unless its
+ *     name starts with `h_` (host).  The library allocates no memory and keeps
+ *     no pointer after a call returns.  Device base pointers must be 16-byte
+ *     aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls enqueue work on `stream` and return without waiting for it.
+ *   - Return value: EQAT_OK, or a negative eqat_status decided on the host
+ *     BEFORE anything is launched (outputs untouched), or EQAT_ERR_CUDA if the
+ *     runtime rejected a launch.  A kernel that gives up a bounded wait records
+ *     it in a device status word read by eqat_device_status().
+ *   - Gradients are overwritten, never accumulated.  No bias term (the
+ *     quantised layers of the paper have none).
+ *   - Tensor contents are not inspected: s <= 0, NaN or Inf give undefined
+ *     values (never out-of-bounds accesses).
+ *
+ * Supported geometry: bits in {2,3,4}; group in {32,64,128,256} or a larger
+ * multiple of 32 dividing in_features (e.g. group == in_features, one group
+ * per row) for the element-wise and codec entry points; in_features a
+ * multiple of 128.  The GEMM entry points also need out_features a multiple
+ * of 64; tokens may be any positive number.  The packed-weight GEMMs need
+ * group in {64,128,256}.
+ */
+#ifndef EQAT_H_
+#define EQAT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint16_t eqat_bf16;   /* bfloat16 bit pattern */
+typedef uint16_t eqat_fp16;   /* IEEE binary16 bit pattern */
+
+typedef enum {
+  EQAT_OK = 0,
+  EQAT_ERR_NULL = -1,         /* a required pointer is NULL                          */
+  EQAT_ERR_SHAPE = -2,        /* a size is non-positive or violates a divisibility   */
+  EQAT_ERR_ALIGN = -3,        /* a device pointer is not 16-byte aligned             */
+  EQAT_ERR_UNSUPPORTED = -4,  /* bits / group / mode outside the supported set       */
+  EQAT_ERR_WORKSPACE = -5,    /* workspace missing, misaligned or too small          */
+  EQAT_ERR_CUDA = -6,         /* the CUDA runtime or driver reported an error        */
+  EQAT_ERR_TIMEOUT = -7       /* a kernel gave up a bounded wait (device status)     */
+} eqat_status;
+
+/* Problem descriptor: plain data, read during the call, never retained. */
+typedef struct {
+  int32_t bits;               /* N: 2, 3 or 4                                         */
+  int32_t group;              /* g: elements per quantisation group along in_features */
+  int32_t out_features;
+  int32_t in_features;
+  int64_t tokens;             /* rows of X / dY (ignored by weight-only entry points) */
+  int32_t dz_mode;            /* clamped-branch value of d w_hat / d z:
+                                 0 = -s (derivative of Eq. 2 at a saturated code),
+                                 1 = -1 (Eq. 4 as printed)                            */
+  int32_t reserved;           /* must be 0                                            */
+} eqat_desc;
+
+/* Operations that need caller-provided scratch memory (eqat_workspace_bytes). */
+enum { EQAT_OP_FAKEQUANT_BWD = 1, EQAT_OP_PACKED_BWD_DS = 2 };
+
+const char* eqat_status_string(int status);
+int eqat_version(void);
+
+/* Bytes of device scratch the given operation needs for this problem (0 if none,
+ * (size_t)-1 if desc/op is invalid).  The workspace must be 256-byte aligned. */
+size_t eqat_workspace_bytes(const eqat_desc* desc, int op);
+
+/* Reads and clears the device status word of the current device (synchronises
+ * the device).  *h_status receives EQAT_OK or EQAT_ERR_TIMEOUT; *h_detail (may be
+ * NULL) a code naming the wait that was abandoned. */
+int eqat_device_status(int* h_status, int* h_detail);
+
+/* ------------------------------------------------------------------ helpers */
+
+/* Round-to-nearest initialisation of the quantisation parameters from each
+ * group's range (the paper does not describe its initialisation; this is the
+ * min/max rule):  s = max((max - min) / (2^N - 1), 2^-14),
+ * z = clamp(-round(min / s), 0, 2^N - 1), evaluated in binary32.
+ *   W [out,in] bf16 (in)   s, z [out,in/g] fp32 (out; z is integer valued) */
+int eqat_minmax_init(const eqat_desc* desc, const eqat_bf16* W, float* s, float* z, void* stream);
+
+/* ------------------------------------------------------------------ Block-AP */
+
+/* Eq. 1 followed by Eq. 2: W_hat = (clamp(round(W/s) + round(z), 0, 2^N-1) - round(z)) * s.
+ * The quotient W/s is an IEEE binary32 division, rounded half-to-even.
+ *   W [out,in] bf16, s, z [out,in/g] fp32 (in)   W_hat [out,in] bf16 (out) */
+int eqat_fakequant_weight(const eqat_desc* desc, const eqat_bf16* W, const float* s, const float* z,
+                          eqat_bf16* W_hat, void* stream);
+
+/* Block-AP forward (Sec. 3.2): W_hat as above, then Y = X * W_hat^T with fp32
+ * accumulation.  W_hat is written out because the backward pass reads it.
+ *   X [T,in] bf16, W, s, z (in)   Y [T,out] bf16, W_hat [out,in] bf16 (out) */
+int qlinear_fakequant_fwd(const eqat_desc* desc, const eqat_bf16* X, const eqat_bf16* W, const float* s,
+                          const float* z, eqat_bf16* Y, eqat_bf16* W_hat, void* stream);
+
+/* Straight-through backward of the fake quantiser (Eqs. 3-5, upper bound read
+ * as 2^N - 1 as in Eq. 1, bounds inclusive).  With p = round(w/s) + round(z):
+ *   dW      = dW_hat            if 0 <= p <= 2^N-1, else 0
+ *   ds[o,g] = sum over the group of dW_hat * (round(w/s) - w/s | -z | 2^N-1-z)
+ *   dz[o,g] = sum over the group of dW_hat * (0 | -s | -s)      (dz_mode 1: -1)
+ *   dW_hat, W [out,in] bf16, s, z fp32 (in)   dW bf16, ds, dz fp32 (out)
+ * dz may be NULL (not computed). */
+int eqat_ste_bwd(const eqat_desc* desc, const eqat_bf16* dW_hat, const eqat_bf16* W, const float* s,
+                 const float* z, eqat_bf16* dW, float* ds, float* dz, void* stream);
+
+/* Block-AP backward: dX = dY * W_hat, dW_hat = dY^T * X (kept in bf16 in the
+ * workspace), then eqat_ste_bwd.  Needs eqat_workspace_bytes(desc,
+ * EQAT_OP_FAKEQUANT_BWD) bytes of scratch.
+ *   X [T,in], dY [T,out], W, W_hat [out,in] bf16, s, z (in)
+ *   dX [T,in] bf16, dW [out,in] bf16, ds, dz [out,in/g] fp32 (out) */
+int qlinear_fakequant_bwd(const eqat_desc* desc, const eqat_bf16* X, const eqat_bf16* dY, const eqat_bf16* W,
+                          const float* s, const float* z, const eqat_bf16* W_hat,
+                          eqat_bf16* dX, eqat_bf16* dW, float* ds, float* dz,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------ storage format */
+/* The paper stores W_int and z in N bits and s in fp16 (Sec. 3.2, last
+ * paragraph; N + (N+16)/g bits per parameter, appendix "Size of Quantized
+ * Models") but gives no bit order.  This library's: each row of W_int is a
+ * dense little-endian bit stream, code j in stream bits [N*j, N*j+N), stream
+ * bit b = bit (b % 8) of byte (b / 8); row pitch in*N/8 bytes. */
+
+/* Hand-off from Block-AP to E2E-QP: codes of Eq. 1 packed, zero points as
+ * bytes, step sizes rounded to fp16.
+ *   W, s, z (in)   Wq_packed [out, in*N/8] u8, z8 [out,in/g] u8, s16 [out,in/g] fp16 (out) */
+int eqat_quantize_pack(const eqat_desc* desc, const eqat_bf16* W, const float* s, const float* z,
+                       uint8_t* Wq_packed, uint8_t* z8, eqat_fp16* s16, void* stream);
+
+/* codes [out,in] u8 (each < 2^N) <-> Wq_packed [out, in*N/8]. */
+int eqat_pack(const eqat_desc* desc, const uint8_t* codes, uint8_t* Wq_packed, void* stream);
+int eqat_unpack(const eqat_desc* desc, const uint8_t* Wq_packed, uint8_t* codes, void* stream);
+
+/* Zero points for storage: z8 [out*in/g] u8 <-> one flat N-bit stream of
+ * out*in/g*N/8 bytes with the same bit rule (the count must be a multiple of 8). */
+int eqat_pack_zeros(const eqat_desc* desc, const uint8_t* z8, uint8_t* z_packed, void* stream);
+int eqat_unpack_zeros(const eqat_desc* desc, const uint8_t* z_packed, uint8_t* z8, void* stream);
+
+/* ------------------------------------------------------------------ E2E-QP */
+
+/* Y = X * ((W_int - z) * s)^T, the packed codes expanded tile by tile in
+ * shared memory inside the GEMM (Eq. 2; Sec. 3.3).
+ *   X [T,in] bf16, Wq_packed, s16, z8 (in)   Y [T,out] bf16 (out) */
+int qlinear_packed_fwd(const eqat_desc* desc, const eqat_bf16* X, const uint8_t* Wq_packed,
+                       const eqat_fp16* s16, const uint8_t* z8, eqat_bf16* Y, void* stream);
+
+/* dX = dY * ((W_int - z) * s).
+ *   dY [T,out] bf16, Wq_packed, s16, z8 (in)   dX [T,in] bf16 (out) */
+int qlinear_packed_bwd_dx(const eqat_desc* desc, const eqat_bf16* dY, const uint8_t* Wq_packed,
+                          const eqat_fp16* s16, const uint8_t* z8, eqat_bf16* dX, void* stream);
+
+/* Step-size gradient (Sec. 3.3, d w_hat/d s = w_q - z):
+ *   ds[o,g] = sum_{j in g} (sum_t dY[t,o] X[t,j]) * (W_int[o,j] - z[o,g]),
+ * reduced in the epilogue of the weight-gradient GEMM; the [out,in] weight
+ * gradient is never written to memory.  If dz is not NULL it also receives the
+ * zero-point gradient of the same layer (the Sec. 3.3 variant that trains z),
+ * dz[o,g] = -s[o,g] * sum_{j in g} G[o,j]; s16 is then required, else it may be
+ * NULL.  Needs eqat_workspace_bytes(desc, EQAT_OP_PACKED_BWD_DS) bytes of
+ * scratch (0 for every supported shape: workspace may then be NULL).
+ *   X [T,in], dY [T,out] bf16, Wq_packed, z8 (in)   ds [out,in/g] fp32 (out) */
+int qlinear_packed_bwd_ds(const eqat_desc* desc, const eqat_bf16* X, const eqat_bf16* dY,
+                          const uint8_t* Wq_packed, const uint8_t* z8, const eqat_fp16* s16,
+                          float* ds, float* dz, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* EQAT_H_ */
