@@ -1,0 +1,197 @@
+// C ABI (include/eqat.h): argument validation on the host, then launches.
+#include <stdint.h>
+
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "gemm.cuh"
+
+namespace {
+
+using namespace eqat;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+// Geometry every entry point shares.
+int check_weight_desc(const eqat_desc* d) {
+  if (d == nullptr) return EQAT_ERR_NULL;
+  if (d->reserved != 0) return EQAT_ERR_UNSUPPORTED;
+  if (d->bits < 2 || d->bits > 4) return EQAT_ERR_UNSUPPORTED;
+  if (d->dz_mode != 0 && d->dz_mode != 1) return EQAT_ERR_UNSUPPORTED;
+  if (d->out_features <= 0 || d->in_features <= 0 || d->group <= 0) return EQAT_ERR_SHAPE;
+  if (d->in_features % 128 != 0) return EQAT_ERR_SHAPE;
+  if (d->group % 32 != 0 || d->in_features % d->group != 0) return EQAT_ERR_SHAPE;
+  if (d->group <= 256 && !is_pow2(d->group)) return EQAT_ERR_UNSUPPORTED;
+  if (d->group > 32768) return EQAT_ERR_UNSUPPORTED;
+  if ((int64_t)d->out_features * d->in_features > ((int64_t)1 << 34)) return EQAT_ERR_SHAPE;
+  return EQAT_OK;
+}
+
+int check_gemm_desc(const eqat_desc* d, bool packed) {
+  const int rc = check_weight_desc(d);
+  if (rc != EQAT_OK) return rc;
+  if (d->tokens <= 0 || d->tokens > (int64_t)1 << 30) return EQAT_ERR_SHAPE;
+  if (d->out_features % 64 != 0) return EQAT_ERR_SHAPE;
+  if (packed && !(d->group == 64 || d->group == 128 || d->group == 256)) return EQAT_ERR_UNSUPPORTED;
+  return EQAT_OK;
+}
+
+template <typename... P>
+int check_ptrs(P... ptrs) {
+  const void* v[] = {static_cast<const void*>(ptrs)...};
+  for (const void* p : v)
+    if (p == nullptr) return EQAT_ERR_NULL;
+  for (const void* p : v)
+    if (!aligned16(p)) return EQAT_ERR_ALIGN;
+  return EQAT_OK;
+}
+
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+#define EQAT_TRY(expr)            \
+  do {                            \
+    const int rc__ = (expr);      \
+    if (rc__ != EQAT_OK) return rc__; \
+  } while (0)
+
+}  // namespace
+
+extern "C" {
+
+const char* eqat_status_string(int status) {
+  switch (status) {
+    case EQAT_OK: return "ok";
+    case EQAT_ERR_NULL: return "null pointer";
+    case EQAT_ERR_SHAPE: return "invalid shape";
+    case EQAT_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case EQAT_ERR_UNSUPPORTED: return "unsupported bits/group/mode";
+    case EQAT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case EQAT_ERR_CUDA: return "CUDA error";
+    case EQAT_ERR_TIMEOUT: return "a kernel abandoned a bounded wait";
+    default: return "unknown status";
+  }
+}
+
+int eqat_version(void) { return 100; }
+
+size_t eqat_workspace_bytes(const eqat_desc* d, int op) {
+  if (op == EQAT_OP_FAKEQUANT_BWD) {
+    if (check_gemm_desc(d, false) != EQAT_OK) return (size_t)-1;
+    return (size_t)d->out_features * d->in_features * sizeof(eqat_bf16);   // dW_hat in bf16
+  }
+  if (op == EQAT_OP_PACKED_BWD_DS) {
+    if (check_gemm_desc(d, true) != EQAT_OK) return (size_t)-1;
+    return 0;
+  }
+  return (size_t)-1;
+}
+
+int eqat_device_status(int* h_status, int* h_detail) {
+  if (h_status == nullptr) return EQAT_ERR_NULL;
+  return read_device_status(h_status, h_detail);
+}
+
+int eqat_minmax_init(const eqat_desc* d, const eqat_bf16* W, float* s, float* z, void* stream) {
+  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_ptrs(W, s, z));
+  return launch_minmax(*d, W, s, z, as_stream(stream));
+}
+
+int eqat_fakequant_weight(const eqat_desc* d, const eqat_bf16* W, const float* s, const float* z, eqat_bf16* W_hat,
+                          void* stream) {
+  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_ptrs(W, s, z, W_hat));
+  return launch_fakequant(*d, W, s, z, W_hat, as_stream(stream));
+}
+
+int qlinear_fakequant_fwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* W, const float* s, const float* z,
+                          eqat_bf16* Y, eqat_bf16* W_hat, void* stream) {
+  EQAT_TRY(check_gemm_desc(d, false));
+  EQAT_TRY(check_ptrs(X, W, s, z, Y, W_hat));
+  EQAT_TRY(launch_fakequant(*d, W, s, z, W_hat, as_stream(stream)));
+  return launch_dense_fwd(*d, X, W_hat, Y, as_stream(stream));
+}
+
+int eqat_ste_bwd(const eqat_desc* d, const eqat_bf16* dW_hat, const eqat_bf16* W, const float* s, const float* z,
+                 eqat_bf16* dW, float* ds, float* dz, void* stream) {
+  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_ptrs(dW_hat, W, s, z, dW, ds));
+  if (dz != nullptr && !aligned16(dz)) return EQAT_ERR_ALIGN;
+  return launch_ste_bwd(*d, dW_hat, W, s, z, dW, ds, dz, as_stream(stream));
+}
+
+int qlinear_fakequant_bwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* dY, const eqat_bf16* W,
+                          const float* s, const float* z, const eqat_bf16* W_hat, eqat_bf16* dX, eqat_bf16* dW,
+                          float* ds, float* dz, void* workspace, size_t workspace_bytes, void* stream) {
+  EQAT_TRY(check_gemm_desc(d, false));
+  EQAT_TRY(check_ptrs(X, dY, W, s, z, W_hat, dX, dW, ds));
+  if (dz != nullptr && !aligned16(dz)) return EQAT_ERR_ALIGN;
+  const size_t need = (size_t)d->out_features * d->in_features * sizeof(eqat_bf16);
+  if (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+    return EQAT_ERR_WORKSPACE;
+  eqat_bf16* dW_hat = static_cast<eqat_bf16*>(workspace);
+  cudaStream_t st = as_stream(stream);
+  EQAT_TRY(launch_dense_dx(*d, dY, W_hat, dX, st));
+  EQAT_TRY(launch_dense_dw(*d, dY, X, dW_hat, st));
+  return launch_ste_bwd(*d, dW_hat, W, s, z, dW, ds, dz, st);
+}
+
+int eqat_quantize_pack(const eqat_desc* d, const eqat_bf16* W, const float* s, const float* z, uint8_t* Wq_packed,
+                       uint8_t* z8, eqat_fp16* s16, void* stream) {
+  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_ptrs(W, s, z, Wq_packed, z8, s16));
+  return launch_quantize_pack(*d, W, s, z, Wq_packed, z8, s16, as_stream(stream));
+}
+
+int eqat_pack(const eqat_desc* d, const uint8_t* codes, uint8_t* Wq_packed, void* stream) {
+  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_ptrs(codes, Wq_packed));
+  return launch_pack(*d, codes, Wq_packed, as_stream(stream));
+}
+
+int eqat_unpack(const eqat_desc* d, const uint8_t* Wq_packed, uint8_t* codes, void* stream) {
+  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_ptrs(Wq_packed, codes));
+  return launch_unpack(*d, Wq_packed, codes, as_stream(stream));
+}
+
+int eqat_pack_zeros(const eqat_desc* d, const uint8_t* z8, uint8_t* z_packed, void* stream) {
+  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_ptrs(z8, z_packed));
+  if (((int64_t)d->out_features * d->in_features / d->group) % 8 != 0) return EQAT_ERR_SHAPE;
+  return launch_pack_zeros(*d, z8, z_packed, as_stream(stream));
+}
+
+int eqat_unpack_zeros(const eqat_desc* d, const uint8_t* z_packed, uint8_t* z8, void* stream) {
+  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_ptrs(z_packed, z8));
+  if (((int64_t)d->out_features * d->in_features / d->group) % 8 != 0) return EQAT_ERR_SHAPE;
+  return launch_unpack_zeros(*d, z_packed, z8, as_stream(stream));
+}
+
+int qlinear_packed_fwd(const eqat_desc* d, const eqat_bf16* X, const uint8_t* Wq_packed, const eqat_fp16* s16,
+                       const uint8_t* z8, eqat_bf16* Y, void* stream) {
+  EQAT_TRY(check_gemm_desc(d, true));
+  EQAT_TRY(check_ptrs(X, Wq_packed, s16, z8, Y));
+  return launch_packed_fwd(*d, X, Wq_packed, s16, z8, Y, as_stream(stream));
+}
+
+int qlinear_packed_bwd_dx(const eqat_desc* d, const eqat_bf16* dY, const uint8_t* Wq_packed, const eqat_fp16* s16,
+                          const uint8_t* z8, eqat_bf16* dX, void* stream) {
+  EQAT_TRY(check_gemm_desc(d, true));
+  EQAT_TRY(check_ptrs(dY, Wq_packed, s16, z8, dX));
+  return launch_packed_dx(*d, dY, Wq_packed, s16, z8, dX, as_stream(stream));
+}
+
+int qlinear_packed_bwd_ds(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* dY, const uint8_t* Wq_packed,
+                          const uint8_t* z8, const eqat_fp16* s16, float* ds, float* dz, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  (void)workspace;
+  (void)workspace_bytes;
+  EQAT_TRY(check_gemm_desc(d, true));
+  EQAT_TRY(check_ptrs(X, dY, Wq_packed, z8, ds));
+  if (dz != nullptr) EQAT_TRY(check_ptrs(dz, s16));
+  return launch_packed_ds(*d, X, dY, Wq_packed, z8, s16, ds, dz, as_stream(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,615 @@
+// tcgen05 GEMM kernels for the quantised linear layer.
+//
+// One persistent, warp-specialised kernel template computes
+//     D[M,N] = sum_k A[m,k] * B[n,k]          (bf16 x bf16 -> fp32 in TMEM)
+// for the three contractions of the layer.  Each operand is either K-major
+// (rows of K contiguous elements) or MN-major (the row-major transpose), so no
+// transposed copy of X, dY or W_hat is ever materialised:
+//     Y    = X  * W_hat^T : A = X  [T,in]  K-major,  B = W_hat [out,in] K-major
+//     dX   = dY * W_hat   : A = dY [T,out] K-major,  B = W_hat [out,in] MN-major
+//     dW^  = dY^T * X     : A = dY [T,out] MN-major, B = X     [T,in]  MN-major
+//
+// Roles inside a CTA (one CTA per SM, 128 x BN output tile, 64-deep K blocks):
+//   warp 0      TMA producer: fills a ring of 128B-swizzled shared-memory stages
+//   warp 1      MMA issuer: one thread issues tcgen05.mma into one of two TMEM
+//               accumulators, frees stages with tcgen05.commit
+//   warps 2-5   epilogue: tcgen05.ld the finished accumulator (one TMEM lane
+//               quadrant each) while the next tile is already being multiplied
+//   warps 6-13  (packed-weight kernels only) expand N-bit codes into the bf16 B
+//               operand stage: (q - z) * s in fp32, rounded once to bf16
+// The epilogue either stores the tile as bf16 or, for the E2E-QP step-size
+// gradient, multiplies each accumulator row by (q - z) of the matching packed
+// codes and reduces runs of `group` columns, so the [out,in] weight gradient
+// never leaves the chip.
+//
+// Every wait on an mbarrier is bounded in time; a role that gives up raises a
+// CTA-wide abort flag, records the site in a device status word and all roles
+// fall through to a teardown that drains copies in flight and frees TMEM.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "codec.cuh"
+#include "gemm.cuh"
+#include "ptx.cuh"
+
+namespace eqat {
+
+__device__ int g_device_status[2];   // [0] = eqat_status, [1] = WaitSite
+
+namespace {
+
+constexpr int BM = 128;          // tile rows = TMEM lanes
+constexpr int BK = 64;           // K per stage: one 128-byte swizzle span of bf16
+constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit inputs
+constexpr int kEpiWarp0 = 2;
+constexpr int kDeqWarp0 = 6;
+constexpr int kDeqWarps = 8;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s per wait
+constexpr uint64_t kDrainLimitNs = 50000000ull;    // 50 ms per stage at teardown
+
+enum Epilogue : int { EPI_STORE = 0, EPI_DS = 1 };
+
+struct GemmParams {
+  int M, N, K;
+  eqat_bf16* D;              // EPI_STORE: [M,N] row-major
+  // packed weight (B operand of the packed kernels, epilogue operand of EPI_DS)
+  const uint8_t* Wq;         // [out, in*bits/8]
+  const eqat_fp16* s16;      // [out, in/group]
+  const uint8_t* z8;         // [out, in/group]
+  int out_features, in_features;
+  int group_shift;           // log2(group)
+  float* ds;                 // EPI_DS outputs [out, in/group]
+  float* dz;                 // may be null
+};
+
+template <int BN, bool PACKED>
+struct Cfg {
+  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr int kABytes = BM * BK * 2;
+  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kThreads = PACKED ? (kDeqWarp0 + kDeqWarps) * 32 : kDeqWarp0 * 32;
+  static constexpr int kTmemCols = 2 * BN;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct Control {
+  uint64_t full[8];
+  uint64_t empty[8];
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort;
+};
+static_assert(sizeof(Control) <= 256, "control block must fit its reservation");
+
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort, int site,
+                                             uint64_t limit_ns = kWaitLimitNs) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = ptx::globaltimer_ns();
+  uint32_t n = 0;
+  while (!ptx::mbar_try_wait(bar, parity)) {
+    if ((++n & 31u) == 0u) {
+      if (*abort) return false;
+      if (ptx::globaltimer_ns() - t0 > limit_ns) {
+        *abort = 1;
+        atomicExch(&g_device_status[1], site);
+        atomicExch(&g_device_status[0], (int)EQAT_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, 8-row atoms 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024u >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ void tile_coords(int tile, int num_m, int num_n, int& m_blk, int& n_blk) {
+  // Bands of 16 row-tiles, row-tile fastest inside a band: the ~148 tiles in
+  // flight share 16 A panels and ~9 B panels in L2.
+  const int band_tiles = 16 * num_n;
+  const int band = tile / band_tiles;
+  const int r = tile - band * band_tiles;
+  const int m0 = band * 16;
+  const int h = min(16, num_m - m0);
+  m_blk = m0 + r % h;
+  n_blk = r / h;
+}
+
+// Expand 64 consecutive codes of one weight row into one 128-byte swizzled
+// shared-memory row: element e of the row goes to 16-byte chunk (e/8) ^ rx.
+template <int BITS>
+__device__ __forceinline__ void dequant_row64(const uint32_t (&w)[2 * BITS], float s, float z, uint8_t* row, int rx) {
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  const float zoff = 8388608.0f + z;                    // codes enter as 2^23 + q (exact)
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int j = 8 * c + i;
+        const int bit = BITS * j, word = bit >> 5, off = bit & 31;
+        uint32_t x = w[h * BITS + word] >> off;
+        if (off + BITS > 32) x |= w[h * BITS + word + 1] << (32 - off);
+        v[i] = (__uint_as_float((x & mask) | 0x4B000000u) - zoff) * s;
+      }
+      const uint4 o = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                                 pack_bf16x2(v[6], v[7]));
+      *reinterpret_cast<uint4*>(row + (((h * 4 + c) ^ rx) << 4)) = o;
+    }
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ void load_codes64(const uint8_t* p, uint32_t (&w)[2 * BITS]) {
+  if constexpr (BITS == 2) {
+    const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
+    w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+  } else if constexpr (BITS == 3) {
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+      const uint2 t = __ldg(reinterpret_cast<const uint2*>(p) + i);
+      w[2 * i] = t.x; w[2 * i + 1] = t.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const uint4 t = __ldg(reinterpret_cast<const uint4*>(p) + i);
+      w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
+    }
+  }
+}
+
+// A_MN / B_MN: operand is MN-major.  PACKED: B is expanded from N-bit codes.
+// BITS is used by PACKED and by EPI_DS.
+template <int BN, bool A_MN, bool B_MN, bool PACKED, int EPI, int BITS>
+__global__ void __launch_bounds__(Cfg<BN, PACKED>::kThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+            const GemmParams p) {
+  using C = Cfg<BN, PACKED>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+  const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+  uint8_t* smem = smem_raw + pad;                                  // 1024-byte aligned stages
+  const uint32_t smem_base = raw_addr + pad;
+  Control* ctl = reinterpret_cast<Control*>(smem + C::kStages * C::kStageBytes);
+  volatile int* abort_flag = &ctl->abort;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int num_m = (p.M + BM - 1) / BM;
+  const int num_n = (p.N + BN - 1) / BN;
+  const int num_tiles = num_m * num_n;
+  const int num_kb = (p.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), PACKED ? 1 + kDeqWarps : 1);
+      ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[a]), 1);
+      ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[a]), 4);
+    }
+    ptx::mbar_init(ptx::smem_addr(&ctl->drain), 1);
+    ctl->abort = 0;
+    ptx::fence_mbar_init();
+    ptx::tma_prefetch_desc(&tmap_a);
+    if (!PACKED) ptx::tma_prefetch_desc(&tmap_b);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_base), C::kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      long issued = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int m_blk, n_blk;
+        tile_coords(tile, num_m, num_n, m_blk, n_blk);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_PRODUCER_EMPTY)) {
+            ok = false;
+            break;
+          }
+          const uint32_t full = ptx::smem_addr(&ctl->full[stage]);
+          const uint32_t a_dst = smem_base + stage * C::kStageBytes;
+          const uint32_t b_dst = a_dst + C::kABytes;
+          ptx::mbar_expect_tx(full, PACKED ? C::kABytes : C::kStageBytes);
+          if (A_MN) {
+#pragma unroll
+            for (int b = 0; b < BM / 64; ++b)
+              ptx::tma_load_2d(a_dst + b * (BK * 128), &tmap_a, m_blk * BM + b * 64, kb * BK, full);
+          } else {
+            ptx::tma_load_2d(a_dst, &tmap_a, kb * BK, m_blk * BM, full);
+          }
+          if (!PACKED) {
+            if (B_MN) {
+#pragma unroll
+              for (int b = 0; b < BN / 64; ++b)
+                ptx::tma_load_2d(b_dst + b * (BK * 128), &tmap_b, n_blk * BN + b * 64, kb * BK, full);
+            } else {
+              ptx::tma_load_2d(b_dst, &tmap_b, kb * BK, n_blk * BN, full);
+            }
+          }
+          ++issued;
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok || *abort_flag) {
+        // Drain: every copy this thread started must land before the CTA exits.
+        const long first = issued > C::kStages ? issued - C::kStages : 0;
+        for (long i = first; i < issued; ++i) {
+          const uint32_t bar = ptx::smem_addr(&ctl->full[i % C::kStages]);
+          const uint32_t par = (uint32_t)((i / C::kStages) & 1);
+          const uint64_t t0 = ptx::globaltimer_ns();
+          while (!ptx::mbar_try_wait(bar, par)) {
+            if (ptx::globaltimer_ns() - t0 > kDrainLimitNs) {
+              atomicExch(&g_device_status[1], (int)WAIT_TEARDOWN);
+              break;
+            }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
+                                 ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      constexpr uint32_t a_lbo = A_MN ? BK * 128 : 16, b_lbo = B_MN ? BK * 128 : 16;
+      constexpr uint32_t a_step = A_MN ? UMMA_K * 128 : UMMA_K * 2, b_step = B_MN ? UMMA_K * 128 : UMMA_K * 2;
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        if (!wait_bounded(ptx::smem_addr(&ctl->acc_empty[acc]), acc_phase ^ 1u, abort_flag, WAIT_MMA_ACC_EMPTY)) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!wait_bounded(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL)) {
+            ok = false;
+            break;
+          }
+          ptx::tc_fence_after();
+          const uint32_t a_addr = smem_base + stage * C::kStageBytes;
+          const uint32_t b_addr = a_addr + C::kABytes;
+#pragma unroll
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            ptx::mma_bf16_ss(d_tmem, smem_desc(a_addr + kk * a_step, a_lbo), smem_desc(b_addr + kk * b_step, b_lbo),
+                             idesc, (kb | kk) != 0 ? 1u : 0u);
+          }
+          ptx::mma_commit(ptx::smem_addr(&ctl->empty[stage]));
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::mma_commit(ptx::smem_addr(&ctl->acc_full[acc]));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      // All MMAs of this thread must have retired before TMEM is freed.
+      ptx::mma_commit(ptx::smem_addr(&ctl->drain));
+      wait_bounded(ptx::smem_addr(&ctl->drain), 0u, abort_flag, WAIT_TEARDOWN, kDrainLimitNs * 4);
+    }
+  } else if (warp < kDeqWarp0) {
+    // ------------------------------------------------------------ epilogue
+    const int quad = warp & 3;                        // TMEM lane quadrant this warp may read
+    const int row_in_tile = quad * 32 + lane;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+      int m_blk, n_blk;
+      tile_coords(tile, num_m, num_n, m_blk, n_blk);
+      if (!wait_bounded(ptx::smem_addr(&ctl->acc_full[acc]), acc_phase, abort_flag, WAIT_EPI_ACC_FULL)) break;
+      ptx::tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
+      const int m = m_blk * BM + row_in_tile;
+      if constexpr (EPI == EPI_STORE) {
+        eqat_bf16* drow = p.D + (size_t)m * p.N;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32(t_row + c * 32, r);
+          ptx::tmem_ld_wait();
+          const int col0 = n_blk * BN + c * 32;
+          if (m < p.M) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              if (col0 + v * 8 < p.N) {
+                const uint4 o = make_uint4(
+                    pack_bf16x2(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1])),
+                    pack_bf16x2(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3])),
+                    pack_bf16x2(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5])),
+                    pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])));
+                *reinterpret_cast<uint4*>(drow + col0 + v * 8) = o;
+              }
+            }
+          }
+        }
+      } else {
+        // Row m of the tile is output row o = m of the weight; columns are input
+        // features.  ds[o,g] = sum_{j in g} G[o,j] * (q[o,j] - z[o,g]).
+        const int groups_per_row = p.in_features >> p.group_shift;
+        const int chunks_per_group = 1 << (p.group_shift - 5);
+        const uint8_t* qrow = p.Wq + (size_t)m * ((size_t)p.in_features * BITS / 8);
+        float acc_s = 0.0f, acc_g = 0.0f;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32(t_row + c * 32, r);
+          ptx::tmem_ld_wait();
+          const int col0 = n_blk * BN + c * 32;
+          if (m < p.M && col0 < p.N) {
+            uint32_t words[BITS];
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(qrow) + (size_t)(col0 >> 5) * BITS;
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) words[i] = __ldg(src + i);
+            uint32_t codes[32];
+            unpack32<BITS>(words, codes);
+            const int g = col0 >> p.group_shift;
+            const float zf = (float)__ldg(p.z8 + (size_t)m * groups_per_row + g);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float gv = __uint_as_float(r[i]);
+              acc_s = fmaf(gv, (float)codes[i] - zf, acc_s);
+              acc_g += gv;
+            }
+            if (((c + 1) & (chunks_per_group - 1)) == 0) {
+              const size_t idx = (size_t)m * groups_per_row + g;
+              p.ds[idx] = acc_s;
+              if (p.dz != nullptr) p.dz[idx] = -__half2float(__ushort_as_half(__ldg(p.s16 + idx))) * acc_g;
+              acc_s = 0.0f;
+              acc_g = 0.0f;
+            }
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[acc]));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  } else {
+    // ------------------------------------------------------------ dequantiser (PACKED only)
+    if constexpr (PACKED) {
+      const int t = threadIdx.x - kDeqWarp0 * 32;                 // 0..255, one 64-code unit per stage
+      const size_t pitch = (size_t)p.in_features * BITS / 8;      // bytes per packed row
+      const int groups_per_row = p.in_features >> p.group_shift;
+      const int chunks_in = p.in_features >> 6;                   // 64-code units per row
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      // unit -> (weight row, 64-code unit in the row, shared-memory row)
+      //   B K-major  (Y):  tile row n = t is weight row n0 + t, unit = kb
+      //   B MN-major (dX): k-row t/4 is weight row kb*64 + t/4, unit = n0/64 + t%4 (box t%4)
+      const int smem_row_off = B_MN ? ((t & 3) * (BK * 128) + (t >> 2) * 128) : t * 128;
+      const int rx = B_MN ? ((t >> 2) & 7) : (t & 7);
+      struct Unit {
+        uint32_t w[2 * BITS];
+        float s, z;
+        bool valid;
+      };
+      auto fetch = [&](Unit& u, int n_blk, int kb) {
+        const int wrow = B_MN ? kb * BK + (t >> 2) : n_blk * BN + t;
+        const int unit = B_MN ? n_blk * (BN / 64) + (t & 3) : kb;
+        u.valid = wrow < p.out_features && unit < chunks_in;
+        if (u.valid) {
+          load_codes64<BITS>(p.Wq + (size_t)wrow * pitch + (size_t)unit * (8 * BITS), u.w);
+          const size_t gi = (size_t)wrow * groups_per_row + ((unit << 6) >> p.group_shift);
+          u.s = __half2float(__ushort_as_half(__ldg(p.s16 + gi)));
+          u.z = (float)__ldg(p.z8 + gi);
+        }
+      };
+      Unit cur, nxt;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int m_blk, n_blk;
+        tile_coords(tile, num_m, num_n, m_blk, n_blk);
+        fetch(cur, n_blk, 0);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          // the next unit's loads fly while this one waits for its stage and is expanded
+          if (kb + 1 < num_kb) fetch(nxt, n_blk, kb + 1);
+          if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_DEQ_OPERAND_EMPTY)) {
+            ok = false;
+            break;
+          }
+          uint8_t* row = smem + stage * C::kStageBytes + C::kABytes + smem_row_off;
+          if (cur.valid) {
+            dequant_row64<BITS>(cur.w, cur.s, cur.z, row, rx);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) reinterpret_cast<uint4*>(row)[c] = make_uint4(0u, 0u, 0u, 0u);
+          }
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full[stage]));
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+          cur = nxt;
+        }
+      }
+    }
+  }
+
+  __syncwarp();
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, C::kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+  static EncodeFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeFn>(p);
+  }();
+  return fn;
+}
+
+// bf16 matrix [outer, inner] row-major; box = 64 elements (128 bytes) x box_outer rows, 128-byte swizzle.
+bool make_tmap(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer, uint32_t box_outer) {
+  EncodeFn enc = encode_fn();
+  if (enc == nullptr) return false;
+  const cuuint64_t dims[2] = {inner, outer};
+  const cuuint64_t strides[1] = {inner * 2};
+  const cuuint32_t box[2] = {64, box_outer};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = [] {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return v;
+  }();
+  return n;
+}
+
+template <int BN, bool A_MN, bool B_MN, bool PACKED, int EPI, int BITS>
+int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cudaStream_t st) {
+  using C = Cfg<BN, PACKED>;
+  auto kern = gemm_kernel<BN, A_MN, B_MN, PACKED, EPI, BITS>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
+    return EQAT_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return EQAT_ERR_CUDA;
+  const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
+  const int grid = tiles < sms ? tiles : sms;
+  kern<<<grid, C::kThreads, C::kSmemBytes, st>>>(ta, tb, p);
+  return launch_status();
+}
+
+int log2_exact(int v) {
+  int s = 0;
+  while ((1 << s) < v) ++s;
+  return s;
+}
+
+GemmParams base_params(int M, int N, int K) {
+  GemmParams p{};
+  p.M = M; p.N = N; p.K = K;
+  return p;
+}
+
+void set_weight(GemmParams& p, const eqat_desc& d, const uint8_t* Wq, const eqat_fp16* s16, const uint8_t* z8) {
+  p.Wq = Wq; p.s16 = s16; p.z8 = z8;
+  p.out_features = d.out_features;
+  p.in_features = d.in_features;
+  p.group_shift = log2_exact(d.group);
+}
+
+}  // namespace
+
+int launch_dense_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* What, eqat_bf16* Y, cudaStream_t st) {
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, X, d.in_features, d.tokens, BM) || !make_tmap(&tb, What, d.in_features, d.out_features, 256))
+    return EQAT_ERR_CUDA;
+  GemmParams p = base_params((int)d.tokens, d.out_features, d.in_features);
+  p.D = Y;
+  return launch<256, false, false, false, EPI_STORE, 2>(ta, tb, p, st);
+}
+
+int launch_dense_dx(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* What, eqat_bf16* dX, cudaStream_t st) {
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, dY, d.out_features, d.tokens, BM) || !make_tmap(&tb, What, d.in_features, d.out_features, BK))
+    return EQAT_ERR_CUDA;
+  GemmParams p = base_params((int)d.tokens, d.in_features, d.out_features);
+  p.D = dX;
+  return launch<256, false, true, false, EPI_STORE, 2>(ta, tb, p, st);
+}
+
+int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X, eqat_bf16* dWhat, cudaStream_t st) {
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, dY, d.out_features, d.tokens, BK) || !make_tmap(&tb, X, d.in_features, d.tokens, BK))
+    return EQAT_ERR_CUDA;
+  GemmParams p = base_params(d.out_features, d.in_features, (int)d.tokens);
+  p.D = dWhat;
+  return launch<256, true, true, false, EPI_STORE, 2>(ta, tb, p, st);
+}
+
+int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
+                      const uint8_t* z8, eqat_bf16* Y, cudaStream_t st) {
+  CUtensorMap ta;
+  if (!make_tmap(&ta, X, d.in_features, d.tokens, BM)) return EQAT_ERR_CUDA;
+  GemmParams p = base_params((int)d.tokens, d.out_features, d.in_features);
+  p.D = Y;
+  set_weight(p, d, Wq, s16, z8);
+  switch (d.bits) {
+    case 2: return launch<256, false, false, true, EPI_STORE, 2>(ta, ta, p, st);
+    case 3: return launch<256, false, false, true, EPI_STORE, 3>(ta, ta, p, st);
+    default: return launch<256, false, false, true, EPI_STORE, 4>(ta, ta, p, st);
+  }
+}
+
+int launch_packed_dx(const eqat_desc& d, const eqat_bf16* dY, const uint8_t* Wq, const eqat_fp16* s16,
+                     const uint8_t* z8, eqat_bf16* dX, cudaStream_t st) {
+  CUtensorMap ta;
+  if (!make_tmap(&ta, dY, d.out_features, d.tokens, BM)) return EQAT_ERR_CUDA;
+  GemmParams p = base_params((int)d.tokens, d.in_features, d.out_features);
+  p.D = dX;
+  set_weight(p, d, Wq, s16, z8);
+  switch (d.bits) {
+    case 2: return launch<256, false, true, true, EPI_STORE, 2>(ta, ta, p, st);
+    case 3: return launch<256, false, true, true, EPI_STORE, 3>(ta, ta, p, st);
+    default: return launch<256, false, true, true, EPI_STORE, 4>(ta, ta, p, st);
+  }
+}
+
+int launch_packed_ds(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* dY, const uint8_t* Wq,
+                     const uint8_t* z8, const eqat_fp16* s16, float* ds, float* dz, cudaStream_t st) {
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, dY, d.out_features, d.tokens, BK) || !make_tmap(&tb, X, d.in_features, d.tokens, BK))
+    return EQAT_ERR_CUDA;
+  GemmParams p = base_params(d.out_features, d.in_features, (int)d.tokens);
+  set_weight(p, d, Wq, s16, z8);
+  p.ds = ds;
+  p.dz = dz;
+  switch (d.bits) {
+    case 2: return launch<256, true, true, false, EPI_DS, 2>(ta, tb, p, st);
+    case 3: return launch<256, true, true, false, EPI_DS, 3>(ta, tb, p, st);
+    default: return launch<256, true, true, false, EPI_DS, 4>(ta, tb, p, st);
+  }
+}
+
+int read_device_status(int* status, int* detail) {
+  int h[2] = {0, 0};
+  if (cudaDeviceSynchronize() != cudaSuccess) return EQAT_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(h, g_device_status, sizeof(h)) != cudaSuccess) return EQAT_ERR_CUDA;
+  const int zero[2] = {0, 0};
+  if (cudaMemcpyToSymbol(g_device_status, zero, sizeof(zero)) != cudaSuccess) return EQAT_ERR_CUDA;
+  *status = h[0];
+  if (detail != nullptr) *detail = h[1];
+  return EQAT_OK;
+}
+
+}  // namespace eqat

@@ -1,0 +1,26 @@
+// Host launchers of the tcgen05 GEMM kernels (arguments already validated).
+#pragma once
+#include <cuda_runtime.h>
+#include "eqat.h"
+
+namespace eqat {
+
+// Y[T,out] = X[T,in] * What[out,in]^T
+int launch_dense_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* What, eqat_bf16* Y, cudaStream_t st);
+// dX[T,in] = dY[T,out] * What[out,in]
+int launch_dense_dx(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* What, eqat_bf16* dX, cudaStream_t st);
+// dWhat[out,in] = dY[T,out]^T * X[T,in]
+int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X, eqat_bf16* dWhat, cudaStream_t st);
+// Y = X * dequant(Wq)^T and dX = dY * dequant(Wq), codes expanded in shared memory
+int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
+                      const uint8_t* z8, eqat_bf16* Y, cudaStream_t st);
+int launch_packed_dx(const eqat_desc& d, const eqat_bf16* dY, const uint8_t* Wq, const eqat_fp16* s16,
+                     const uint8_t* z8, eqat_bf16* dX, cudaStream_t st);
+// ds (and optionally dz) reduced in the epilogue of dY^T * X
+int launch_packed_ds(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* dY, const uint8_t* Wq,
+                     const uint8_t* z8, const eqat_fp16* s16, float* ds, float* dz, cudaStream_t st);
+
+// Reads and clears the device status word ({status, wait site}); synchronises.
+int read_device_status(int* status, int* detail);
+
+}  // namespace eqat

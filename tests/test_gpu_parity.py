@@ -1,0 +1,282 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle.
+
+Integer outputs (codes, packed bytes, zero points, fp16 step sizes) must be
+bit-exact; floating-point outputs must be within 5e-3 relative Frobenius error
+of the oracle (bf16 inputs, fp32 accumulation on the GPU, fp64 in the oracle).
+"""
+import numpy as np
+import pytest
+import torch
+
+from helpers import TOL, bf16_round, bits_to_torch, f32, rel_err, torch_to_f64
+from oracle import eqat_oracle as O
+from workloads import CONFIGS, Config, Linear, activations_for, get_config, normal_bf16, to_bf16_bits, weight_for
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def eqat():
+    from paper_2407_11062_b200.build import build_library
+    build_library()
+    from paper_2407_11062_b200 import binding
+    return binding
+
+
+@pytest.fixture(autouse=True)
+def _device_status_clean(eqat):
+    yield
+    torch.cuda.synchronize()
+    assert eqat.device_status() == (0, 0)
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda()
+
+
+def small_cfg(name, out, in_f, bits, group, tokens, dist="normal", scale=0.02, outl=0.0):
+    return Config(name, (Linear("l", out, in_f, 1),), bits, group, tokens, ("block_ap", "e2e_qp"), dist, scale, outl)
+
+
+def variants(W32, bits, group):
+    """(name, s, z) triples: min/max initialisation, a shrunk step size (forces
+    clamping on both sides) and a shifted zero point."""
+    s, z = O.minmax_init(W32, bits, group)
+    Q = (1 << bits) - 1
+    yield "minmax", s, z
+    s2 = (s * np.float32(0.7)).astype(np.float32)
+    yield "shrunk", s2, z
+    yield "shifted", s, np.clip(z + 1, 0, Q).astype(np.float32)
+
+
+# --------------------------------------------------------------------------- element-wise kernels
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("group", [32, 64, 128, 256, 512])
+def test_minmax_fakequant_ste_pack(eqat, bits, group):
+    out, in_f = 192, 512                      # 98304 elements: several blocks and a ragged last block
+    cfg = small_cfg(f"ew_{bits}_{group}", out, in_f, bits, group, 0, "student_t4", 0.02, 0.01)
+    Wb = weight_for(cfg, cfg.linears[0]); W32 = f32(Wb)
+    d = eqat.make_desc(bits, group, out, in_f)
+    Wd = bits_to_torch(Wb)
+    ng = in_f // group
+
+    # min/max initialisation: bit-exact (binary32 arithmetic on both sides)
+    s_o, z_o = O.minmax_init(W32, bits, group)
+    s_g = torch.empty(out, ng, device="cuda"); z_g = torch.empty(out, ng, device="cuda")
+    eqat.eqat_minmax_init(d, Wd, s_g, z_g)
+    assert np.array_equal(s_g.cpu().numpy(), s_o)
+    assert np.array_equal(z_g.cpu().numpy(), z_o)
+
+    Gb = normal_bf16((out, in_f), 1e-2, cfg.name, "G"); G32 = f32(Gb); Gd = bits_to_torch(Gb)
+    for name, s, z in variants(W32, bits, group):
+        sd, zd = dev(s), dev(z)
+        q_o, _, p_o = O.quantize_codes(W32, s, z, bits, group)
+        if name == "shrunk":
+            assert (p_o < 0).any() and (p_o > (1 << bits) - 1).any()       # both clamped branches are exercised
+        if name == "shifted":
+            assert (p_o > (1 << bits) - 1).any()
+        # quantise + pack: bit-exact codes, zero points, fp16 step sizes
+        P = torch.empty(out, in_f * bits // 8, dtype=torch.uint8, device="cuda")
+        z8 = torch.empty(out, ng, dtype=torch.uint8, device="cuda")
+        s16 = torch.empty(out, ng, dtype=torch.float16, device="cuda")
+        eqat.eqat_quantize_pack(d, Wd, sd, zd, P, z8, s16)
+        P_o, z8_o, s16_o = O.quantize_pack(W32, s, z, bits, group)
+        assert np.array_equal(P.cpu().numpy(), P_o), name
+        assert np.array_equal(z8.cpu().numpy(), z8_o)
+        assert np.array_equal(s16.cpu().numpy().view(np.uint16), s16_o.view(np.uint16))
+        # unpack / pack round trip against the oracle's codes
+        codes = torch.empty(out, in_f, dtype=torch.uint8, device="cuda")
+        eqat.eqat_unpack(d, P, codes)
+        assert np.array_equal(codes.cpu().numpy(), q_o.astype(np.uint8))
+        P2 = torch.empty_like(P)
+        eqat.eqat_pack(d, dev(q_o.astype(np.uint8)), P2)
+        assert np.array_equal(P2.cpu().numpy(), P_o)
+        # fake quantiser
+        What = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
+        eqat.eqat_fakequant_weight(d, Wd, sd, zd, What)
+        What_o = O.dequantize(q_o, s, z, group)
+        assert rel_err(torch_to_f64(What), What_o) <= TOL
+        # the GPU value is the oracle's rounded to bf16, up to one bf16 ulp where the
+        # fp32 product sits next to a rounding boundary
+        ulp = np.abs(What_o) * 2.0 ** -7 + 1e-30
+        assert (np.abs(torch_to_f64(What) - What_o) <= ulp).all()
+        # STE backward, both readings of Eq. 4
+        for dz_mode in (0, 1):
+            dd = eqat.make_desc(bits, group, out, in_f, 0, dz_mode)
+            dW = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
+            ds = torch.empty(out, ng, device="cuda"); dz = torch.empty(out, ng, device="cuda")
+            eqat.eqat_ste_bwd(dd, Gd, Wd, sd, zd, dW, ds, dz)
+            dW_o, ds_o, dz_o = O.ste_bwd(G32, W32, s, z, bits, group, dz_mode)
+            assert np.array_equal(torch_to_f64(dW), dW_o)            # a masked copy: exact
+            assert rel_err(torch_to_f64(ds), ds_o) <= TOL, (name, dz_mode)
+            if np.linalg.norm(dz_o) > 0:
+                assert rel_err(torch_to_f64(dz), dz_o) <= TOL, (name, dz_mode)
+            else:
+                assert not torch_to_f64(dz).any()
+        ds_only = torch.empty(out, ng, device="cuda")
+        eqat.eqat_ste_bwd(d, Gd, Wd, sd, zd, dW, ds_only, None)      # dz is optional
+        _, ds_o, _ = O.ste_bwd(G32, W32, s, z, bits, group, 0)
+        assert rel_err(torch_to_f64(ds_only), ds_o) <= TOL
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_zero_point_stream(eqat, bits):
+    out, in_f, group = 64, 512, 64
+    d = eqat.make_desc(bits, group, out, in_f)
+    z = np.random.default_rng(bits).integers(0, 1 << bits, out * in_f // group).astype(np.uint8)
+    zp = torch.empty(z.size * bits // 8, dtype=torch.uint8, device="cuda")
+    eqat.eqat_pack_zeros(d, dev(z), zp)
+    assert np.array_equal(zp.cpu().numpy(), O.pack_stream(z, bits))
+    back = torch.empty(z.size, dtype=torch.uint8, device="cuda")
+    eqat.eqat_unpack_zeros(d, zp, back)
+    assert np.array_equal(back.cpu().numpy(), z)
+
+
+def test_fractional_zero_point_is_rounded(eqat):
+    out, in_f, bits, group = 64, 128, 2, 64
+    cfg = small_cfg("fracz", out, in_f, bits, group, 0)
+    Wb = weight_for(cfg, cfg.linears[0]); W32 = f32(Wb)
+    s, z = O.minmax_init(W32, bits, group)
+    zf = (z + np.float32(0.3)).astype(np.float32)
+    d = eqat.make_desc(bits, group, out, in_f)
+    A = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda"); B = torch.empty_like(A)
+    eqat.eqat_fakequant_weight(d, bits_to_torch(Wb), dev(s), dev(z), A)
+    eqat.eqat_fakequant_weight(d, bits_to_torch(Wb), dev(s), dev(zf), B)
+    assert torch.equal(A, B)
+
+
+# --------------------------------------------------------------------------- Block-AP layer
+def run_block_ap(eqat, cfg, lin, tokens, s, z, dz_mode=0):
+    Wb = weight_for(cfg, lin); Xb, dYb = activations_for(cfg, lin, tokens)
+    out, in_f, ng = lin.out_features, lin.in_features, lin.in_features // cfg.group
+    d = eqat.make_desc(cfg.bits, cfg.group, out, in_f, tokens, dz_mode)
+    Wd, Xd, dYd, sd, zd = bits_to_torch(Wb), bits_to_torch(Xb), bits_to_torch(dYb), dev(s), dev(z)
+    Y = torch.empty(tokens, out, dtype=torch.bfloat16, device="cuda")
+    What = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
+    eqat.qlinear_fakequant_fwd(d, Xd, Wd, sd, zd, Y, What)
+    dX = torch.empty(tokens, in_f, dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
+    ds = torch.empty(out, ng, device="cuda"); dz = torch.empty(out, ng, device="cuda")
+    ws = torch.empty(eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD), dtype=torch.uint8, device="cuda")
+    eqat.qlinear_fakequant_bwd(d, Xd, dYd, Wd, sd, zd, What, dX, dW, ds, dz, ws)
+    torch.cuda.synchronize()
+    return dict(W=f32(Wb), X=f32(Xb), dY=f32(dYb), Y=Y, What=What, dX=dX, dW=dW, ds=ds, dz=dz)
+
+
+def check_block_ap(r, s, z, bits, group, dz_mode=0):
+    What_o = O.fake_quant_weight(r["W"], s, z, bits, group)
+    assert rel_err(torch_to_f64(r["What"]), What_o) <= TOL
+    assert rel_err(torch_to_f64(r["Y"]), O.linear_fwd(r["X"], What_o)) <= TOL
+    assert rel_err(torch_to_f64(r["dX"]), O.linear_bwd_dx(r["dY"], What_o)) <= TOL
+    G = O.weight_grad(r["dY"], r["X"])
+    dW_o, ds_o, dz_o = O.ste_bwd(G, r["W"], s, z, bits, group, dz_mode)
+    assert rel_err(torch_to_f64(r["dW"]), dW_o) <= TOL
+    assert rel_err(torch_to_f64(r["ds"]), ds_o) <= TOL
+    if np.linalg.norm(dz_o) > 0:
+        assert rel_err(torch_to_f64(r["dz"]), dz_o) <= TOL
+    else:
+        assert not torch_to_f64(r["dz"]).any()
+
+
+def test_block_ap_config1(eqat):
+    cfg = get_config("c1"); lin = cfg.linears[0]
+    W32 = f32(weight_for(cfg, lin))
+    for name, s, z in variants(W32, cfg.bits, cfg.group):
+        for dz_mode in (0, 1):
+            r = run_block_ap(eqat, cfg, lin, cfg.tokens, s, z, dz_mode)
+            check_block_ap(r, s, z, cfg.bits, cfg.group, dz_mode)
+
+
+@pytest.mark.parametrize("out,in_f,tokens,bits,group", [
+    (192, 384, 300, 4, 128),        # ragged in every dimension: 2 row tiles with a tail, 1.5 column tiles
+    (64, 128, 1, 2, 64),            # a single token, a single K block pair
+    (320, 640, 129, 3, 128),        # one row past a tile boundary
+    (1024, 256, 520, 2, 256),
+])
+def test_block_ap_ragged(eqat, out, in_f, tokens, bits, group):
+    cfg = small_cfg(f"rag_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens, "student_t4", 0.02, 0.01)
+    lin = cfg.linears[0]
+    s, z = O.minmax_init(f32(weight_for(cfg, lin)), bits, group)
+    s = (s * np.float32(0.8)).astype(np.float32)
+    r = run_block_ap(eqat, cfg, lin, tokens, s, z)
+    check_block_ap(r, s, z, bits, group)
+
+
+def test_block_ap_is_deterministic(eqat):
+    cfg = get_config("c1"); lin = cfg.linears[0]
+    s, z = O.minmax_init(f32(weight_for(cfg, lin)), cfg.bits, cfg.group)
+    a = run_block_ap(eqat, cfg, lin, cfg.tokens, s, z)
+    b = run_block_ap(eqat, cfg, lin, cfg.tokens, s, z)
+    for k in ("Y", "What", "dX", "dW", "ds", "dz"):
+        assert torch.equal(a[k], b[k]), k
+
+
+# --------------------------------------------------------------------------- E2E-QP layer
+def run_e2e(eqat, cfg, lin, tokens, with_dz=True, fp16_steps=False):
+    """Hand-off (quantise + pack on the oracle's side) then the three packed-weight calls."""
+    Wb = weight_for(cfg, lin); W32 = f32(Wb)
+    Xb, dYb = activations_for(cfg, lin, tokens)
+    out, in_f, ng = lin.out_features, lin.in_features, lin.in_features // cfg.group
+    s, z = O.minmax_init(W32, cfg.bits, cfg.group)
+    if fp16_steps:
+        s = s.astype(np.float16).astype(np.float32)
+    P_o, z8_o, s16_o = O.quantize_pack(W32, s, z, cfg.bits, cfg.group)
+    d = eqat.make_desc(cfg.bits, cfg.group, out, in_f, tokens)
+    Pd, z8d = dev(P_o), dev(z8_o)
+    s16d = torch.from_numpy(s16_o.view(np.int16)).view(torch.float16).cuda()
+    Xd, dYd = bits_to_torch(Xb), bits_to_torch(dYb)
+    Y = torch.empty(tokens, out, dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty(tokens, in_f, dtype=torch.bfloat16, device="cuda")
+    ds = torch.empty(out, ng, device="cuda")
+    dz = torch.empty(out, ng, device="cuda") if with_dz else None
+    eqat.qlinear_packed_fwd(d, Xd, Pd, s16d, z8d, Y)
+    eqat.qlinear_packed_bwd_dx(d, dYd, Pd, s16d, z8d, dX)
+    eqat.qlinear_packed_bwd_ds(d, Xd, dYd, Pd, z8d, s16d, ds, dz)
+    torch.cuda.synchronize()
+    q = O.unpack_rows(P_o, cfg.bits, in_f)
+    return dict(X=f32(Xb), dY=f32(dYb), q=q, z8=z8_o, s16=s16_o.astype(np.float32), Y=Y, dX=dX, ds=ds, dz=dz,
+                W=W32, s=s, z=z)
+
+
+def check_e2e(r, group):
+    What_o = O.dequantize(r["q"], r["s16"], r["z8"], group)
+    assert rel_err(torch_to_f64(r["Y"]), O.linear_fwd(r["X"], What_o)) <= TOL
+    assert rel_err(torch_to_f64(r["dX"]), O.linear_bwd_dx(r["dY"], What_o)) <= TOL
+    assert rel_err(torch_to_f64(r["ds"]), O.e2e_ds(r["dY"], r["X"], r["q"], r["z8"], group)) <= TOL
+    if r["dz"] is not None:
+        assert rel_err(torch_to_f64(r["dz"]), O.e2e_dz(r["dY"], r["X"], r["s16"], group)) <= TOL
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("group", [64, 128, 256])
+def test_e2e_small(eqat, bits, group):
+    cfg = small_cfg(f"e2e_{bits}_{group}", 512, 512, bits, group, 256, "student_t4", 0.02, 0.01)
+    check_e2e(run_e2e(eqat, cfg, cfg.linears[0], 256), group)
+
+
+@pytest.mark.parametrize("out,in_f,tokens,bits,group", [
+    (192, 384, 300, 2, 64),
+    (64, 128, 1, 4, 128),
+    (320, 640, 129, 3, 128),
+    (1024, 256, 520, 2, 64),
+])
+def test_e2e_ragged(eqat, out, in_f, tokens, bits, group):
+    cfg = small_cfg(f"e2er_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens)
+    check_e2e(run_e2e(eqat, cfg, cfg.linears[0], tokens, with_dz=(bits != 4)), group)
+
+
+def test_e2e_is_deterministic_and_matches_block_ap_forward(eqat):
+    """Packed forward == fake-quant forward when s is representable in fp16."""
+    cfg = small_cfg("cross", 512, 512, 2, 64, 256)
+    lin = cfg.linears[0]
+    a = run_e2e(eqat, cfg, lin, 256, fp16_steps=True)
+    b = run_e2e(eqat, cfg, lin, 256, fp16_steps=True)
+    for k in ("Y", "dX", "ds", "dz"):
+        assert torch.equal(a[k], b[k]), k
+    assert np.array_equal(a["s"], a["s16"])       # the step sizes survive the fp16 hand-off unchanged
+    r = run_block_ap(eqat, cfg, lin, 256, a["s"], a["z"])
+    assert rel_err(torch_to_f64(r["Y"]), torch_to_f64(a["Y"])) <= 2e-3
+    assert rel_err(torch_to_f64(r["dX"]), torch_to_f64(a["dX"])) <= 2e-3

@@ -1,0 +1,81 @@
+"""The shared library loads without a GPU, exports every symbol the header
+declares, and rejects bad arguments on the host before launching anything."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def eqat():
+    from paper_2407_11062_b200.build import build_library
+    build_library()
+    from paper_2407_11062_b200 import binding
+    return binding
+
+
+def _declared():
+    src = open(os.path.join(ROOT, "include", "eqat.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b((?:eqat|qlinear)_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_every_declared_symbol_is_exported(eqat):
+    names = _declared()
+    assert len(names) >= 17
+    raw = ctypes.CDLL(eqat.LIB_PATH)
+    for n in names:
+        assert hasattr(raw, n), n
+        assert hasattr(eqat, n) or hasattr(eqat.lib, n)
+
+
+def test_status_strings(eqat):
+    assert eqat.status_string(0) == "ok"
+    seen = {eqat.status_string(s) for s in range(-7, 1)}
+    assert len(seen) == 8
+    assert eqat.lib.eqat_version() >= 100
+
+
+def test_workspace_sizes(eqat):
+    d = eqat.make_desc(2, 64, 512, 512, 256)
+    assert eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD) == 512 * 512 * 2
+    assert eqat.workspace_bytes(d, eqat.EQAT_OP_PACKED_BWD_DS) == 0
+    with pytest.raises(eqat.EqatError):
+        eqat.workspace_bytes(d, 99)
+
+
+@pytest.mark.parametrize("kw,status", [
+    (dict(bits=5), -4), (dict(bits=1), -4), (dict(group=48), -2), (dict(group=96), -2), (dict(in_features=500), -2),
+    (dict(out_features=0), -2), (dict(dz_mode=2), -4), (dict(group=1024), -2),
+])
+def test_bad_descriptors_are_rejected_on_the_host(eqat, kw, status):
+    base = dict(bits=2, group=64, out_features=512, in_features=512, tokens=256, dz_mode=0)
+    base.update(kw)
+    d = eqat.make_desc(**base)
+    fake = ctypes.c_void_p(0x1000)       # never dereferenced: validation fails first
+    rc = eqat.lib.eqat_fakequant_weight(ctypes.byref(d), fake, fake, fake, fake, None)
+    assert rc == status
+
+
+def test_null_and_misaligned_pointers(eqat):
+    d = eqat.make_desc(2, 64, 512, 512, 256)
+    ok, odd = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1004)
+    assert eqat.lib.eqat_fakequant_weight(ctypes.byref(d), ok, ok, None, ok, None) == eqat.EQAT_ERR_NULL
+    assert eqat.lib.eqat_fakequant_weight(ctypes.byref(d), ok, odd, ok, ok, None) == eqat.EQAT_ERR_ALIGN
+    assert eqat.lib.eqat_fakequant_weight(None, ok, ok, ok, ok, None) == eqat.EQAT_ERR_NULL
+    assert eqat.lib.qlinear_packed_fwd(ctypes.byref(d), ok, ok, ok, ok, None, None) == eqat.EQAT_ERR_NULL
+    # packed GEMMs accept group 64/128/256 only; GEMMs need tokens > 0 and out % 64 == 0
+    d32 = eqat.make_desc(2, 32, 512, 512, 256)
+    assert eqat.lib.qlinear_packed_fwd(ctypes.byref(d32), ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_UNSUPPORTED
+    d0 = eqat.make_desc(2, 64, 512, 512, 0)
+    assert eqat.lib.qlinear_packed_fwd(ctypes.byref(d0), ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_SHAPE
+    d96 = eqat.make_desc(2, 64, 96, 512, 256)
+    assert eqat.lib.qlinear_fakequant_fwd(ctypes.byref(d96), ok, ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_SHAPE
+    # workspace: missing, too small, misaligned
+    args = [ok] * 10
+    assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(d), *args, None, 0, None) == eqat.EQAT_ERR_WORKSPACE
+    assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(d), *args, ok, 16, None) == eqat.EQAT_ERR_WORKSPACE
+    assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(d), *args, ctypes.c_void_p(0x1010), 1 << 20, None) == eqat.EQAT_ERR_WORKSPACE
