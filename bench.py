@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the quantised-linear hot path on the Llama-2-7B w2g64 block workload.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+One step = one pass of the whole path over the seven linear layers of a
+Llama-2-7B decoder block at 2 bits, group 64:
+    min/max init, Block-AP forward and backward at 4096 tokens (batch 2 x 2048),
+    hand-off (quantise + pack, unpack), E2E-QP forward / dX / ds at 16384 tokens.
+Prints one JSON line (rank 0).  `value` is the tensor-core throughput of the six
+contractions per linear (2*T*in*out flop each) over the whole step, all kernels
+included in the time; dequantisation, STE and epilogue arithmetic are not counted
+as flops.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from workloads import LINEARS
+
+BITS, GROUP = 2, 64
+T_BLOCK_AP, T_E2E = 4096, 16384
+WORKLOAD = "llama2-7b decoder-block linears, w2g64: Block-AP fwd+bwd @4096 tok, hand-off, E2E-QP fwd/dX/ds @16384 tok"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["source"] = "fallback"
+    return d
+
+
+def step_flops(t_block_ap=T_BLOCK_AP, t_e2e=T_E2E):
+    per_token = sum(2 * l.in_features * l.out_features * l.count for l in LINEARS["7b"])
+    return 3 * per_token * t_block_ap, 3 * per_token * t_e2e
+
+
+# ----------------------------------------------------------------------------- distributed plumbing
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def max_over_ranks(value: float, device) -> float:
+    """Largest value over all ranks (the slowest rank defines the step time)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- the workload on one GPU
+class BlockWorkload:
+    """Device buffers for the seven linears; activations shared per shape, weights per linear."""
+
+    def __init__(self, eqat, device, seed, t_block_ap=T_BLOCK_AP, t_e2e=T_E2E):
+        self.eqat, self.device = eqat, device
+        self.t_ap, self.t_e2e = t_block_ap, t_e2e
+        g = torch.Generator(device=device); g.manual_seed(seed)
+        bf, dev = torch.bfloat16, device
+        self.shapes, self.layers = {}, []
+        for lin in LINEARS["7b"]:
+            out, in_f, ng = lin.out_features, lin.in_features, lin.in_features // GROUP
+            sh = dict(lin=lin,
+                      X=torch.randn(t_e2e, in_f, generator=g, device=dev, dtype=torch.float32).to(bf),
+                      dY=(torch.randn(t_e2e, out, generator=g, device=dev, dtype=torch.float32) * 1e-2).to(bf),
+                      Y=torch.empty(t_e2e, out, dtype=bf, device=dev), dX=torch.empty(t_e2e, in_f, dtype=bf, device=dev),
+                      What=torch.empty(out, in_f, dtype=bf, device=dev), dW=torch.empty(out, in_f, dtype=bf, device=dev),
+                      ds=torch.empty(out, ng, device=dev), dz=torch.empty(out, ng, device=dev),
+                      ds2=torch.empty(out, ng, device=dev),
+                      codes=torch.empty(out, in_f, dtype=torch.uint8, device=dev),
+                      d_ap=eqat.make_desc(BITS, GROUP, out, in_f, t_block_ap), d_e2e=eqat.make_desc(BITS, GROUP, out, in_f, t_e2e))
+            sh["ws"] = torch.empty(eqat.workspace_bytes(sh["d_ap"], eqat.EQAT_OP_FAKEQUANT_BWD), dtype=torch.uint8, device=dev)
+            self.shapes[lin.name] = sh
+            for i in range(lin.count):
+                W = (torch.randn(out, in_f, generator=g, device=dev, dtype=torch.float32) * 0.02).to(bf)
+                self.layers.append(dict(shape=lin.name, W=W,
+                                        s=torch.empty(out, ng, device=dev), z=torch.empty(out, ng, device=dev),
+                                        P=torch.empty(out, in_f * BITS // 8, dtype=torch.uint8, device=dev),
+                                        z8=torch.empty(out, ng, dtype=torch.uint8, device=dev),
+                                        s16=torch.empty(out, ng, dtype=torch.float16, device=dev)))
+        self.calls_per_step = 8 * len(self.layers)
+        self.kernels_per_step = 11 * len(self.layers)     # fwd = 2 kernels, bwd = 3, the other six calls 1 each
+
+    def step(self, timers=None):
+        e = self.eqat
+        def timed(name, fn):
+            if timers is None:
+                fn(); return
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            timers.setdefault(name, []).append((a, b))
+        for L in self.layers:
+            S = self.shapes[L["shape"]]
+            Xa, dYa, Ya, dXa = S["X"][: self.t_ap], S["dY"][: self.t_ap], S["Y"][: self.t_ap], S["dX"][: self.t_ap]
+            tag = L["shape"]
+            timed("minmax_init/" + tag, lambda: e.eqat_minmax_init(S["d_ap"], L["W"], L["s"], L["z"]))
+            timed("fakequant_fwd/" + tag, lambda: e.qlinear_fakequant_fwd(S["d_ap"], Xa, L["W"], L["s"], L["z"], Ya, S["What"]))
+            timed("fakequant_bwd/" + tag, lambda: e.qlinear_fakequant_bwd(S["d_ap"], Xa, dYa, L["W"], L["s"], L["z"], S["What"],
+                                                                            dXa, S["dW"], S["ds"], S["dz"], S["ws"]))
+            timed("quantize_pack/" + tag, lambda: e.eqat_quantize_pack(S["d_ap"], L["W"], L["s"], L["z"], L["P"], L["z8"], L["s16"]))
+            timed("unpack/" + tag, lambda: e.eqat_unpack(S["d_ap"], L["P"], S["codes"]))
+            timed("packed_fwd/" + tag, lambda: e.qlinear_packed_fwd(S["d_e2e"], S["X"], L["P"], L["s16"], L["z8"], S["Y"]))
+            timed("packed_bwd_dx/" + tag, lambda: e.qlinear_packed_bwd_dx(S["d_e2e"], S["dY"], L["P"], L["s16"], L["z8"], S["dX"]))
+            timed("packed_bwd_ds/" + tag, lambda: e.qlinear_packed_bwd_ds(S["d_e2e"], S["X"], S["dY"], L["P"], L["z8"], L["s16"], S["ds2"]))
+
+
+class HostStaging:
+    """Pinned host copies of each shape's activations and gradient outputs for the end-to-end leg."""
+
+    def __init__(self, wl: BlockWorkload):
+        self.wl = wl
+        self.host = {}
+        for name, S in wl.shapes.items():
+            self.host[name] = dict(
+                X=S["X"].cpu().pin_memory(), dY=S["dY"].cpu().pin_memory(),
+                dW=torch.empty(S["dW"].shape, dtype=S["dW"].dtype).pin_memory(),
+                ds=torch.empty(S["ds"].shape).pin_memory(), dz=torch.empty(S["dz"].shape).pin_memory(),
+                ds2=torch.empty(S["ds2"].shape).pin_memory())
+        self.h2d = sum(self.host[L["shape"]]["X"].nbytes + self.host[L["shape"]]["dY"].nbytes for L in wl.layers)
+        self.d2h = sum(sum(self.host[L["shape"]][k].nbytes for k in ("dW", "ds", "dz", "ds2")) for L in wl.layers)
+
+    def step(self):
+        wl, e = self.wl, self.wl.eqat
+        for L in wl.layers:
+            S, H = wl.shapes[L["shape"]], self.host[L["shape"]]
+            S["X"].copy_(H["X"], non_blocking=True)
+            S["dY"].copy_(H["dY"], non_blocking=True)
+            Xa, dYa, Ya, dXa = S["X"][: wl.t_ap], S["dY"][: wl.t_ap], S["Y"][: wl.t_ap], S["dX"][: wl.t_ap]
+            e.eqat_minmax_init(S["d_ap"], L["W"], L["s"], L["z"])
+            e.qlinear_fakequant_fwd(S["d_ap"], Xa, L["W"], L["s"], L["z"], Ya, S["What"])
+            e.qlinear_fakequant_bwd(S["d_ap"], Xa, dYa, L["W"], L["s"], L["z"], S["What"], dXa, S["dW"], S["ds"], S["dz"], S["ws"])
+            e.eqat_quantize_pack(S["d_ap"], L["W"], L["s"], L["z"], L["P"], L["z8"], L["s16"])
+            e.eqat_unpack(S["d_ap"], L["P"], S["codes"])
+            e.qlinear_packed_fwd(S["d_e2e"], S["X"], L["P"], L["s16"], L["z8"], S["Y"])
+            e.qlinear_packed_bwd_dx(S["d_e2e"], S["dY"], L["P"], L["s16"], L["z8"], S["dX"])
+            e.qlinear_packed_bwd_ds(S["d_e2e"], S["X"], S["dY"], L["P"], L["z8"], L["s16"], S["ds2"])
+            for k in ("dW", "ds", "dz", "ds2"):
+                H[k].copy_(S[k], non_blocking=True)
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(seed=0):
+    """The oracle on a bounded sample of the same workload: the 4096x4096 linear,
+    element-wise steps on 512 output rows, contractions on 256 token rows x 512
+    output rows.  Returns (flops counted the same way, seconds, description)."""
+    from oracle import eqat_oracle as O
+    from workloads import from_bf16_bits, get_config, normal_bf16
+    rows, toks, in_f = 512, 256, 4096
+    Wb = normal_bf16((rows, in_f), 0.02, "bench_oracle", seed, "W")
+    Xb = normal_bf16((toks, in_f), 1.0, "bench_oracle", seed, "X")
+    dYb = normal_bf16((toks, rows), 1e-2, "bench_oracle", seed, "dY")
+    W, X, dY = from_bf16_bits(Wb), from_bf16_bits(Xb), from_bf16_bits(dYb)
+    t0 = time.perf_counter()
+    s, z = O.minmax_init(W, BITS, GROUP)
+    What = O.fake_quant_weight(W, s, z, BITS, GROUP)
+    Y = O.linear_fwd(X, What); dX = O.linear_bwd_dx(dY, What)
+    G = O.weight_grad(dY, X)
+    O.ste_bwd(G, W, s, z, BITS, GROUP)
+    P, z8, s16 = O.quantize_pack(W, s, z, BITS, GROUP)
+    q = O.unpack_rows(P, BITS, in_f)
+    Wq = O.dequantize(q, s16.astype(np.float32), z8, GROUP)
+    O.linear_fwd(X, Wq); O.linear_bwd_dx(dY, Wq)
+    O.e2e_ds(dY, X, q, z8, GROUP)
+    dt = time.perf_counter() - t0
+    flops = 6 * 2 * toks * in_f * rows
+    return flops, dt, f"4096-wide linear, {rows} output rows x {toks} tokens, all steps of the path (w2g64)"
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(budget_s=15.0):
+    flops, dt, what = oracle_sample(0)
+    reps, total_f, total_t = 1, flops, dt
+    while total_t < budget_s and reps < 64:
+        f, t, _ = oracle_sample(reps)
+        total_f += f; total_t += t; reps += 1
+    return {"value": total_f / total_t / 1e12, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle",
+            "sample": f"{reps} x ({what}); {total_t:.1f} s of CPU time"}
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    times, flops = [], 0
+    for i in range(args.warmup + args.steps):
+        f, t, what = oracle_sample(i)
+        if i >= args.warmup:
+            times.append(t); flops = f
+    ms = 1e3 * sum(times) / len(times)
+    val = flops / (ms * 1e-3) / 1e12
+    out = {"impl": "reference", "metric": "QLinear fwd+bwd TFLOP/s", "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": WORKLOAD, "step": "bounded sample: " + what},
+           "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle", "sample": what},
+           "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+# ----------------------------------------------------------------------------- main
+def summarise(timers):
+    out = {}
+    for name, pairs in timers.items():
+        ms = [a.elapsed_time(b) for a, b in pairs]
+        out[name] = {"launches": len(ms), "avg_ms": sum(ms) / len(ms), "total_ms": sum(ms)}
+    return out
+
+
+def run_ours(args):
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2407_11062_b200.build import build_library
+    build_library()
+    from paper_2407_11062_b200 import binding as eqat
+    peaks = load_peaks()
+
+    wl = BlockWorkload(eqat, device, seed=20240711 + rank)     # each rank: its own token batch (weak scaling)
+    for _ in range(max(args.warmup, 3)):
+        wl.step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    timers = {}
+    barrier(); torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        wl.step(timers)
+    t1.record()
+    torch.cuda.synchronize(); barrier()
+    ms_local = t0.elapsed_time(t1) / args.steps
+    ms = max_over_ranks(ms_local, device)
+    clocks = sampler.stop() if rank == 0 else None
+    st = eqat.device_status()
+    if st != (0, 0):
+        raise SystemExit(f"device status {st}: a kernel abandoned a wait")
+
+    # end-to-end leg: host buffers in, gradients out, copies inside the timed region
+    stage = HostStaging(wl)
+    e2e_steps = max(1, min(args.steps, 3))
+    stage.step(); torch.cuda.synchronize(); barrier()
+    t0.record()
+    for _ in range(e2e_steps):
+        stage.step()
+    t1.record()
+    torch.cuda.synchronize(); barrier()
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1) / e2e_steps, device)
+
+    f_ap, f_e2e = step_flops()
+    flops = (f_ap + f_e2e) * world
+    if rank == 0:
+        kern = summarise(timers)
+        by_class = {}
+        for name, v in kern.items():
+            c = name.split("/")[0]
+            by_class.setdefault(c, 0.0)
+            by_class[c] += v["total_ms"]
+        top_class = max(by_class, key=by_class.get)
+        # roofline of the dominant kernel (each packed_* call is exactly one kernel launch)
+        t_tok = {"packed_fwd": T_E2E, "packed_bwd_dx": T_E2E, "packed_bwd_ds": T_E2E}
+        roof = None
+        if top_class in t_tok:
+            tot_f = sum(2 * T_E2E * l.in_features * l.out_features * l.count for l in LINEARS["7b"]) * args.steps
+            tot_ms = by_class[top_class]
+            ach = tot_f / (tot_ms * 1e-3) / 1e12
+            peak = peaks["bf16_tflops_sustained"]
+            roof = {"kernel": "gemm_kernel (" + top_class + ")", "bound": "tensor", "achieved": ach, "peak": peak,
+                    "unit": "TFLOP/s", "frac": ach / peak, "peak_source": peaks["source"] + " (sustained)", "traffic": None}
+        classes = {c: {"total_ms_per_step": t / args.steps, "share": t / sum(by_class.values())} for c, t in by_class.items()}
+        out = {"metric": "QLinear fwd+bwd TFLOP/s", "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": world,
+               "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+               "config": {"workload": WORKLOAD, "bits": BITS, "group": GROUP, "tokens_block_ap": T_BLOCK_AP, "tokens_e2e_qp": T_E2E,
+                          "l2": "inputs larger than L2 (working set > 2 GB per shape, weights per linear)"},
+               "pct_of_bf16_peak": 100.0 * flops / world / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+               "block_tokens_per_s": {"block_ap": None, "e2e_qp": None},
+               "roofline": roof, "kernel_classes": classes, "clocks": clocks,
+               "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                       "h2d_bytes_per_step": stage.h2d, "d2h_bytes_per_step": stage.d2h},
+               "gpu_launches": wl.kernels_per_step * args.steps}
+        ap_ms = sum(by_class.get(c, 0.0) for c in ("fakequant_fwd", "fakequant_bwd")) / args.steps
+        qp_ms = sum(by_class.get(c, 0.0) for c in ("packed_fwd", "packed_bwd_dx", "packed_bwd_ds")) / args.steps
+        out["block_tokens_per_s"] = {"block_ap": world * T_BLOCK_AP / (ap_ms * 1e-3), "e2e_qp": world * T_E2E / (qp_ms * 1e-3)}
+        out["tflops_by_mode"] = {"block_ap": f_ap / (ap_ms * 1e-3) / 1e12, "e2e_qp": f_e2e / (qp_ms * 1e-3) / 1e12}
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline()
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
