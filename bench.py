@@ -382,15 +382,40 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_kernel_case(args):
+    """One call class on one linear shape, a few launches: the small case used for ncu captures."""
+    torch.cuda.set_device(0)
+    from paper_2407_11062_b200.build import build_library
+    build_library()
+    from paper_2407_11062_b200 import binding as eqat
+    wl = BlockWorkload(eqat, torch.device("cuda", 0), seed=1, t_block_ap=args.case_tokens, t_e2e=args.case_tokens)
+    wl.layers = [L for L in wl.layers if L["shape"] == args.case_shape][:1]
+    for _ in range(2):
+        wl.step()                       # fills s, z, packed codes
+    torch.cuda.synchronize()
+    timers = {}
+    for _ in range(args.case_iters):
+        wl.step(timers)
+    torch.cuda.synchronize()
+    assert eqat.device_status() == (0, 0)
+    print(json.dumps({k: v for k, v in summarise(timers).items()}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--kernel-case", action="store_true", help="run one linear shape a few times (for profilers)")
+    ap.add_argument("--case-shape", default="qkvo", choices=[l.name for l in LINEARS["7b"]])
+    ap.add_argument("--case-tokens", type=int, default=16384)
+    ap.add_argument("--case-iters", type=int, default=2)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.kernel_case:
+        run_kernel_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
