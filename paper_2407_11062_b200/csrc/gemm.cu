@@ -9,14 +9,16 @@
 //     dX   = dY * W_hat   : A = dY [T,out] K-major,  B = W_hat [out,in] MN-major
 //     dW^  = dY^T * X     : A = dY [T,out] MN-major, B = X     [T,in]  MN-major
 //
-// Roles inside a CTA (one CTA per SM, 128 x BN output tile, 64-deep K blocks):
+// Roles inside a CTA (one CTA per SM, (MT*128) x BN output tile, 64-deep K blocks;
+// MT = 1 with two TMEM accumulator sets so the epilogue overlaps the next tile,
+// MT = 2 for the packed-weight kernels so each expanded B stage feeds two MMAs):
 //   warp 0      TMA producer: fills a ring of 128B-swizzled shared-memory stages
 //   warp 1      MMA issuer: one thread issues tcgen05.mma into one of two TMEM
 //               accumulators, frees stages with tcgen05.commit
 //   warps 2-5   epilogue: tcgen05.ld the finished accumulator (one TMEM lane
 //               quadrant each) while the next tile is already being multiplied
 //   warps 6-13  (packed-weight kernels only) expand N-bit codes into the bf16 B
-//               operand stage: (q - z) * s in fp32, rounded once to bf16
+//               operand stage: (q - z) * s exactly in fp32, rounded once to bf16
 // The epilogue either stores the tile as bf16 or, for the E2E-QP step-size
 // gradient, multiplies each accumulator row by (q - z) of the matching packed
 // codes and reduces runs of `group` columns, so the [out,in] weight gradient
@@ -38,10 +40,9 @@ __device__ int g_device_status[2];   // [0] = eqat_status, [1] = WaitSite
 
 namespace {
 
-constexpr int BM = 128;          // tile rows = TMEM lanes
+constexpr int BM = 128;          // rows per MMA = TMEM lanes
 constexpr int BK = 64;           // K per stage: one 128-byte swizzle span of bf16
 constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit inputs
-constexpr int kEpiWarp0 = 2;
 constexpr int kDeqWarp0 = 6;
 constexpr int kDeqWarps = 8;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s per wait
@@ -62,14 +63,16 @@ struct GemmParams {
   float* dz;                 // may be null
 };
 
-template <int BN, bool PACKED>
+template <int BN, int MT, bool PACKED>
 struct Cfg {
-  static constexpr int kStages = BN == 256 ? 4 : 6;
-  static constexpr int kABytes = BM * BK * 2;
+  static constexpr int kTileM = MT * BM;                 // output rows per CTA tile
+  static constexpr int kAccSets = MT == 1 ? 2 : 1;       // TMEM holds kAccSets * MT accumulators of BN columns
+  static constexpr int kStages = MT == 2 ? 3 : (BN == 256 ? 4 : 6);
+  static constexpr int kABytes = kTileM * BK * 2;
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kThreads = PACKED ? (kDeqWarp0 + kDeqWarps) * 32 : kDeqWarp0 * 32;
-  static constexpr int kTmemCols = 2 * BN;
+  static constexpr int kTmemCols = kAccSets * MT * BN;
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
@@ -123,26 +126,76 @@ __device__ __forceinline__ void tile_coords(int tile, int num_m, int num_n, int&
 
 // Expand 64 consecutive codes of one weight row into one 128-byte swizzled
 // shared-memory row: element e of the row goes to 16-byte chunk (e/8) ^ rx.
+//
+// A code q is dropped into bits 16..23 of the float 0x4B000000 (= 2^23), giving
+// x = 2^23 + 65536*q exactly.  Then fma(x, s/65536, -(128 + z)*s) = (q - z)*s:
+// s is an fp16 value (11 significant bits), so s/65536 and (128 + z)*s are
+// exact in fp32 and so is the result; the only rounding is the final one to
+// bf16.  For 2 and 4 bits the codes reach byte positions with one shift+mask
+// per 4 codes and one byte permute each; 3-bit codes are shifted individually.
+struct DequantScale {
+  float sp, cz;
+  __device__ __forceinline__ DequantScale(float s, float z) : sp(s * (1.0f / 65536.0f)), cz(-(128.0f + z) * s) {}
+  __device__ __forceinline__ float operator()(uint32_t xbits) const { return fmaf(__uint_as_float(xbits), sp, cz); }
+};
+
+__device__ __forceinline__ void store_chunk(uint8_t* row, int chunk, int rx, const float (&v)[8]) {
+  const uint4 o = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                             pack_bf16x2(v[6], v[7]));
+  *reinterpret_cast<uint4*>(row + ((chunk ^ rx) << 4)) = o;
+}
+
 template <int BITS>
 __device__ __forceinline__ void dequant_row64(const uint32_t (&w)[2 * BITS], float s, float z, uint8_t* row, int rx) {
-  constexpr uint32_t mask = (1u << BITS) - 1u;
-  const float zoff = 8388608.0f + z;                    // codes enter as 2^23 + q (exact)
+  const DequantScale f(s, z);
+  constexpr uint32_t kMagic = 0x4B000000u;
+  if constexpr (BITS == 2) {
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
+    for (int i = 0; i < 4; ++i) {                       // word i: codes 16i .. 16i+15
+      uint32_t m[4];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+      for (int r = 0; r < 4; ++r) m[r] = (w[i] >> (2 * r)) & 0x03030303u;    // byte b of m[r] = code 4b + r
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int k = 8 * c + e;                      // code index in the word
+          v[e] = f(__byte_perm(m[k & 3], kMagic, 0x7044u | ((uint32_t)(k >> 2) << 8)));
+        }
+        store_chunk(row, 2 * i + c, rx, v);
+      }
+    }
+  } else if constexpr (BITS == 4) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {                       // word i: codes 8i .. 8i+7
+      const uint32_t m0 = w[i] & 0x0F0F0F0Fu, m1 = (w[i] >> 4) & 0x0F0F0F0Fu;   // byte b = code 2b (+1)
       float v[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int j = 8 * c + i;
-        const int bit = BITS * j, word = bit >> 5, off = bit & 31;
-        uint32_t x = w[h * BITS + word] >> off;
-        if (off + BITS > 32) x |= w[h * BITS + word + 1] << (32 - off);
-        v[i] = (__uint_as_float((x & mask) | 0x4B000000u) - zoff) * s;
+      for (int e = 0; e < 8; ++e)
+        v[e] = f(__byte_perm((e & 1) ? m1 : m0, kMagic, 0x7044u | ((uint32_t)(e >> 1) << 8)));
+      store_chunk(row, i, rx, v);
+    }
+  } else {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {                       // 32 codes = 3 words
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int bit = 3 * (8 * c + e), word = bit >> 5, off = bit & 31;
+          uint32_t t;
+          if (off <= 16) {
+            t = w[3 * h + word] << (16 - off);
+          } else {
+            const uint32_t hi = (off + 3 > 32) ? w[3 * h + word + 1] : 0u;
+            t = __funnelshift_r(w[3 * h + word], hi, off - 16);
+          }
+          v[e] = f((t & 0x00070000u) | kMagic);
+        }
+        store_chunk(row, 4 * h + c, rx, v);
       }
-      const uint4 o = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
-                                 pack_bf16x2(v[6], v[7]));
-      *reinterpret_cast<uint4*>(row + (((h * 4 + c) ^ rx) << 4)) = o;
     }
   }
 }
@@ -169,11 +222,11 @@ __device__ __forceinline__ void load_codes64(const uint8_t* p, uint32_t (&w)[2 *
 
 // A_MN / B_MN: operand is MN-major.  PACKED: B is expanded from N-bit codes.
 // BITS is used by PACKED and by EPI_DS.
-template <int BN, bool A_MN, bool B_MN, bool PACKED, int EPI, int BITS>
-__global__ void __launch_bounds__(Cfg<BN, PACKED>::kThreads, 1)
+template <int BN, int MT, bool A_MN, bool B_MN, bool PACKED, int EPI, int BITS>
+__global__ void __launch_bounds__(Cfg<BN, MT, PACKED>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const GemmParams p) {
-  using C = Cfg<BN, PACKED>;
+  using C = Cfg<BN, MT, PACKED>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_addr(smem_raw);
   const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
@@ -184,7 +237,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int num_m = (p.M + BM - 1) / BM;
+  const int num_m = (p.M + C::kTileM - 1) / C::kTileM;
   const int num_n = (p.N + BN - 1) / BN;
   const int num_tiles = num_m * num_n;
   const int num_kb = (p.K + BK - 1) / BK;
@@ -194,7 +247,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), PACKED ? 1 + kDeqWarps : 1);
       ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), 1);
     }
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < C::kAccSets; ++a) {
       ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[a]), 1);
       ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[a]), 4);
     }
@@ -234,10 +287,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           ptx::mbar_expect_tx(full, PACKED ? C::kABytes : C::kStageBytes);
           if (A_MN) {
 #pragma unroll
-            for (int b = 0; b < BM / 64; ++b)
-              ptx::tma_load_2d(a_dst + b * (BK * 128), &tmap_a, m_blk * BM + b * 64, kb * BK, full);
+            for (int b = 0; b < C::kTileM / 64; ++b)
+              ptx::tma_load_2d(a_dst + b * (BK * 128), &tmap_a, m_blk * C::kTileM + b * 64, kb * BK, full);
           } else {
-            ptx::tma_load_2d(a_dst, &tmap_a, kb * BK, m_blk * BM, full);
+            ptx::tma_load_2d(a_dst, &tmap_a, kb * BK, m_blk * C::kTileM, full);
           }
           if (!PACKED) {
             if (B_MN) {
@@ -275,6 +328,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                                  ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       constexpr uint32_t a_lbo = A_MN ? BK * 128 : 16, b_lbo = B_MN ? BK * 128 : 16;
       constexpr uint32_t a_step = A_MN ? UMMA_K * 128 : UMMA_K * 2, b_step = B_MN ? UMMA_K * 128 : UMMA_K * 2;
+      constexpr uint32_t a_half = BM * BK * 2;        // second 128-row half of the A stage (either major)
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -283,7 +337,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         if (!wait_bounded(ptx::smem_addr(&ctl->acc_empty[acc]), acc_phase ^ 1u, abort_flag, WAIT_MMA_ACC_EMPTY)) break;
         ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MT * BN);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!wait_bounded(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL)) {
             ok = false;
@@ -294,15 +348,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const uint32_t b_addr = a_addr + C::kABytes;
 #pragma unroll
           for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-            ptx::mma_bf16_ss(d_tmem, smem_desc(a_addr + kk * a_step, a_lbo), smem_desc(b_addr + kk * b_step, b_lbo),
-                             idesc, (kb | kk) != 0 ? 1u : 0u);
+            const uint64_t b_desc = smem_desc(b_addr + kk * b_step, b_lbo);
+#pragma unroll
+            for (int h = 0; h < MT; ++h)
+              ptx::mma_bf16_ss(d_tmem + h * BN, smem_desc(a_addr + h * a_half + kk * a_step, a_lbo), b_desc, idesc,
+                               (kb | kk) != 0 ? 1u : 0u);
           }
           ptx::mma_commit(ptx::smem_addr(&ctl->empty[stage]));
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         ptx::mma_commit(ptx::smem_addr(&ctl->acc_full[acc]));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        if (++acc == C::kAccSets) { acc = 0; acc_phase ^= 1u; }
       }
       // All MMAs of this thread must have retired before TMEM is freed.
       ptx::mma_commit(ptx::smem_addr(&ctl->drain));
@@ -319,64 +376,67 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       tile_coords(tile, num_m, num_n, m_blk, n_blk);
       if (!wait_bounded(ptx::smem_addr(&ctl->acc_full[acc]), acc_phase, abort_flag, WAIT_EPI_ACC_FULL)) break;
       ptx::tc_fence_after();
-      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
-      const int m = m_blk * BM + row_in_tile;
-      if constexpr (EPI == EPI_STORE) {
-        eqat_bf16* drow = p.D + (size_t)m * p.N;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r[32];
-          ptx::tmem_ld_32x32(t_row + c * 32, r);
-          ptx::tmem_ld_wait();
-          const int col0 = n_blk * BN + c * 32;
-          if (m < p.M) {
+      for (int h = 0; h < MT; ++h) {
+        const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MT + h) * BN);
+        const int m = m_blk * C::kTileM + h * BM + row_in_tile;
+        if constexpr (EPI == EPI_STORE) {
+          eqat_bf16* drow = p.D + (size_t)m * p.N;
+#pragma unroll 1
+          for (int c = 0; c < BN / 32; ++c) {
+            uint32_t r[32];
+            ptx::tmem_ld_32x32(t_row + c * 32, r);
+            ptx::tmem_ld_wait();
+            const int col0 = n_blk * BN + c * 32;
+            if (m < p.M) {
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              if (col0 + v * 8 < p.N) {
-                const uint4 o = make_uint4(
-                    pack_bf16x2(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1])),
-                    pack_bf16x2(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3])),
-                    pack_bf16x2(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5])),
-                    pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])));
-                *reinterpret_cast<uint4*>(drow + col0 + v * 8) = o;
+              for (int v = 0; v < 4; ++v) {
+                if (col0 + v * 8 < p.N) {
+                  const uint4 o = make_uint4(
+                      pack_bf16x2(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1])),
+                      pack_bf16x2(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3])),
+                      pack_bf16x2(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5])),
+                      pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])));
+                  *reinterpret_cast<uint4*>(drow + col0 + v * 8) = o;
+                }
               }
             }
           }
-        }
-      } else {
-        // Row m of the tile is output row o = m of the weight; columns are input
-        // features.  ds[o,g] = sum_{j in g} G[o,j] * (q[o,j] - z[o,g]).
-        const int groups_per_row = p.in_features >> p.group_shift;
-        const int chunks_per_group = 1 << (p.group_shift - 5);
-        const uint8_t* qrow = p.Wq + (size_t)m * ((size_t)p.in_features * BITS / 8);
-        float acc_s = 0.0f, acc_g = 0.0f;
+        } else {
+          // Row m of the tile is output row o = m of the weight; columns are input
+          // features.  ds[o,g] = sum_{j in g} G[o,j] * (q[o,j] - z[o,g]).
+          const int groups_per_row = p.in_features >> p.group_shift;
+          const int chunks_per_group = 1 << (p.group_shift - 5);
+          const uint8_t* qrow = p.Wq + (size_t)m * ((size_t)p.in_features * BITS / 8);
+          float acc_s = 0.0f, acc_g = 0.0f;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r[32];
-          ptx::tmem_ld_32x32(t_row + c * 32, r);
-          ptx::tmem_ld_wait();
-          const int col0 = n_blk * BN + c * 32;
-          if (m < p.M && col0 < p.N) {
-            uint32_t words[BITS];
-            const uint32_t* src = reinterpret_cast<const uint32_t*>(qrow) + (size_t)(col0 >> 5) * BITS;
+          for (int c = 0; c < BN / 32; ++c) {
+            uint32_t r[32];
+            ptx::tmem_ld_32x32(t_row + c * 32, r);
+            ptx::tmem_ld_wait();
+            const int col0 = n_blk * BN + c * 32;
+            if (m < p.M && col0 < p.N) {
+              uint32_t words[BITS];
+              const uint32_t* src = reinterpret_cast<const uint32_t*>(qrow) + (size_t)(col0 >> 5) * BITS;
 #pragma unroll
-            for (int i = 0; i < BITS; ++i) words[i] = __ldg(src + i);
-            uint32_t codes[32];
-            unpack32<BITS>(words, codes);
-            const int g = col0 >> p.group_shift;
-            const float zf = (float)__ldg(p.z8 + (size_t)m * groups_per_row + g);
+              for (int i = 0; i < BITS; ++i) words[i] = __ldg(src + i);
+              uint32_t codes[32];
+              unpack32<BITS>(words, codes);
+              const int g = col0 >> p.group_shift;
+              const float zf = (float)__ldg(p.z8 + (size_t)m * groups_per_row + g);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float gv = __uint_as_float(r[i]);
-              acc_s = fmaf(gv, (float)codes[i] - zf, acc_s);
-              acc_g += gv;
-            }
-            if (((c + 1) & (chunks_per_group - 1)) == 0) {
-              const size_t idx = (size_t)m * groups_per_row + g;
-              p.ds[idx] = acc_s;
-              if (p.dz != nullptr) p.dz[idx] = -__half2float(__ushort_as_half(__ldg(p.s16 + idx))) * acc_g;
-              acc_s = 0.0f;
-              acc_g = 0.0f;
+              for (int i = 0; i < 32; ++i) {
+                const float gv = __uint_as_float(r[i]);
+                acc_s = fmaf(gv, (float)codes[i] - zf, acc_s);
+                acc_g += gv;
+              }
+              if (((c + 1) & (chunks_per_group - 1)) == 0) {
+                const size_t idx = (size_t)m * groups_per_row + g;
+                p.ds[idx] = acc_s;
+                if (p.dz != nullptr) p.dz[idx] = -__half2float(__ushort_as_half(__ldg(p.s16 + idx))) * acc_g;
+                acc_s = 0.0f;
+                acc_g = 0.0f;
+              }
             }
           }
         }
@@ -384,7 +444,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[acc]));
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      if (++acc == C::kAccSets) { acc = 0; acc_phase ^= 1u; }
     }
   } else {
     // ------------------------------------------------------------ dequantiser (PACKED only)
@@ -495,15 +555,15 @@ int sm_count() {
   return n;
 }
 
-template <int BN, bool A_MN, bool B_MN, bool PACKED, int EPI, int BITS>
+template <int BN, int MT, bool A_MN, bool B_MN, bool PACKED, int EPI, int BITS>
 int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cudaStream_t st) {
-  using C = Cfg<BN, PACKED>;
-  auto kern = gemm_kernel<BN, A_MN, B_MN, PACKED, EPI, BITS>;
+  using C = Cfg<BN, MT, PACKED>;
+  auto kern = gemm_kernel<BN, MT, A_MN, B_MN, PACKED, EPI, BITS>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
     return EQAT_ERR_CUDA;
   const int sms = sm_count();
   if (sms <= 0) return EQAT_ERR_CUDA;
-  const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
+  const int tiles = ((p.M + C::kTileM - 1) / C::kTileM) * ((p.N + BN - 1) / BN);
   const int grid = tiles < sms ? tiles : sms;
   kern<<<grid, C::kThreads, C::kSmemBytes, st>>>(ta, tb, p);
   return launch_status();
@@ -536,7 +596,7 @@ int launch_dense_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* Wh
     return EQAT_ERR_CUDA;
   GemmParams p = base_params((int)d.tokens, d.out_features, d.in_features);
   p.D = Y;
-  return launch<256, false, false, false, EPI_STORE, 2>(ta, tb, p, st);
+  return launch<256, 1, false, false, false, EPI_STORE, 2>(ta, tb, p, st);
 }
 
 int launch_dense_dx(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* What, eqat_bf16* dX, cudaStream_t st) {
@@ -545,7 +605,7 @@ int launch_dense_dx(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* Wh
     return EQAT_ERR_CUDA;
   GemmParams p = base_params((int)d.tokens, d.in_features, d.out_features);
   p.D = dX;
-  return launch<256, false, true, false, EPI_STORE, 2>(ta, tb, p, st);
+  return launch<256, 1, false, true, false, EPI_STORE, 2>(ta, tb, p, st);
 }
 
 int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X, eqat_bf16* dWhat, cudaStream_t st) {
@@ -554,34 +614,34 @@ int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X,
     return EQAT_ERR_CUDA;
   GemmParams p = base_params(d.out_features, d.in_features, (int)d.tokens);
   p.D = dWhat;
-  return launch<256, true, true, false, EPI_STORE, 2>(ta, tb, p, st);
+  return launch<256, 1, true, true, false, EPI_STORE, 2>(ta, tb, p, st);
 }
 
 int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
                       const uint8_t* z8, eqat_bf16* Y, cudaStream_t st) {
   CUtensorMap ta;
-  if (!make_tmap(&ta, X, d.in_features, d.tokens, BM)) return EQAT_ERR_CUDA;
+  if (!make_tmap(&ta, X, d.in_features, d.tokens, 2 * BM)) return EQAT_ERR_CUDA;
   GemmParams p = base_params((int)d.tokens, d.out_features, d.in_features);
   p.D = Y;
   set_weight(p, d, Wq, s16, z8);
   switch (d.bits) {
-    case 2: return launch<256, false, false, true, EPI_STORE, 2>(ta, ta, p, st);
-    case 3: return launch<256, false, false, true, EPI_STORE, 3>(ta, ta, p, st);
-    default: return launch<256, false, false, true, EPI_STORE, 4>(ta, ta, p, st);
+    case 2: return launch<256, 2, false, false, true, EPI_STORE, 2>(ta, ta, p, st);
+    case 3: return launch<256, 2, false, false, true, EPI_STORE, 3>(ta, ta, p, st);
+    default: return launch<256, 2, false, false, true, EPI_STORE, 4>(ta, ta, p, st);
   }
 }
 
 int launch_packed_dx(const eqat_desc& d, const eqat_bf16* dY, const uint8_t* Wq, const eqat_fp16* s16,
                      const uint8_t* z8, eqat_bf16* dX, cudaStream_t st) {
   CUtensorMap ta;
-  if (!make_tmap(&ta, dY, d.out_features, d.tokens, BM)) return EQAT_ERR_CUDA;
+  if (!make_tmap(&ta, dY, d.out_features, d.tokens, 2 * BM)) return EQAT_ERR_CUDA;
   GemmParams p = base_params((int)d.tokens, d.in_features, d.out_features);
   p.D = dX;
   set_weight(p, d, Wq, s16, z8);
   switch (d.bits) {
-    case 2: return launch<256, false, true, true, EPI_STORE, 2>(ta, ta, p, st);
-    case 3: return launch<256, false, true, true, EPI_STORE, 3>(ta, ta, p, st);
-    default: return launch<256, false, true, true, EPI_STORE, 4>(ta, ta, p, st);
+    case 2: return launch<256, 2, false, true, true, EPI_STORE, 2>(ta, ta, p, st);
+    case 3: return launch<256, 2, false, true, true, EPI_STORE, 3>(ta, ta, p, st);
+    default: return launch<256, 2, false, true, true, EPI_STORE, 4>(ta, ta, p, st);
   }
 }
 
@@ -595,9 +655,9 @@ int launch_packed_ds(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* dY
   p.ds = ds;
   p.dz = dz;
   switch (d.bits) {
-    case 2: return launch<256, true, true, false, EPI_DS, 2>(ta, tb, p, st);
-    case 3: return launch<256, true, true, false, EPI_DS, 3>(ta, tb, p, st);
-    default: return launch<256, true, true, false, EPI_DS, 4>(ta, tb, p, st);
+    case 2: return launch<256, 1, true, true, false, EPI_DS, 2>(ta, tb, p, st);
+    case 3: return launch<256, 1, true, true, false, EPI_DS, 3>(ta, tb, p, st);
+    default: return launch<256, 1, true, true, false, EPI_DS, 4>(ta, tb, p, st);
   }
 }
 
