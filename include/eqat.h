@@ -135,6 +135,31 @@ int qlinear_fakequant_bwd(const eqat_desc* desc, const eqat_bf16* X, const eqat_
                           eqat_bf16* dX, eqat_bf16* dW, float* ds, float* dz,
                           void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same computation as qlinear_fakequant_bwd, for callers that cannot
+ * allocate device memory (no counterpart in the paper: it is a deployment
+ * convenience of this library).  Typical cases: the process's device memory is
+ * already owned by another framework's pool, or the caller sits in a section
+ * where the device-wide synchronisation that cudaMalloc / cudaFree may imply is
+ * not acceptable.  The out*in bf16 values of scratch live in a fixed array
+ * inside the library, so
+ *   - out_features * in_features must not exceed EQAT_NOALLOC_MAX_WEIGHT_ELEMS
+ *     (8 MiB of bf16); larger problems return EQAT_ERR_WORKSPACE and launch
+ *     nothing.  Every GPU that loads the library holds those 8 MiB until exit;
+ *   - the first call on each device looks the array's address up (a runtime
+ *     call that is not stream work): make that first call before any stream
+ *     capture begins on that device;
+ *   - all calls on a device share the one array.  Its previous contents do not
+ *     matter (every value read is written earlier in the same call), but two
+ *     calls whose kernels overlap on the GPU (different streams) race on it:
+ *     serialise them;
+ *   - it calls no cudaMalloc, cudaFree or other allocating routine.
+ * Arguments, outputs and status codes are otherwise those of
+ * qlinear_fakequant_bwd. */
+#define EQAT_NOALLOC_MAX_WEIGHT_ELEMS (4u << 20)
+int qlinear_fakequant_bwd_noalloc(const eqat_desc* desc, const eqat_bf16* X, const eqat_bf16* dY,
+                                  const eqat_bf16* W, const float* s, const float* z, const eqat_bf16* W_hat,
+                                  eqat_bf16* dX, eqat_bf16* dW, float* ds, float* dz, void* stream);
+
 /* ------------------------------------------------------------------ storage format */
 /* The paper stores W_int and z in N bits and s in fp16 (Sec. 3.2, last
  * paragraph; N + (N+16)/g bits per parameter, appendix "Size of Quantized

@@ -49,6 +49,7 @@ def _load():
         "qlinear_fakequant_fwd": (c_int, [D, P, P, P, P, P, P, P]),
         "eqat_ste_bwd": (c_int, [D, P, P, P, P, P, P, P, P]),
         "qlinear_fakequant_bwd": (c_int, [D, P, P, P, P, P, P, P, P, P, P, P, c_size_t, P]),
+        "qlinear_fakequant_bwd_noalloc": (c_int, [D, P, P, P, P, P, P, P, P, P, P, P]),
         "eqat_quantize_pack": (c_int, [D, P, P, P, P, P, P, P]),
         "eqat_pack": (c_int, [D, P, P, P]),
         "eqat_unpack": (c_int, [D, P, P, P]),
@@ -130,6 +131,19 @@ def qlinear_fakequant_bwd(desc, X, dY, W, s, z, W_hat, dX, dW, ds, dz, workspace
     _check(lib.qlinear_fakequant_bwd(ctypes.byref(desc), _ptr(X), _ptr(dY), _ptr(W), _ptr(s), _ptr(z), _ptr(W_hat),
                                      _ptr(dX), _ptr(dW), _ptr(ds), _ptr(dz), _ptr(workspace), nbytes, _stream()),
            "qlinear_fakequant_bwd")
+
+
+NOALLOC_MAX_WEIGHT_ELEMS = 4 << 20
+
+
+def qlinear_fakequant_bwd_noalloc(desc, X, dY, W, s, z, W_hat, dX, dW, ds, dz):
+    """Block-AP backward without a caller-provided workspace: for callers that
+    cannot allocate device memory (the scratch is a fixed 8 MiB array inside the
+    library, so out*in <= NOALLOC_MAX_WEIGHT_ELEMS; calls on one device must not
+    overlap; make the first call on a device outside any stream capture)."""
+    _check(lib.qlinear_fakequant_bwd_noalloc(ctypes.byref(desc), _ptr(X), _ptr(dY), _ptr(W), _ptr(s), _ptr(z),
+                                             _ptr(W_hat), _ptr(dX), _ptr(dW), _ptr(ds), _ptr(dz), _stream()),
+           "qlinear_fakequant_bwd_noalloc")
 
 
 def eqat_quantize_pack(desc, W, s, z, Wq_packed, z8, s16):
