@@ -87,12 +87,17 @@ struct Control {
 };
 static_assert(sizeof(Control) <= 256, "control block must fit its reservation");
 
+// Bounded wait on an mbarrier phase.  `sleep_ns` > 0 backs off between polls so
+// that a role with nothing to do for a long time (the epilogue during a main
+// loop, the producer on a full ring) leaves the issue slots to the warps that
+// are working; latency-critical waits pass 0.
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort, int site,
-                                             uint64_t limit_ns = kWaitLimitNs) {
+                                             uint32_t sleep_ns = 0, uint64_t limit_ns = kWaitLimitNs) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = ptx::globaltimer_ns();
   uint32_t n = 0;
   while (!ptx::mbar_try_wait(bar, parity)) {
+    if (sleep_ns != 0) __nanosleep(sleep_ns);
     if ((++n & 31u) == 0u) {
       if (*abort) return false;
       if (ptx::globaltimer_ns() - t0 > limit_ns) {
@@ -131,8 +136,9 @@ __device__ __forceinline__ void tile_coords(int tile, int num_m, int num_n, int&
 // x = 2^23 + 65536*q exactly.  Then fma(x, s/65536, -(128 + z)*s) = (q - z)*s:
 // s is an fp16 value (11 significant bits), so s/65536 and (128 + z)*s are
 // exact in fp32 and so is the result; the only rounding is the final one to
-// bf16.  For 2 and 4 bits the codes reach byte positions with one shift+mask
-// per 4 codes and one byte permute each; 3-bit codes are shifted individually.
+// bf16.  4-bit codes reach byte positions with one shift+mask per 4 codes and
+// one byte permute each; 3-bit codes are shifted individually; 2-bit codes use
+// a 4-entry table per group instead (see below).
 struct DequantScale {
   float sp, cz;
   __device__ __forceinline__ DequantScale(float s, float z) : sp(s * (1.0f / 65536.0f)), cz(-(128.0f + z) * s) {}
@@ -150,20 +156,30 @@ __device__ __forceinline__ void dequant_row64(const uint32_t (&w)[2 * BITS], flo
   const DequantScale f(s, z);
   constexpr uint32_t kMagic = 0x4B000000u;
   if constexpr (BITS == 2) {
+    // Four possible values per group: build them once, exactly, as bf16
+    // ((q - z)*s has at most 13 significant bits, so the fp32 value is exact and
+    // the conversion is the only rounding), then look each code up with a byte
+    // permute.  lut01 = (v0, v1), lut23 = (v2, v3); value q occupies bytes 2q, 2q+1
+    // of the 8-byte pair, so the selector byte of a code is 0x10 + 0x22*q.
+    const float zs = z * s;
+    const uint32_t lut01 = pack_bf16x2(-zs, s - zs);
+    const uint32_t lut23 = pack_bf16x2(fmaf(2.0f, s, -zs), fmaf(3.0f, s, -zs));
 #pragma unroll
     for (int i = 0; i < 4; ++i) {                       // word i: codes 16i .. 16i+15
-      uint32_t m[4];
+      uint32_t sel[4];                                  // byte b of sel[r] = selector byte of code 4b + r
 #pragma unroll
-      for (int r = 0; r < 4; ++r) m[r] = (w[i] >> (2 * r)) & 0x03030303u;    // byte b of m[r] = code 4b + r
+      for (int r = 0; r < 4; ++r) sel[r] = ((w[i] >> (2 * r)) & 0x03030303u) * 0x22u + 0x10101010u;
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
-        float v[8];
+        uint32_t o[4];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int k = 8 * c + e;                      // code index in the word
-          v[e] = f(__byte_perm(m[k & 3], kMagic, 0x7044u | ((uint32_t)(k >> 2) << 8)));
+        for (int pr = 0; pr < 4; ++pr) {
+          const int k = 8 * c + 2 * pr;                 // even code of the pair; k = 4b + r with r in {0, 2}
+          const uint32_t b = (uint32_t)(k >> 2), r = (uint32_t)(k & 3);
+          const uint32_t pair_sel = __byte_perm(sel[r], sel[r + 1], b | ((4u + b) << 4));
+          o[pr] = __byte_perm(lut01, lut23, pair_sel);
         }
-        store_chunk(row, 2 * i + c, rx, v);
+        *reinterpret_cast<uint4*>(row + (((2 * i + c) ^ rx) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
   } else if constexpr (BITS == 4) {
@@ -277,7 +293,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         int m_blk, n_blk;
         tile_coords(tile, num_m, num_n, m_blk, n_blk);
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_PRODUCER_EMPTY)) {
+          if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_PRODUCER_EMPTY, 64)) {
             ok = false;
             break;
           }
@@ -335,11 +351,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        if (!wait_bounded(ptx::smem_addr(&ctl->acc_empty[acc]), acc_phase ^ 1u, abort_flag, WAIT_MMA_ACC_EMPTY)) break;
+        if (!wait_bounded(ptx::smem_addr(&ctl->acc_empty[acc]), acc_phase ^ 1u, abort_flag, WAIT_MMA_ACC_EMPTY, 64)) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MT * BN);
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!wait_bounded(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL)) {
+          if (!wait_bounded(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL, PACKED ? 32 : 0)) {
             ok = false;
             break;
           }
@@ -363,7 +379,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       }
       // All MMAs of this thread must have retired before TMEM is freed.
       ptx::mma_commit(ptx::smem_addr(&ctl->drain));
-      wait_bounded(ptx::smem_addr(&ctl->drain), 0u, abort_flag, WAIT_TEARDOWN, kDrainLimitNs * 4);
+      wait_bounded(ptx::smem_addr(&ctl->drain), 0u, abort_flag, WAIT_TEARDOWN, 64, kDrainLimitNs * 4);
     }
   } else if (warp < kDeqWarp0) {
     // ------------------------------------------------------------ epilogue
@@ -374,7 +390,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
       int m_blk, n_blk;
       tile_coords(tile, num_m, num_n, m_blk, n_blk);
-      if (!wait_bounded(ptx::smem_addr(&ctl->acc_full[acc]), acc_phase, abort_flag, WAIT_EPI_ACC_FULL)) break;
+      if (!wait_bounded(ptx::smem_addr(&ctl->acc_full[acc]), acc_phase, abort_flag, WAIT_EPI_ACC_FULL, MT == 2 ? 512 : 128)) break;
       ptx::tc_fence_after();
 #pragma unroll 1
       for (int h = 0; h < MT; ++h) {
@@ -458,17 +474,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       bool ok = true;
       // unit -> (weight row, 64-code unit in the row, shared-memory row)
       //   B K-major  (Y):  tile row n = t is weight row n0 + t, unit = kb
-      //   B MN-major (dX): k-row t/4 is weight row kb*64 + t/4, unit = n0/64 + t%4 (box t%4)
-      const int smem_row_off = B_MN ? ((t & 3) * (BK * 128) + (t >> 2) * 128) : t * 128;
-      const int rx = B_MN ? ((t >> 2) & 7) : (t & 7);
+      //   B MN-major (dX): k-row kr is weight row kb*64 + kr, unit = n0/64 + box (64-column box).
+      // The 8 lanes of a quarter-warp (one 16-byte store wavefront) always own 8
+      // consecutive rows, whose swizzled chunks fall in 8 different bank groups.
+      const int kr = (t & 7) | ((t >> 5) << 3);                   // MN-major: k-row 0..63
+      const int box = (t >> 3) & 3;                               // MN-major: 64-column box 0..3
+      const int smem_row_off = B_MN ? (box * (BK * 128) + kr * 128) : t * 128;
+      const int rx = B_MN ? (kr & 7) : (t & 7);
       struct Unit {
         uint32_t w[2 * BITS];
         float s, z;
         bool valid;
       };
       auto fetch = [&](Unit& u, int n_blk, int kb) {
-        const int wrow = B_MN ? kb * BK + (t >> 2) : n_blk * BN + t;
-        const int unit = B_MN ? n_blk * (BN / 64) + (t & 3) : kb;
+        const int wrow = B_MN ? kb * BK + kr : n_blk * BN + t;
+        const int unit = B_MN ? n_blk * (BN / 64) + box : kb;
         u.valid = wrow < p.out_features && unit < chunks_in;
         if (u.valid) {
           load_codes64<BITS>(p.Wq + (size_t)wrow * pitch + (size_t)unit * (8 * BITS), u.w);
@@ -477,30 +497,39 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           u.z = (float)__ldg(p.z8 + gi);
         }
       };
-      Unit cur, nxt;
+      // Register ring of units: the loads for K block kb + kRing are issued as soon
+      // as block kb has been expanded, so they have kRing - 1 whole stages to land.
+      constexpr int kRing = 4;
+      Unit ring[kRing];
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
         tile_coords(tile, num_m, num_n, m_blk, n_blk);
-        fetch(cur, n_blk, 0);
-        for (int kb = 0; kb < num_kb; ++kb) {
-          // the next unit's loads fly while this one waits for its stage and is expanded
-          if (kb + 1 < num_kb) fetch(nxt, n_blk, kb + 1);
-          if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_DEQ_OPERAND_EMPTY)) {
-            ok = false;
-            break;
-          }
-          uint8_t* row = smem + stage * C::kStageBytes + C::kABytes + smem_row_off;
-          if (cur.valid) {
-            dequant_row64<BITS>(cur.w, cur.s, cur.z, row, rx);
-          } else {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) reinterpret_cast<uint4*>(row)[c] = make_uint4(0u, 0u, 0u, 0u);
+        for (int j = 0; j < kRing; ++j)
+          if (j < num_kb) fetch(ring[j], n_blk, j);
+        for (int kb0 = 0; kb0 < num_kb && ok; kb0 += kRing) {
+#pragma unroll
+          for (int j = 0; j < kRing; ++j) {
+            const int kb = kb0 + j;
+            if (ok && kb < num_kb) {
+              if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_DEQ_OPERAND_EMPTY)) {
+                ok = false;
+              } else {
+                uint8_t* row = smem + stage * C::kStageBytes + C::kABytes + smem_row_off;
+                if (ring[j].valid) {
+                  dequant_row64<BITS>(ring[j].w, ring[j].s, ring[j].z, row, rx);
+                } else {
+#pragma unroll
+                  for (int c = 0; c < 8; ++c) reinterpret_cast<uint4*>(row)[c] = make_uint4(0u, 0u, 0u, 0u);
+                }
+                if (kb + kRing < num_kb) fetch(ring[j], n_blk, kb + kRing);
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full[stage]));
+                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+              }
+            }
           }
-          ptx::fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full[stage]));
-          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
-          cur = nxt;
         }
       }
     }
