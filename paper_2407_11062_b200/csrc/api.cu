@@ -88,7 +88,13 @@ size_t eqat_workspace_bytes(const eqat_desc* d, int op) {
 
 int eqat_device_status(int* h_status, int* h_detail) {
   if (h_status == nullptr) return EQAT_ERR_NULL;
-  return read_device_status(h_status, h_detail);
+  int st[2] = {0, 0}, det[2] = {0, 0};
+  EQAT_TRY(read_device_status(&st[0], &det[0]));      // GEMM kernels
+  EQAT_TRY(read_stream_status(&st[1], &det[1]));      // staged streaming kernels
+  const int k = st[0] != EQAT_OK ? 0 : 1;
+  *h_status = st[k];
+  if (h_detail != nullptr) *h_detail = det[k];
+  return EQAT_OK;
 }
 
 int eqat_minmax_init(const eqat_desc* d, const eqat_bf16* W, float* s, float* z, void* stream) {

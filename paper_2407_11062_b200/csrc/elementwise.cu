@@ -49,6 +49,7 @@ __device__ __forceinline__ void quant_terms(float w, float s, float zr, float& t
 __device__ __forceinline__ float clamp_code(float p, float Q) { return fminf(fmaxf(p, 0.0f), Q); }
 
 // ------------------------------------------------------------------ Eq. 1 + Eq. 2
+// (used for groups longer than 256 elements; shorter groups take the staged kernel in stream.cu)
 __global__ void __launch_bounds__(kThreads)
 fakequant_kernel(const eqat_bf16* __restrict__ W, const float* __restrict__ s, const float* __restrict__ z,
                  eqat_bf16* __restrict__ What, size_t n_vec, uint32_t vec_per_group, float Q) {
@@ -81,54 +82,7 @@ fakequant_kernel(const eqat_bf16* __restrict__ W, const float* __restrict__ s, c
 }
 
 // ------------------------------------------------------------------ Eqs. 3-5 + group sums
-// LPG = lanes per group (group / 8), a power of two <= 32.
-template <int LPG>
-__global__ void __launch_bounds__(kThreads)
-ste_bwd_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __restrict__ W,
-               const float* __restrict__ s, const float* __restrict__ z,
-               eqat_bf16* __restrict__ dW, float* __restrict__ ds, float* __restrict__ dz,
-               size_t n_vec, float Q, int dz_literal) {
-  const size_t base = (size_t)blockIdx.x * (kThreads * 2) + threadIdx.x;
-#pragma unroll
-  for (int u = 0; u < 2; ++u) {
-    const size_t v = base + (size_t)u * kThreads;
-    const bool live = v < n_vec;
-    const size_t g = v / LPG;
-    float acc_s = 0.0f, acc_z = 0.0f;
-    if (live) {
-      const Vec8 gr = load_bf16x8(dWhat, v);
-      const Vec8 w = load_bf16x8(W, v);
-      const float sv = __ldg(s + g);
-      const float zr = rintf(__ldg(z + g));
-      const float dz_clamped = dz_literal ? -1.0f : -sv;
-      Vec8 o;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        float t, r, p;
-        quant_terms(w.v[i], sv, zr, t, r, p);
-        const bool below = p < 0.0f;
-        const bool above = p > Q;
-        const bool inside = !(below || above);
-        o.v[i] = inside ? gr.v[i] : 0.0f;                                  // Eq. 5
-        const float ds_el = inside ? (r - t) : (below ? -zr : Q - zr);    // Eq. 3
-        const float dz_el = inside ? 0.0f : dz_clamped;                    // Eq. 4
-        acc_s = fmaf(gr.v[i], ds_el, acc_s);
-        acc_z = fmaf(gr.v[i], dz_el, acc_z);
-      }
-      store_bf16x8(dW, v, o);
-    }
-#pragma unroll
-    for (int d = LPG / 2; d >= 1; d >>= 1) {
-      acc_s += __shfl_xor_sync(0xFFFFFFFFu, acc_s, d);
-      acc_z += __shfl_xor_sync(0xFFFFFFFFu, acc_z, d);
-    }
-    if (live && (v % LPG) == 0) {
-      ds[g] = acc_s;
-      if (dz != nullptr) dz[g] = acc_z;
-    }
-  }
-}
-
+// (groups of at most 256 elements are handled by the staged kernel in stream.cu)
 // One block per group, for groups longer than 256 elements (e.g. channel-wise).
 __global__ void __launch_bounds__(kThreads)
 ste_bwd_long_group_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __restrict__ W,
@@ -354,6 +308,7 @@ inline unsigned blocks_for(size_t items, size_t per_block) { return (unsigned)((
 // ------------------------------------------------------------------ host launchers
 int launch_fakequant(const eqat_desc& d, const eqat_bf16* W, const float* s, const float* z, eqat_bf16* What,
                      cudaStream_t st) {
+  if (d.group <= 256) return launch_fakequant_stream(d, W, s, z, What, st);
   const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
   const float Q = (float)((1 << d.bits) - 1);
   fakequant_kernel<<<blocks_for(n_vec, kThreads * 2), kThreads, 0, st>>>(W, s, z, What, n_vec,
@@ -363,20 +318,11 @@ int launch_fakequant(const eqat_desc& d, const eqat_bf16* W, const float* s, con
 
 int launch_ste_bwd(const eqat_desc& d, const eqat_bf16* dWhat, const eqat_bf16* W, const float* s, const float* z,
                    eqat_bf16* dW, float* ds, float* dz, cudaStream_t st) {
-  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
+  if (d.group <= 256) return launch_ste_bwd_stream(d, dWhat, W, s, z, dW, ds, dz, st);
   const float Q = (float)((1 << d.bits) - 1);
-  const unsigned nb = blocks_for(n_vec, kThreads * 2);
-  const int lit = d.dz_mode == 1;
-  switch (d.group) {
-    case 32:  ste_bwd_kernel<4><<<nb, kThreads, 0, st>>>(dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit); break;
-    case 64:  ste_bwd_kernel<8><<<nb, kThreads, 0, st>>>(dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit); break;
-    case 128: ste_bwd_kernel<16><<<nb, kThreads, 0, st>>>(dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit); break;
-    case 256: ste_bwd_kernel<32><<<nb, kThreads, 0, st>>>(dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit); break;
-    default: {
-      const size_t n_groups = (size_t)d.out_features * d.in_features / d.group;
-      ste_bwd_long_group_kernel<<<(unsigned)n_groups, kThreads, 0, st>>>(dWhat, W, s, z, dW, ds, dz, d.group / 8, Q, lit);
-    }
-  }
+  const size_t n_groups = (size_t)d.out_features * d.in_features / d.group;
+  ste_bwd_long_group_kernel<<<(unsigned)n_groups, kThreads, 0, st>>>(dWhat, W, s, z, dW, ds, dz, d.group / 8, Q,
+                                                                     d.dz_mode == 1);
   return launch_status();
 }
 

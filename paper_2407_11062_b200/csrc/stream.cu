@@ -1,0 +1,357 @@
+// Streaming kernels with TMA-staged inputs: fake quantiser (Eq. 1 + Eq. 2) and
+// its straight-through backward (Eqs. 3-5) for groups of at most 256 elements.
+//
+// These kernels are bound by HBM bandwidth, and what decides how close they
+// get to it is the number of bytes in flight per SM.  A plain "load, compute,
+// store" thread keeps its loads in flight only until its arithmetic starts,
+// and the arithmetic here is long (a division-free but exact quantiser per
+// element).  So the loads are taken out of the compute threads: each persistent
+// CTA has one producer thread that streams 8 KB chunks of the input(s) into a
+// shared-memory ring with bulk asynchronous copies (cp.async.bulk, completion
+// on an mbarrier), several chunks ahead, while 8 consumer warps pull 16-byte
+// vectors from the ring, compute, and write results to global memory with
+// coalesced 16-byte stores.  Three CTAs fit on an SM, so about 150 KB of reads
+// are in flight per SM whatever the consumers are doing.
+//
+// A quantisation group is contiguous in the flattened weight and owned by
+// group/8 adjacent lanes of one warp; group sums are fixed-order shuffles, so
+// results are run-to-run identical.
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "ptx.cuh"
+
+namespace eqat {
+
+__device__ int g_stream_status[2];   // [0] = eqat_status, [1] = WaitSite
+
+namespace {
+
+constexpr int kConsumers = 256;
+constexpr int kThreadsS = kConsumers + 32;           // + one producer warp
+constexpr int kChunkVec = 2 * kConsumers;            // 16-byte vectors per chunk and stream (8 KB)
+constexpr int kChunkBytes = kChunkVec * 16;
+constexpr uint64_t kStreamWaitLimitNs = 2000000000ull;
+
+template <int NIN>
+struct Ring {
+  static constexpr int kStages = NIN == 1 ? 6 : 4;
+  static constexpr int kStageBytes = NIN * kChunkBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 256;
+};
+
+struct RingCtl {
+  uint64_t full[8];
+  uint64_t empty[8];
+  int abort;
+};
+static_assert(sizeof(RingCtl) <= 256, "ring control block must fit its reservation");
+
+__device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity, volatile int* abort, int site,
+                                          uint32_t sleep_ns) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = ptx::globaltimer_ns();
+  uint32_t n = 0;
+  while (!ptx::mbar_try_wait(bar, parity)) {
+    if (sleep_ns != 0) __nanosleep(sleep_ns);
+    if ((++n & 31u) == 0u) {
+      if (*abort) return false;
+      if (ptx::globaltimer_ns() - t0 > kStreamWaitLimitNs) {
+        *abort = 1;
+        atomicExch(&g_stream_status[1], site);
+        atomicExch(&g_stream_status[0], (int)EQAT_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Runs `body(v, raw)` on every consumer thread for every chunk this CTA owns:
+// v is the index of the thread's first vector, raw[i][u] the thread's vector
+// u (v + u * 256) of input stream i.  Vectors at or beyond n_vec hold stale
+// shared memory and must be ignored by the body.
+template <int NIN, typename Body>
+__device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], size_t n_vec, Body&& body) {
+  using R = Ring<NIN>;
+  extern __shared__ __align__(128) uint8_t smem[];
+  RingCtl* ctl = reinterpret_cast<RingCtl*>(smem + R::kStages * R::kStageBytes);
+  volatile int* abort_flag = &ctl->abort;
+  const uint32_t smem_base = ptx::smem_addr(smem);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const size_t n_chunks = (n_vec + kChunkVec - 1) / kChunkVec;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < R::kStages; ++s) {
+      ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), 1);
+      ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), kConsumers / 32);
+    }
+    ctl->abort = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+
+  if (warp == kConsumers / 32) {
+    // ---------------------------------------------------------------- producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      size_t issued = 0;
+      bool ok = true;
+      for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+        if (!ring_wait(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_PRODUCER_EMPTY, 32)) {
+          ok = false;
+          break;
+        }
+        const size_t v0 = chunk * kChunkVec;
+        const uint32_t bytes = (uint32_t)((n_vec - v0 < (size_t)kChunkVec ? n_vec - v0 : (size_t)kChunkVec) * 16);
+        const uint32_t full = ptx::smem_addr(&ctl->full[stage]);
+        ptx::mbar_expect_tx(full, NIN * bytes);
+#pragma unroll
+        for (int i = 0; i < NIN; ++i)
+          bulk_load(smem_base + stage * R::kStageBytes + i * kChunkBytes, src[i] + v0 * 16, bytes, full);
+        ++issued;
+        if (++stage == R::kStages) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok || *abort_flag) {
+        // every copy this thread started must land before the CTA exits
+        const size_t first = issued > (size_t)R::kStages ? issued - R::kStages : 0;
+        for (size_t i = first; i < issued; ++i) {
+          const uint32_t bar = ptx::smem_addr(&ctl->full[i % R::kStages]);
+          const uint32_t par = (uint32_t)((i / R::kStages) & 1);
+          const uint64_t t0 = ptx::globaltimer_ns();
+          while (!ptx::mbar_try_wait(bar, par)) {
+            if (ptx::globaltimer_ns() - t0 > 50000000ull) {
+              atomicExch(&g_stream_status[1], (int)WAIT_TEARDOWN);
+              break;
+            }
+          }
+        }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- consumers
+    int stage = 0;
+    uint32_t phase = 0;
+    for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+      if (!ring_wait(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL, 0)) break;
+      uint4 raw[NIN][2];
+      const uint8_t* st = smem + stage * R::kStageBytes;
+#pragma unroll
+      for (int i = 0; i < NIN; ++i)
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+          raw[i][u] = *reinterpret_cast<const uint4*>(st + i * kChunkBytes + (u * kConsumers + threadIdx.x) * 16);
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->empty[stage]));   // the stage can be refilled now
+      if (++stage == R::kStages) { stage = 0; phase ^= 1u; }
+      body(chunk * kChunkVec + threadIdx.x, raw);
+    }
+  }
+}
+
+__device__ __forceinline__ void unpack8(const uint4& raw, float (&v)[8]) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+__device__ __forceinline__ uint4 pack8(const float (&v)[8]) {
+  return make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                    pack_bf16x2(v[6], v[7]));
+}
+
+// 1/s to within 1 ulp (rcp.approx.f32); NaN, which forces the exact path below,
+// when the reciprocal is subnormal or not finite and the error bound would not hold.
+__device__ __forceinline__ float group_rcp(float s) {
+  float rs;
+  asm("rcp.approx.f32 %0, %1;" : "=f"(rs) : "f"(s));
+  return (fabsf(rs) >= 1.17549435e-38f && fabsf(rs) <= 3.402823466e+38f) ? rs : __int_as_float(0x7FC00000);
+}
+
+// Eq. 1 for the eight elements of a vector: r = round(w/s) and the STE term
+// r - w/s.  The code is DEFINED by a correctly rounded binary32 division
+// followed by round-half-to-even, r = rintf(__fdiv_rn(w, s)).  Division and
+// rintf run on the quarter-rate special-function pipe, which would cap these
+// kernels below the memory roofline, so the common case takes a shortcut that
+// provably gives the same r:
+//   with rs a reciprocal of s good to 1 ulp, the exact product w*rs differs from
+//   the exact quotient by at most 2^-23 |q| and from rn(w/s) by at most
+//   1.5 * 2^-23 |q|.  r0 = rint(w*rs) (one fused multiply-add with 1.5 * 2^23,
+//   which rounds the exact product half-to-even, then a subtraction) can differ
+//   from rint(rn(w/s)) only if a half-integer lies between the two values; for
+//   |q| <= 512 that needs w*rs within 2^-13 of a half-integer.
+//   d = w*rs - r0 (one more fused multiply-add) is the distance to the integer.
+//   Unless every element of the vector has |d| < 0.5 - 2^-12 and |r0| <= 512,
+//   the whole vector is redone with the exact sequence (rare).
+// The STE term r - w/s is returned as -d in the common case (2^-23 relative away
+// from the exact one, immaterial for a gradient).
+__device__ __forceinline__ void quotient_round8(const float (&w)[8], float s, float rs, float (&r)[8],
+                                                float (&r_minus_t)[8]) {
+  float dmax = 0.0f, rmax = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float r0 = fmaf(w[i], rs, 12582912.0f) - 12582912.0f;
+    const float d = fmaf(w[i], rs, -r0);
+    r[i] = r0;
+    r_minus_t[i] = -d;
+    dmax = fmaxf(dmax, fabsf(d));
+    rmax = fmaxf(rmax, fabsf(r0));
+  }
+  if (!(dmax < 0.499755859375f && rmax <= 512.0f)) {      // also taken when anything is NaN
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float q = __fdiv_rn(w[i], s);
+      r[i] = rintf(q);
+      r_minus_t[i] = r[i] - q;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ Eq. 1 + Eq. 2
+// (clamp(r + z, 0, Q) - z) * s == clamp(r, -z, Q - z) * s for integer r and z.
+__global__ void __launch_bounds__(kThreadsS)
+fakequant_stream_kernel(const eqat_bf16* __restrict__ W, const float* __restrict__ s, const float* __restrict__ z,
+                        eqat_bf16* __restrict__ What, size_t n_vec, int vec_shift, float Q) {
+  const uint8_t* const src[1] = {reinterpret_cast<const uint8_t*>(W)};
+  stream_chunks<1>(src, n_vec, [&](size_t v0, const uint4 (&raw)[1][2]) {
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const size_t v = v0 + (size_t)u * kConsumers;
+      if (v < n_vec) {
+        const size_t g = v >> vec_shift;
+        const float sv = __ldg(s + g);
+        const float zr = rintf(__ldg(z + g));
+        const float rs = group_rcp(sv);
+        const float lo = -zr, hi = Q - zr;
+        float w[8], r[8], rt[8];
+        unpack8(raw[0][u], w);
+        quotient_round8(w, sv, rs, r, rt);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = fminf(fmaxf(r[i], lo), hi) * sv;
+        reinterpret_cast<uint4*>(What)[v] = pack8(w);
+      }
+    }
+  });
+}
+
+// ------------------------------------------------------------------ Eqs. 3-5 + group sums
+// With lo = -z, hi = Q - z and c = clamp(r, lo, hi): the element is in range iff
+// c == r, and on the clamped branches Eq. 3's value (-z or Q - z) is c itself.
+// Eq. 4 is a constant per group times the sum of the gradient over the clamped
+// elements.  LPG = lanes per group (group / 8).
+template <int LPG>
+__global__ void __launch_bounds__(kThreadsS)
+ste_bwd_stream_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __restrict__ W,
+                      const float* __restrict__ s, const float* __restrict__ z, eqat_bf16* __restrict__ dW,
+                      float* __restrict__ ds, float* __restrict__ dz, size_t n_vec, float Q, int dz_literal) {
+  const uint8_t* const src[2] = {reinterpret_cast<const uint8_t*>(dWhat), reinterpret_cast<const uint8_t*>(W)};
+  stream_chunks<2>(src, n_vec, [&](size_t v0, const uint4 (&raw)[2][2]) {
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const size_t v = v0 + (size_t)u * kConsumers;
+      const bool live = v < n_vec;                      // uniform over the lanes of a group
+      const size_t g = v / LPG;
+      float acc_s = 0.0f, acc_g = 0.0f, sv = 1.0f;
+      if (live) {
+        sv = __ldg(s + g);
+        const float zr = rintf(__ldg(z + g));
+        const float rs = group_rcp(sv);
+        const float lo = -zr, hi = Q - zr;
+        float gr[8], w[8], r[8], rt[8];
+        unpack8(raw[0][u], gr);
+        unpack8(raw[1][u], w);
+        quotient_round8(w, sv, rs, r, rt);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float c = fminf(fmaxf(r[i], lo), hi);
+          const bool inside = (c == r[i]);
+          acc_s = fmaf(gr[i], inside ? rt[i] : c, acc_s);     // Eq. 3
+          acc_g += inside ? 0.0f : gr[i];                      // Eq. 4
+          w[i] = inside ? gr[i] : 0.0f;                        // Eq. 5
+        }
+        reinterpret_cast<uint4*>(dW)[v] = pack8(w);
+      }
+#pragma unroll
+      for (int d = LPG / 2; d >= 1; d >>= 1) {
+        acc_s += __shfl_xor_sync(0xFFFFFFFFu, acc_s, d);
+        acc_g += __shfl_xor_sync(0xFFFFFFFFu, acc_g, d);
+      }
+      if (live && (v % LPG) == 0) {
+        ds[g] = acc_s;
+        if (dz != nullptr) dz[g] = (dz_literal ? -1.0f : -sv) * acc_g;
+      }
+    }
+  });
+}
+
+// Persistent grid: every CTA resident at once, never more CTAs than chunks.
+template <typename K>
+unsigned stream_grid(K kernel, int smem_bytes, size_t n_vec) {
+  int dev = 0, sms = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreadsS, smem_bytes) != cudaSuccess ||
+      sms <= 0 || per_sm <= 0) {
+    (void)cudaGetLastError();
+    return 0;
+  }
+  const size_t chunks = (n_vec + kChunkVec - 1) / kChunkVec;
+  const size_t resident = (size_t)sms * per_sm;
+  return (unsigned)(chunks < resident ? chunks : resident);
+}
+
+template <typename K, typename... Args>
+int launch_stream(K kernel, int smem_bytes, size_t n_vec, cudaStream_t st, Args... args) {
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
+    return EQAT_ERR_CUDA;
+  const unsigned grid = stream_grid(kernel, smem_bytes, n_vec);
+  if (grid == 0) return EQAT_ERR_CUDA;
+  kernel<<<grid, kThreadsS, smem_bytes, st>>>(args...);
+  return launch_status();
+}
+
+}  // namespace
+
+int launch_fakequant_stream(const eqat_desc& d, const eqat_bf16* W, const float* s, const float* z, eqat_bf16* What,
+                            cudaStream_t st) {
+  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
+  const float Q = (float)((1 << d.bits) - 1);
+  int vec_shift = 0;
+  while ((8 << vec_shift) < d.group) ++vec_shift;
+  return launch_stream(fakequant_stream_kernel, Ring<1>::kSmemBytes, n_vec, st, W, s, z, What, n_vec, vec_shift, Q);
+}
+
+int launch_ste_bwd_stream(const eqat_desc& d, const eqat_bf16* dWhat, const eqat_bf16* W, const float* s,
+                          const float* z, eqat_bf16* dW, float* ds, float* dz, cudaStream_t st) {
+  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
+  const float Q = (float)((1 << d.bits) - 1);
+  const int lit = d.dz_mode == 1;
+  constexpr int smem = Ring<2>::kSmemBytes;
+  switch (d.group) {
+    case 32:  return launch_stream(ste_bwd_stream_kernel<4>, smem, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    case 64:  return launch_stream(ste_bwd_stream_kernel<8>, smem, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    case 128: return launch_stream(ste_bwd_stream_kernel<16>, smem, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    default:  return launch_stream(ste_bwd_stream_kernel<32>, smem, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+  }
+}
+
+int read_stream_status(int* status, int* detail) {
+  int h[2] = {0, 0};
+  if (cudaDeviceSynchronize() != cudaSuccess) return EQAT_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(h, g_stream_status, sizeof(h)) != cudaSuccess) return EQAT_ERR_CUDA;
+  const int zero[2] = {0, 0};
+  if (cudaMemcpyToSymbol(g_stream_status, zero, sizeof(zero)) != cudaSuccess) return EQAT_ERR_CUDA;
+  *status = h[0];
+  *detail = h[1];
+  return EQAT_OK;
+}
+
+}  // namespace eqat

@@ -148,6 +148,53 @@ def test_fractional_zero_point_is_rounded(eqat):
     assert torch.equal(A, B)
 
 
+def test_codes_on_exact_and_near_ties(eqat):
+    """Quotients that sit exactly on, and a few ulps beside, a rounding boundary:
+    w = h * base with h running over integers and half-integers (exact in bf16 for
+    a 3-bit base), s = base moved by -3..+3 fp32 ulps.  Codes must equal the
+    oracle's (binary32 division, ties to even) on every element."""
+    bits, group, in_f = 4, 32, 128
+    hs = np.arange(-8.0, 8.5, 0.5, dtype=np.float32)                       # 33 values
+    bases = np.array([0.015625, 0.01953125, 0.0234375, 0.02734375, 0.0390625, 0.046875, 0.0546875, 1.25, 0.4375],
+                     np.float32)
+    rows, s_rows, z_rows = [], [], []
+    for base in bases:
+        for ulps in range(-3, 4):
+            sv = np.float32(base)
+            for _ in range(abs(ulps)):
+                sv = np.nextafter(sv, np.float32(np.inf if ulps > 0 else -np.inf), dtype=np.float32)
+            for zz in (0.0, 7.0):
+                rows.append(np.resize(hs * base, in_f).astype(np.float32))
+                s_rows.append(np.full(in_f // group, sv, np.float32))
+                z_rows.append(np.full(in_f // group, zz, np.float32))
+    while len(rows) % 64:
+        rows.append(rows[0]); s_rows.append(s_rows[0]); z_rows.append(z_rows[0])
+    W32 = np.stack(rows); s = np.stack(s_rows); z = np.stack(z_rows)
+    Wb = to_bf16_bits(W32)
+    assert np.array_equal(f32(Wb), W32)                                    # the weights are exact in bf16
+    out = W32.shape[0]
+    d = eqat.make_desc(bits, group, out, in_f)
+    P = torch.empty(out, in_f * bits // 8, dtype=torch.uint8, device="cuda")
+    z8 = torch.empty(out, in_f // group, dtype=torch.uint8, device="cuda")
+    s16 = torch.empty(out, in_f // group, dtype=torch.float16, device="cuda")
+    eqat.eqat_quantize_pack(d, bits_to_torch(Wb), dev(s), dev(z), P, z8, s16)
+    q_o, _, _ = O.quantize_codes(W32, s, z, bits, group)
+    ties = np.abs(np.abs(W32 / np.repeat(s, group, 1)) % 1.0 - 0.5) < 1e-6
+    assert ties.sum() > 1000
+    codes = torch.empty(out, in_f, dtype=torch.uint8, device="cuda")
+    eqat.eqat_unpack(d, P, codes)
+    assert np.array_equal(codes.cpu().numpy(), q_o.astype(np.uint8))
+    # the fake quantiser and the STE mask take the same decisions
+    What = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
+    eqat.eqat_fakequant_weight(d, bits_to_torch(Wb), dev(s), dev(z), What)
+    assert np.array_equal(torch_to_f64(What), bf16_round(O.dequantize(q_o, s, z, group)).astype(np.float64))
+    G = np.ones_like(W32); dW = torch.empty_like(What)
+    ds = torch.empty(out, in_f // group, device="cuda")
+    eqat.eqat_ste_bwd(d, bits_to_torch(to_bf16_bits(G)), bits_to_torch(Wb), dev(s), dev(z), dW, ds, None)
+    dW_o, _, _ = O.ste_bwd(G, W32, s, z, bits, group)
+    assert np.array_equal(torch_to_f64(dW), dW_o)
+
+
 # --------------------------------------------------------------------------- Block-AP layer
 def run_block_ap(eqat, cfg, lin, tokens, s, z, dz_mode=0):
     Wb = weight_for(cfg, lin); Xb, dYb = activations_for(cfg, lin, tokens)
