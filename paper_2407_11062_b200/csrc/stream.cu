@@ -71,12 +71,16 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-// Runs `body(v, raw)` on every consumer thread for every chunk this CTA owns:
-// v is the index of the thread's first vector, raw[i][u] the thread's vector
-// u (v + u * 256) of input stream i.  Vectors at or beyond n_vec hold stale
-// shared memory and must be ignored by the body.
-template <int NIN, typename Body>
-__device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], size_t n_vec, Body&& body) {
+// Runs `body(v, raw, params)` on every consumer thread for every chunk this CTA
+// owns: v is the index of the thread's first vector, raw[i][u] the thread's
+// vector u (v + u * 256) of input stream i, and params what `fetch(v)` returned
+// for this chunk.  fetch is called one chunk ahead, so the small per-group loads
+// it makes (step size, zero point) are in flight while the previous chunk is
+// being computed instead of stalling this one.  Vectors at or beyond n_vec hold
+// stale shared memory and must be ignored by the body.
+template <int NIN, typename Params, typename Fetch, typename Body>
+__device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], size_t n_vec, Fetch&& fetch,
+                                              Body&& body) {
   using R = Ring<NIN>;
   extern __shared__ __align__(128) uint8_t smem[];
   RingCtl* ctl = reinterpret_cast<RingCtl*>(smem + R::kStages * R::kStageBytes);
@@ -137,7 +141,10 @@ __device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], 
     // ---------------------------------------------------------------- consumers
     int stage = 0;
     uint32_t phase = 0;
+    Params next = fetch((size_t)blockIdx.x * kChunkVec + threadIdx.x);
     for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+      const Params cur = next;
+      if (chunk + gridDim.x < n_chunks) next = fetch((chunk + gridDim.x) * kChunkVec + threadIdx.x);
       if (!ring_wait(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL, 0)) break;
       uint4 raw[NIN][2];
       const uint8_t* st = smem + stage * R::kStageBytes;
@@ -149,7 +156,7 @@ __device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], 
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->empty[stage]));   // the stage can be refilled now
       if (++stage == R::kStages) { stage = 0; phase ^= 1u; }
-      body(chunk * kChunkVec + threadIdx.x, raw);
+      body(chunk * kChunkVec + threadIdx.x, raw, cur);
     }
   }
 }
@@ -187,10 +194,11 @@ __device__ __forceinline__ float group_rcp(float s) {
 //   1.5 * 2^-23 |q|.  r0 = rint(w*rs) (one fused multiply-add with 1.5 * 2^23,
 //   which rounds the exact product half-to-even, then a subtraction) can differ
 //   from rint(rn(w/s)) only if a half-integer lies between the two values; for
-//   |q| <= 512 that needs w*rs within 2^-13 of a half-integer.
+//   |q| <= 32.5 that needs w*rs within 1.5 * 2^-23 * 32.5 < 2^-17 of a half-integer.
 //   d = w*rs - r0 (one more fused multiply-add) is the distance to the integer.
-//   Unless every element of the vector has |d| < 0.5 - 2^-12 and |r0| <= 512,
-//   the whole vector is redone with the exact sequence (rare).
+//   Unless every element of the vector has |d| < 0.5 - 2^-17 and |r0| <= 32,
+//   the whole vector is redone with the exact sequence (about one vector in
+//   eight thousand on in-range weights; always for quotients far out of range).
 // The STE term r - w/s is returned as -d in the common case (2^-23 relative away
 // from the exact one, immaterial for a gradient).
 __device__ __forceinline__ void quotient_round8(const float (&w)[8], float s, float rs, float (&r)[8],
@@ -205,7 +213,7 @@ __device__ __forceinline__ void quotient_round8(const float (&w)[8], float s, fl
     dmax = fmaxf(dmax, fabsf(d));
     rmax = fmaxf(rmax, fabsf(r0));
   }
-  if (!(dmax < 0.499755859375f && rmax <= 512.0f)) {      // also taken when anything is NaN
+  if (!(dmax < 0.49999237060546875f && rmax <= 32.0f)) {   // also taken when anything is NaN
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float q = __fdiv_rn(w[i], s);
@@ -215,20 +223,42 @@ __device__ __forceinline__ void quotient_round8(const float (&w)[8], float s, fl
   }
 }
 
+// Step size and zero point of the groups of a thread's two vectors.
+struct GroupParams {
+  float s[2], z[2];
+};
+
+__device__ __forceinline__ GroupParams fetch_groups(const float* __restrict__ s, const float* __restrict__ z,
+                                                    size_t v0, size_t n_vec, int vec_shift) {
+  GroupParams p;
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const size_t v = v0 + (size_t)u * kConsumers;
+    p.s[u] = 1.0f;
+    p.z[u] = 0.0f;
+    if (v < n_vec) {
+      p.s[u] = __ldg(s + (v >> vec_shift));
+      p.z[u] = __ldg(z + (v >> vec_shift));
+    }
+  }
+  return p;
+}
+
 // ------------------------------------------------------------------ Eq. 1 + Eq. 2
 // (clamp(r + z, 0, Q) - z) * s == clamp(r, -z, Q - z) * s for integer r and z.
 __global__ void __launch_bounds__(kThreadsS)
 fakequant_stream_kernel(const eqat_bf16* __restrict__ W, const float* __restrict__ s, const float* __restrict__ z,
                         eqat_bf16* __restrict__ What, size_t n_vec, int vec_shift, float Q) {
   const uint8_t* const src[1] = {reinterpret_cast<const uint8_t*>(W)};
-  stream_chunks<1>(src, n_vec, [&](size_t v0, const uint4 (&raw)[1][2]) {
+  stream_chunks<1, GroupParams>(src, n_vec,
+      [&](size_t v0) { return fetch_groups(s, z, v0, n_vec, vec_shift); },
+      [&](size_t v0, const uint4 (&raw)[1][2], const GroupParams& gp) {
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       const size_t v = v0 + (size_t)u * kConsumers;
       if (v < n_vec) {
-        const size_t g = v >> vec_shift;
-        const float sv = __ldg(s + g);
-        const float zr = rintf(__ldg(z + g));
+        const float sv = gp.s[u];
+        const float zr = rintf(gp.z[u]);
         const float rs = group_rcp(sv);
         const float lo = -zr, hi = Q - zr;
         float w[8], r[8], rt[8];
@@ -253,16 +283,19 @@ ste_bwd_stream_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __re
                       const float* __restrict__ s, const float* __restrict__ z, eqat_bf16* __restrict__ dW,
                       float* __restrict__ ds, float* __restrict__ dz, size_t n_vec, float Q, int dz_literal) {
   const uint8_t* const src[2] = {reinterpret_cast<const uint8_t*>(dWhat), reinterpret_cast<const uint8_t*>(W)};
-  stream_chunks<2>(src, n_vec, [&](size_t v0, const uint4 (&raw)[2][2]) {
+  constexpr int vec_shift = LPG == 4 ? 2 : LPG == 8 ? 3 : LPG == 16 ? 4 : 5;
+  stream_chunks<2, GroupParams>(src, n_vec,
+      [&](size_t v0) { return fetch_groups(s, z, v0, n_vec, vec_shift); },
+      [&](size_t v0, const uint4 (&raw)[2][2], const GroupParams& gp) {
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       const size_t v = v0 + (size_t)u * kConsumers;
       const bool live = v < n_vec;                      // uniform over the lanes of a group
       const size_t g = v / LPG;
-      float acc_s = 0.0f, acc_g = 0.0f, sv = 1.0f;
+      float acc_s = 0.0f, acc_g = 0.0f;
+      const float sv = gp.s[u];
       if (live) {
-        sv = __ldg(s + g);
-        const float zr = rintf(__ldg(z + g));
+        const float zr = rintf(gp.z[u]);
         const float rs = group_rcp(sv);
         const float lo = -zr, hi = Q - zr;
         float gr[8], w[8], r[8], rt[8];
