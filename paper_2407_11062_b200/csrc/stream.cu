@@ -6,12 +6,12 @@
 // store" thread keeps its loads in flight only until its arithmetic starts,
 // and the arithmetic here is long (a division-free but exact quantiser per
 // element).  So the loads are taken out of the compute threads: each persistent
-// CTA has one producer thread that streams 8 KB chunks of the input(s) into a
-// shared-memory ring with bulk asynchronous copies (cp.async.bulk, completion
-// on an mbarrier), several chunks ahead, while 8 consumer warps pull 16-byte
-// vectors from the ring, compute, and write results to global memory with
-// coalesced 16-byte stores.  Three CTAs fit on an SM, so about 150 KB of reads
-// are in flight per SM whatever the consumers are doing.
+// CTA has one producer thread that streams 8-16 KB chunks of the input(s) into
+// a four-stage shared-memory ring with bulk asynchronous copies (cp.async.bulk,
+// completion on an mbarrier), several chunks ahead, while 8 consumer warps pull
+// 16-byte vectors from the ring, compute, and write results to global memory
+// with coalesced 16-byte stores.  Three CTAs fit on an SM, so 150-190 KB of
+// reads are in flight per SM whatever the consumers are doing.
 //
 // A quantisation group is contiguous in the flattened weight and owned by
 // group/8 adjacent lanes of one warp; group sums are fixed-order shuffles, so
@@ -28,13 +28,16 @@ namespace {
 
 constexpr int kConsumers = 256;
 constexpr int kThreadsS = kConsumers + 32;           // + one producer warp
-constexpr int kChunkVec = 2 * kConsumers;            // 16-byte vectors per chunk and stream (8 KB)
-constexpr int kChunkBytes = kChunkVec * 16;
+// VPT = 16-byte vectors per consumer thread and chunk (a chunk is VPT * 4 KB per
+// input stream): 4 for the one-input fake quantiser, 2 for the two-input STE
+// backward, whose consumers need twice the registers per vector.
 constexpr uint64_t kStreamWaitLimitNs = 2000000000ull;
 
-template <int NIN>
+template <int NIN, int VPT>
 struct Ring {
-  static constexpr int kStages = NIN == 1 ? 6 : 4;
+  static constexpr int kChunkVec = VPT * kConsumers;          // vectors per chunk and stream
+  static constexpr int kChunkBytes = kChunkVec * 16;
+  static constexpr int kStages = 4;
   static constexpr int kStageBytes = NIN * kChunkBytes;
   static constexpr int kSmemBytes = kStages * kStageBytes + 256;
 };
@@ -78,10 +81,11 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 // it makes (step size, zero point) are in flight while the previous chunk is
 // being computed instead of stalling this one.  Vectors at or beyond n_vec hold
 // stale shared memory and must be ignored by the body.
-template <int NIN, typename Params, typename Fetch, typename Body>
+template <int NIN, int VPT, typename Params, typename Fetch, typename Body>
 __device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], size_t n_vec, Fetch&& fetch,
                                               Body&& body) {
-  using R = Ring<NIN>;
+  using R = Ring<NIN, VPT>;
+  constexpr int kChunkVec = R::kChunkVec, kChunkBytes = R::kChunkBytes;
   extern __shared__ __align__(128) uint8_t smem[];
   RingCtl* ctl = reinterpret_cast<RingCtl*>(smem + R::kStages * R::kStageBytes);
   volatile int* abort_flag = &ctl->abort;
@@ -146,12 +150,12 @@ __device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], 
       const Params cur = next;
       if (chunk + gridDim.x < n_chunks) next = fetch((chunk + gridDim.x) * kChunkVec + threadIdx.x);
       if (!ring_wait(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL, 0)) break;
-      uint4 raw[NIN][2];
+      uint4 raw[NIN][VPT];
       const uint8_t* st = smem + stage * R::kStageBytes;
 #pragma unroll
       for (int i = 0; i < NIN; ++i)
 #pragma unroll
-        for (int u = 0; u < 2; ++u)
+        for (int u = 0; u < VPT; ++u)
           raw[i][u] = *reinterpret_cast<const uint4*>(st + i * kChunkBytes + (u * kConsumers + threadIdx.x) * 16);
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->empty[stage]));   // the stage can be refilled now
@@ -223,16 +227,20 @@ __device__ __forceinline__ void quotient_round8(const float (&w)[8], float s, fl
   }
 }
 
-// Step size and zero point of the groups of a thread's two vectors.
+constexpr int kFakequantVpt = 4, kSteVpt = 2;
+
+// Step size and zero point of the groups of a thread's vectors.
+template <int VPT>
 struct GroupParams {
-  float s[2], z[2];
+  float s[VPT], z[VPT];
 };
 
-__device__ __forceinline__ GroupParams fetch_groups(const float* __restrict__ s, const float* __restrict__ z,
+template <int VPT>
+__device__ __forceinline__ GroupParams<VPT> fetch_groups(const float* __restrict__ s, const float* __restrict__ z,
                                                     size_t v0, size_t n_vec, int vec_shift) {
-  GroupParams p;
+  GroupParams<VPT> p;
 #pragma unroll
-  for (int u = 0; u < 2; ++u) {
+  for (int u = 0; u < VPT; ++u) {
     const size_t v = v0 + (size_t)u * kConsumers;
     p.s[u] = 1.0f;
     p.z[u] = 0.0f;
@@ -250,11 +258,12 @@ __global__ void __launch_bounds__(kThreadsS)
 fakequant_stream_kernel(const eqat_bf16* __restrict__ W, const float* __restrict__ s, const float* __restrict__ z,
                         eqat_bf16* __restrict__ What, size_t n_vec, int vec_shift, float Q) {
   const uint8_t* const src[1] = {reinterpret_cast<const uint8_t*>(W)};
-  stream_chunks<1, GroupParams>(src, n_vec,
-      [&](size_t v0) { return fetch_groups(s, z, v0, n_vec, vec_shift); },
-      [&](size_t v0, const uint4 (&raw)[1][2], const GroupParams& gp) {
+  constexpr int VPT = kFakequantVpt;
+  stream_chunks<1, VPT, GroupParams<VPT>>(src, n_vec,
+      [&](size_t v0) { return fetch_groups<VPT>(s, z, v0, n_vec, vec_shift); },
+      [&](size_t v0, const uint4 (&raw)[1][VPT], const GroupParams<VPT>& gp) {
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < VPT; ++u) {
       const size_t v = v0 + (size_t)u * kConsumers;
       if (v < n_vec) {
         const float sv = gp.s[u];
@@ -284,11 +293,12 @@ ste_bwd_stream_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __re
                       float* __restrict__ ds, float* __restrict__ dz, size_t n_vec, float Q, int dz_literal) {
   const uint8_t* const src[2] = {reinterpret_cast<const uint8_t*>(dWhat), reinterpret_cast<const uint8_t*>(W)};
   constexpr int vec_shift = LPG == 4 ? 2 : LPG == 8 ? 3 : LPG == 16 ? 4 : 5;
-  stream_chunks<2, GroupParams>(src, n_vec,
-      [&](size_t v0) { return fetch_groups(s, z, v0, n_vec, vec_shift); },
-      [&](size_t v0, const uint4 (&raw)[2][2], const GroupParams& gp) {
+  constexpr int VPT = kSteVpt;
+  stream_chunks<2, VPT, GroupParams<VPT>>(src, n_vec,
+      [&](size_t v0) { return fetch_groups<VPT>(s, z, v0, n_vec, vec_shift); },
+      [&](size_t v0, const uint4 (&raw)[2][VPT], const GroupParams<VPT>& gp) {
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < VPT; ++u) {
       const size_t v = v0 + (size_t)u * kConsumers;
       const bool live = v < n_vec;                      // uniform over the lanes of a group
       const size_t g = v / LPG;
@@ -327,7 +337,7 @@ ste_bwd_stream_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __re
 
 // Persistent grid: every CTA resident at once, never more CTAs than chunks.
 template <typename K>
-unsigned stream_grid(K kernel, int smem_bytes, size_t n_vec) {
+unsigned stream_grid(K kernel, int smem_bytes, size_t n_vec, int chunk_vec) {
   int dev = 0, sms = 0, per_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
@@ -336,16 +346,16 @@ unsigned stream_grid(K kernel, int smem_bytes, size_t n_vec) {
     (void)cudaGetLastError();
     return 0;
   }
-  const size_t chunks = (n_vec + kChunkVec - 1) / kChunkVec;
+  const size_t chunks = (n_vec + chunk_vec - 1) / chunk_vec;
   const size_t resident = (size_t)sms * per_sm;
   return (unsigned)(chunks < resident ? chunks : resident);
 }
 
 template <typename K, typename... Args>
-int launch_stream(K kernel, int smem_bytes, size_t n_vec, cudaStream_t st, Args... args) {
+int launch_stream(K kernel, int smem_bytes, int chunk_vec, size_t n_vec, cudaStream_t st, Args... args) {
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
     return EQAT_ERR_CUDA;
-  const unsigned grid = stream_grid(kernel, smem_bytes, n_vec);
+  const unsigned grid = stream_grid(kernel, smem_bytes, n_vec, chunk_vec);
   if (grid == 0) return EQAT_ERR_CUDA;
   kernel<<<grid, kThreadsS, smem_bytes, st>>>(args...);
   return launch_status();
@@ -359,7 +369,8 @@ int launch_fakequant_stream(const eqat_desc& d, const eqat_bf16* W, const float*
   const float Q = (float)((1 << d.bits) - 1);
   int vec_shift = 0;
   while ((8 << vec_shift) < d.group) ++vec_shift;
-  return launch_stream(fakequant_stream_kernel, Ring<1>::kSmemBytes, n_vec, st, W, s, z, What, n_vec, vec_shift, Q);
+  using R = Ring<1, kFakequantVpt>;
+  return launch_stream(fakequant_stream_kernel, R::kSmemBytes, R::kChunkVec, n_vec, st, W, s, z, What, n_vec, vec_shift, Q);
 }
 
 int launch_ste_bwd_stream(const eqat_desc& d, const eqat_bf16* dWhat, const eqat_bf16* W, const float* s,
@@ -367,12 +378,13 @@ int launch_ste_bwd_stream(const eqat_desc& d, const eqat_bf16* dWhat, const eqat
   const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
   const float Q = (float)((1 << d.bits) - 1);
   const int lit = d.dz_mode == 1;
-  constexpr int smem = Ring<2>::kSmemBytes;
+  using R = Ring<2, kSteVpt>;
+  constexpr int smem = R::kSmemBytes, cv = R::kChunkVec;
   switch (d.group) {
-    case 32:  return launch_stream(ste_bwd_stream_kernel<4>, smem, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
-    case 64:  return launch_stream(ste_bwd_stream_kernel<8>, smem, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
-    case 128: return launch_stream(ste_bwd_stream_kernel<16>, smem, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
-    default:  return launch_stream(ste_bwd_stream_kernel<32>, smem, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    case 32:  return launch_stream(ste_bwd_stream_kernel<4>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    case 64:  return launch_stream(ste_bwd_stream_kernel<8>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    case 128: return launch_stream(ste_bwd_stream_kernel<16>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    default:  return launch_stream(ste_bwd_stream_kernel<32>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
   }
 }
 
