@@ -16,9 +16,14 @@
 //   warp 1      MMA issuer: one thread issues tcgen05.mma into one of two TMEM
 //               accumulators, frees stages with tcgen05.commit
 //   warps 2-5   epilogue: tcgen05.ld the finished accumulator (one TMEM lane
-//               quadrant each) while the next tile is already being multiplied
-//   warps 6-13  (packed-weight kernels only) expand N-bit codes into the bf16 B
-//               operand stage: (q - z) * s exactly in fp32, rounded once to bf16
+//               quadrant each); with MT = 1 the next tile is already being
+//               multiplied meanwhile
+//   warps 2-17  (packed-weight kernels only) expand N-bit codes into the bf16 B
+//               operand stage, (q - z) * s exactly, rounded once to bf16; sixteen
+//               warps because the expansion is latency-bound per warp.  Warps
+//               2-5 then run the epilogue of the tile (MT = 2: nothing overlaps it
+//               anyway, and the other twelve warps meanwhile pre-expand the next
+//               tile's first stages up to the point where they need these four)
 // The epilogue either stores the tile as bf16 or, for the E2E-QP step-size
 // gradient, multiplies each accumulator row by (q - z) of the matching packed
 // codes and reduces runs of `group` columns, so the [out,in] weight gradient
@@ -43,8 +48,8 @@ namespace {
 constexpr int BM = 128;          // rows per MMA = TMEM lanes
 constexpr int BK = 64;           // K per stage: one 128-byte swizzle span of bf16
 constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit inputs
-constexpr int kDeqWarp0 = 6;
-constexpr int kDeqWarps = 8;
+constexpr int kEpiWarps = 4;       // dense kernels: warps 2-5 are the epilogue
+constexpr int kDeqWarps = 16;      // packed kernels: warps 2-17 expand codes; warps 2-5 also run the epilogue
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s per wait
 constexpr uint64_t kDrainLimitNs = 50000000ull;    // 50 ms per stage at teardown
 
@@ -71,7 +76,7 @@ struct Cfg {
   static constexpr int kABytes = kTileM * BK * 2;
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kThreads = PACKED ? (kDeqWarp0 + kDeqWarps) * 32 : kDeqWarp0 * 32;
+  static constexpr int kThreads = (2 + (PACKED ? kDeqWarps : kEpiWarps)) * 32;
   static constexpr int kTmemCols = kAccSets * MT * BN;
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
@@ -151,9 +156,10 @@ __device__ __forceinline__ void store_chunk(uint8_t* row, int chunk, int rx, con
   *reinterpret_cast<uint4*>(row + ((chunk ^ rx) << 4)) = o;
 }
 
+// Expands 32 consecutive codes (half h of a 64-code row) into chunks 4h .. 4h+3.
 template <int BITS>
-__device__ __forceinline__ void dequant_row64(const uint32_t (&w)[2 * BITS], float s, float z, uint8_t* row, int rx) {
-  const DequantScale f(s, z);
+__device__ __forceinline__ void dequant_half32(const uint32_t (&w)[BITS], float s, float z, uint8_t* row, int rx,
+                                               int h) {
   constexpr uint32_t kMagic = 0x4B000000u;
   if constexpr (BITS == 2) {
     // Four possible values per group: build them once, exactly, as bf16
@@ -165,7 +171,7 @@ __device__ __forceinline__ void dequant_row64(const uint32_t (&w)[2 * BITS], flo
     const uint32_t lut01 = pack_bf16x2(-zs, s - zs);
     const uint32_t lut23 = pack_bf16x2(fmaf(2.0f, s, -zs), fmaf(3.0f, s, -zs));
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {                       // word i: codes 16i .. 16i+15
+    for (int i = 0; i < 2; ++i) {                       // word i: codes 16i .. 16i+15 of the half
       uint32_t sel[4];                                  // byte b of sel[r] = selector byte of code 4b + r
 #pragma unroll
       for (int r = 0; r < 4; ++r) sel[r] = ((w[i] >> (2 * r)) & 0x03030303u) * 0x22u + 0x10101010u;
@@ -179,60 +185,54 @@ __device__ __forceinline__ void dequant_row64(const uint32_t (&w)[2 * BITS], flo
           const uint32_t pair_sel = __byte_perm(sel[r], sel[r + 1], b | ((4u + b) << 4));
           o[pr] = __byte_perm(lut01, lut23, pair_sel);
         }
-        *reinterpret_cast<uint4*>(row + (((2 * i + c) ^ rx) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<uint4*>(row + (((4 * h + 2 * i + c) ^ rx) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
   } else if constexpr (BITS == 4) {
+    const DequantScale f(s, z);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {                       // word i: codes 8i .. 8i+7
+    for (int i = 0; i < 4; ++i) {                       // word i: codes 8i .. 8i+7 of the half
       const uint32_t m0 = w[i] & 0x0F0F0F0Fu, m1 = (w[i] >> 4) & 0x0F0F0F0Fu;   // byte b = code 2b (+1)
       float v[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e)
         v[e] = f(__byte_perm((e & 1) ? m1 : m0, kMagic, 0x7044u | ((uint32_t)(e >> 1) << 8)));
-      store_chunk(row, i, rx, v);
+      store_chunk(row, 4 * h + i, rx, v);
     }
   } else {
+    const DequantScale f(s, z);
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {                       // 32 codes = 3 words
+    for (int c = 0; c < 4; ++c) {                       // 32 codes = 3 words
+      float v[8];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float v[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int bit = 3 * (8 * c + e), word = bit >> 5, off = bit & 31;
-          uint32_t t;
-          if (off <= 16) {
-            t = w[3 * h + word] << (16 - off);
-          } else {
-            const uint32_t hi = (off + 3 > 32) ? w[3 * h + word + 1] : 0u;
-            t = __funnelshift_r(w[3 * h + word], hi, off - 16);
-          }
-          v[e] = f((t & 0x00070000u) | kMagic);
+      for (int e = 0; e < 8; ++e) {
+        const int bit = 3 * (8 * c + e), word = bit >> 5, off = bit & 31;
+        uint32_t t;
+        if (off <= 16) {
+          t = w[word] << (16 - off);
+        } else {
+          const uint32_t hi = (off + 3 > 32) ? w[word + 1] : 0u;
+          t = __funnelshift_r(w[word], hi, off - 16);
         }
-        store_chunk(row, 4 * h + c, rx, v);
+        v[e] = f((t & 0x00070000u) | kMagic);
       }
+      store_chunk(row, 4 * h + c, rx, v);
     }
   }
 }
 
+// 32 codes = BITS consecutive 32-bit words, at a multiple of 4*BITS bytes.
 template <int BITS>
-__device__ __forceinline__ void load_codes64(const uint8_t* p, uint32_t (&w)[2 * BITS]) {
+__device__ __forceinline__ void load_codes32(const uint8_t* p, uint32_t (&w)[BITS]) {
   if constexpr (BITS == 2) {
-    const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
-    w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+    w[0] = t.x; w[1] = t.y;
   } else if constexpr (BITS == 3) {
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {
-      const uint2 t = __ldg(reinterpret_cast<const uint2*>(p) + i);
-      w[2 * i] = t.x; w[2 * i + 1] = t.y;
-    }
+    for (int i = 0; i < 3; ++i) w[i] = __ldg(reinterpret_cast<const uint32_t*>(p) + i);
   } else {
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const uint4 t = __ldg(reinterpret_cast<const uint4*>(p) + i);
-      w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
-    }
+    const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
+    w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
   }
 }
 
@@ -281,6 +281,86 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+
+  // ---------------------------------------------------------------- epilogue of one tile
+  // Run by four warps, one per TMEM lane quadrant (warp index mod 4).
+  const int quad = warp & 3;
+  const int row_in_tile = quad * 32 + lane;
+  auto epilogue_tile = [&](int m_blk, int n_blk, int acc, uint32_t acc_phase) -> bool {
+    if (!wait_bounded(ptx::smem_addr(&ctl->acc_full[acc]), acc_phase, abort_flag, WAIT_EPI_ACC_FULL,
+                      PACKED ? 0 : (MT == 2 ? 512 : 128)))
+      return false;
+    ptx::tc_fence_after();
+#pragma unroll 1
+    for (int h = 0; h < MT; ++h) {
+      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MT + h) * BN);
+      const int m = m_blk * C::kTileM + h * BM + row_in_tile;
+      if constexpr (EPI == EPI_STORE) {
+        eqat_bf16* drow = p.D + (size_t)m * p.N;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32(t_row + c * 32, r);
+          ptx::tmem_ld_wait();
+          const int col0 = n_blk * BN + c * 32;
+          if (m < p.M) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              if (col0 + v * 8 < p.N) {
+                const uint4 o = make_uint4(
+                    pack_bf16x2(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1])),
+                    pack_bf16x2(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3])),
+                    pack_bf16x2(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5])),
+                    pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])));
+                *reinterpret_cast<uint4*>(drow + col0 + v * 8) = o;
+              }
+            }
+          }
+        }
+      } else {
+        // Row m of the tile is output row o = m of the weight; columns are input
+        // features.  ds[o,g] = sum_{j in g} G[o,j] * (q[o,j] - z[o,g]).
+        const int groups_per_row = p.in_features >> p.group_shift;
+        const int chunks_per_group = 1 << (p.group_shift - 5);
+        const uint8_t* qrow = p.Wq + (size_t)m * ((size_t)p.in_features * BITS / 8);
+        float acc_s = 0.0f, acc_g = 0.0f;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32(t_row + c * 32, r);
+          ptx::tmem_ld_wait();
+          const int col0 = n_blk * BN + c * 32;
+          if (m < p.M && col0 < p.N) {
+            uint32_t words[BITS];
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(qrow) + (size_t)(col0 >> 5) * BITS;
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) words[i] = __ldg(src + i);
+            uint32_t codes[32];
+            unpack32<BITS>(words, codes);
+            const int g = col0 >> p.group_shift;
+            const float zf = (float)__ldg(p.z8 + (size_t)m * groups_per_row + g);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float gv = __uint_as_float(r[i]);
+              acc_s = fmaf(gv, (float)codes[i] - zf, acc_s);
+              acc_g += gv;
+            }
+            if (((c + 1) & (chunks_per_group - 1)) == 0) {
+              const size_t idx = (size_t)m * groups_per_row + g;
+              p.ds[idx] = acc_s;
+              if (p.dz != nullptr) p.dz[idx] = -__half2float(__ushort_as_half(__ldg(p.s16 + idx))) * acc_g;
+              acc_s = 0.0f;
+              acc_g = 0.0f;
+            }
+          }
+        }
+      }
+    }
+    ptx::tc_fence_before();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[acc]));
+    return true;
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -381,133 +461,102 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::mma_commit(ptx::smem_addr(&ctl->drain));
       wait_bounded(ptx::smem_addr(&ctl->drain), 0u, abort_flag, WAIT_TEARDOWN, 64, kDrainLimitNs * 4);
     }
-  } else if (warp < kDeqWarp0) {
-    // ------------------------------------------------------------ epilogue
-    const int quad = warp & 3;                        // TMEM lane quadrant this warp may read
-    const int row_in_tile = quad * 32 + lane;
+  } else if (!PACKED) {
+    // ------------------------------------------------------------ epilogue warps (dense kernels)
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
       int m_blk, n_blk;
       tile_coords(tile, num_m, num_n, m_blk, n_blk);
-      if (!wait_bounded(ptx::smem_addr(&ctl->acc_full[acc]), acc_phase, abort_flag, WAIT_EPI_ACC_FULL, MT == 2 ? 512 : 128)) break;
-      ptx::tc_fence_after();
-#pragma unroll 1
-      for (int h = 0; h < MT; ++h) {
-        const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MT + h) * BN);
-        const int m = m_blk * C::kTileM + h * BM + row_in_tile;
-        if constexpr (EPI == EPI_STORE) {
-          eqat_bf16* drow = p.D + (size_t)m * p.N;
-#pragma unroll 1
-          for (int c = 0; c < BN / 32; ++c) {
-            uint32_t r[32];
-            ptx::tmem_ld_32x32(t_row + c * 32, r);
-            ptx::tmem_ld_wait();
-            const int col0 = n_blk * BN + c * 32;
-            if (m < p.M) {
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                if (col0 + v * 8 < p.N) {
-                  const uint4 o = make_uint4(
-                      pack_bf16x2(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1])),
-                      pack_bf16x2(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3])),
-                      pack_bf16x2(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5])),
-                      pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])));
-                  *reinterpret_cast<uint4*>(drow + col0 + v * 8) = o;
-                }
-              }
-            }
-          }
-        } else {
-          // Row m of the tile is output row o = m of the weight; columns are input
-          // features.  ds[o,g] = sum_{j in g} G[o,j] * (q[o,j] - z[o,g]).
-          const int groups_per_row = p.in_features >> p.group_shift;
-          const int chunks_per_group = 1 << (p.group_shift - 5);
-          const uint8_t* qrow = p.Wq + (size_t)m * ((size_t)p.in_features * BITS / 8);
-          float acc_s = 0.0f, acc_g = 0.0f;
-#pragma unroll 1
-          for (int c = 0; c < BN / 32; ++c) {
-            uint32_t r[32];
-            ptx::tmem_ld_32x32(t_row + c * 32, r);
-            ptx::tmem_ld_wait();
-            const int col0 = n_blk * BN + c * 32;
-            if (m < p.M && col0 < p.N) {
-              uint32_t words[BITS];
-              const uint32_t* src = reinterpret_cast<const uint32_t*>(qrow) + (size_t)(col0 >> 5) * BITS;
-#pragma unroll
-              for (int i = 0; i < BITS; ++i) words[i] = __ldg(src + i);
-              uint32_t codes[32];
-              unpack32<BITS>(words, codes);
-              const int g = col0 >> p.group_shift;
-              const float zf = (float)__ldg(p.z8 + (size_t)m * groups_per_row + g);
-#pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const float gv = __uint_as_float(r[i]);
-                acc_s = fmaf(gv, (float)codes[i] - zf, acc_s);
-                acc_g += gv;
-              }
-              if (((c + 1) & (chunks_per_group - 1)) == 0) {
-                const size_t idx = (size_t)m * groups_per_row + g;
-                p.ds[idx] = acc_s;
-                if (p.dz != nullptr) p.dz[idx] = -__half2float(__ushort_as_half(__ldg(p.s16 + idx))) * acc_g;
-                acc_s = 0.0f;
-                acc_g = 0.0f;
-              }
-            }
-          }
-        }
-      }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[acc]));
+      if (!epilogue_tile(m_blk, n_blk, acc, acc_phase)) break;
       if (++acc == C::kAccSets) { acc = 0; acc_phase ^= 1u; }
     }
   } else {
-    // ------------------------------------------------------------ dequantiser (PACKED only)
+    // ------------------------------------------------------------ dequantisers (+ epilogue on warps 2-5)
     if constexpr (PACKED) {
-      const int t = threadIdx.x - kDeqWarp0 * 32;                 // 0..255, one 64-code unit per stage
+      const int t = threadIdx.x - 64;                             // 0..511, one 32-code half unit per stage
       const size_t pitch = (size_t)p.in_features * BITS / 8;      // bytes per packed row
       const int groups_per_row = p.in_features >> p.group_shift;
       const int chunks_in = p.in_features >> 6;                   // 64-code units per row
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      // unit -> (weight row, 64-code unit in the row, shared-memory row)
-      //   B K-major  (Y):  tile row n = t is weight row n0 + t, unit = kb
-      //   B MN-major (dX): k-row kr is weight row kb*64 + kr, unit = n0/64 + box (64-column box).
-      // The 8 lanes of a quarter-warp (one 16-byte store wavefront) always own 8
-      // consecutive rows, whose swizzled chunks fall in 8 different bank groups.
-      const int kr = (t & 7) | ((t >> 5) << 3);                   // MN-major: k-row 0..63
-      const int box = (t >> 3) & 3;                               // MN-major: 64-column box 0..3
-      const int smem_row_off = B_MN ? (box * (BK * 128) + kr * 128) : t * 128;
-      const int rx = B_MN ? (kr & 7) : (t & 7);
+      // A 64-code unit is one 128-byte shared-memory row; a thread expands half h of it.
+      //   B K-major  (Y):  tile row n is weight row n0 + n, unit = kb
+      //   B MN-major (dX): k-row kr is weight row kb*64 + kr, unit = n0/64 + box (64-column box)
+      // The 8 lanes of a quarter-warp (one 16-byte store wavefront) own the same
+      // half of 8 consecutive rows, whose swizzled chunks fall in 8 different bank groups.
+      const int h = (t >> 3) & 1;
+      const int n_row = (t & 7) | ((t >> 4) << 3);                // K-major: tile row 0..255
+      const int kr = (t & 7) | ((t >> 6) << 3);                   // MN-major: k-row 0..63
+      const int box = (t >> 4) & 3;                               // MN-major: 64-column box 0..3
+      const int smem_row_off = B_MN ? (box * (BK * 128) + kr * 128) : n_row * 128;
+      const int rx = B_MN ? (kr & 7) : (n_row & 7);
       struct Unit {
-        uint32_t w[2 * BITS];
+        uint32_t w[BITS];
         float s, z;
         bool valid;
       };
+      // Step sizes and zero points.  With a K-major B operand a thread stays on one
+      // weight row for a whole tile and walks its groups in order, so it reads
+      // them four groups at a time (one 8-byte and one 4-byte load per four
+      // groups, a block ahead of use) instead of one 2-byte and one 1-byte load
+      // per K block: 32 lanes on 32 different rows make every such load 32
+      // separate L1 transactions, and those were what bounded the kernel.
+      const bool sz_blocks = !B_MN && (groups_per_row & 3) == 0;
+      struct SzBlock {
+        uint2 s4;
+        uint32_t z4;
+      };
+      SzBlock sz_cur = {make_uint2(0u, 0u), 0u}, sz_nxt = {make_uint2(0u, 0u), 0u};
+      int sz_blk = -1;
+      auto fetch_sz = [&](SzBlock& b, int n_blk, int blk) {
+        const int wrow = n_blk * BN + n_row;
+        if (wrow < p.out_features && blk * 4 < groups_per_row) {
+          const size_t gi = (size_t)wrow * groups_per_row + (size_t)blk * 4;
+          b.s4 = __ldg(reinterpret_cast<const uint2*>(p.s16 + gi));
+          b.z4 = __ldg(reinterpret_cast<const uint32_t*>(p.z8 + gi));
+        }
+      };
       auto fetch = [&](Unit& u, int n_blk, int kb) {
-        const int wrow = B_MN ? kb * BK + kr : n_blk * BN + t;
+        const int wrow = B_MN ? kb * BK + kr : n_blk * BN + n_row;
         const int unit = B_MN ? n_blk * (BN / 64) + box : kb;
         u.valid = wrow < p.out_features && unit < chunks_in;
         if (u.valid) {
-          load_codes64<BITS>(p.Wq + (size_t)wrow * pitch + (size_t)unit * (8 * BITS), u.w);
-          const size_t gi = (size_t)wrow * groups_per_row + ((unit << 6) >> p.group_shift);
-          u.s = __half2float(__ushort_as_half(__ldg(p.s16 + gi)));
-          u.z = (float)__ldg(p.z8 + gi);
+          load_codes32<BITS>(p.Wq + (size_t)wrow * pitch + (size_t)(2 * unit + h) * (4 * BITS), u.w);
+          if (!sz_blocks) {
+            const size_t gi = (size_t)wrow * groups_per_row + ((unit << 6) >> p.group_shift);
+            u.s = __half2float(__ushort_as_half(__ldg(p.s16 + gi)));
+            u.z = (float)__ldg(p.z8 + gi);
+          }
         }
       };
       // Register ring of units: the loads for K block kb + kRing are issued as soon
       // as block kb has been expanded, so they have kRing - 1 whole stages to land.
       constexpr int kRing = 4;
       Unit ring[kRing];
+      int acc = 0;
+      uint32_t acc_phase = 0;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
         tile_coords(tile, num_m, num_n, m_blk, n_blk);
 #pragma unroll
         for (int j = 0; j < kRing; ++j)
           if (j < num_kb) fetch(ring[j], n_blk, j);
+        if (sz_blocks) {
+          fetch_sz(sz_cur, n_blk, 0);
+          fetch_sz(sz_nxt, n_blk, 1);
+          sz_blk = 0;
+        }
         for (int kb0 = 0; kb0 < num_kb && ok; kb0 += kRing) {
+          if (sz_blocks) {
+            const int blk = ((kb0 << 6) >> p.group_shift) >> 2;      // constant over the kRing blocks below
+            if (blk != sz_blk) {
+              sz_cur = sz_nxt;
+              sz_blk = blk;
+              fetch_sz(sz_nxt, n_blk, blk + 1);
+            }
+          }
 #pragma unroll
           for (int j = 0; j < kRing; ++j) {
             const int kb = kb0 + j;
@@ -517,10 +566,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
               } else {
                 uint8_t* row = smem + stage * C::kStageBytes + C::kABytes + smem_row_off;
                 if (ring[j].valid) {
-                  dequant_row64<BITS>(ring[j].w, ring[j].s, ring[j].z, row, rx);
+                  float sv = ring[j].s, zv = ring[j].z;
+                  if (sz_blocks) {
+                    const int sub = ((kb << 6) >> p.group_shift) & 3;
+                    const uint32_t sw = (sub & 2) ? sz_cur.s4.y : sz_cur.s4.x;
+                    sv = __half2float(__ushort_as_half((unsigned short)((sub & 1) ? (sw >> 16) : (sw & 0xFFFFu))));
+                    zv = (float)((sz_cur.z4 >> (8 * sub)) & 0xFFu);
+                  }
+                  dequant_half32<BITS>(ring[j].w, sv, zv, row, rx, h);
                 } else {
 #pragma unroll
-                  for (int c = 0; c < 8; ++c) reinterpret_cast<uint4*>(row)[c] = make_uint4(0u, 0u, 0u, 0u);
+                  for (int c = 0; c < 4; ++c)
+                    *reinterpret_cast<uint4*>(row + (((4 * h + c) ^ rx) << 4)) = make_uint4(0u, 0u, 0u, 0u);
                 }
                 if (kb + kRing < num_kb) fetch(ring[j], n_blk, kb + kRing);
                 ptx::fence_proxy_async_smem();
@@ -530,6 +587,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
               }
             }
           }
+        }
+        if (warp < 2 + kEpiWarps && ok) {
+          ok = epilogue_tile(m_blk, n_blk, acc, acc_phase);
+          if (++acc == C::kAccSets) { acc = 0; acc_phase ^= 1u; }
         }
       }
     }
