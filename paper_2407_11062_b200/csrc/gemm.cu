@@ -78,11 +78,7 @@ struct Cfg {
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kThreads = (2 + (PACKED ? kDeqWarps : kEpiWarps)) * 32;
   static constexpr int kTmemCols = kAccSets * MT * BN;
-  // packed kernels: per stage, the packed codes of the B tile as TMA delivers them (2048 * bits bytes, at most 8 KB)
-  static constexpr int kRawBytes = PACKED ? 8192 : 0;
-  static constexpr int kRawOffset = kStages * kStageBytes;
-  static constexpr int kCtlOffset = kRawOffset + kStages * kRawBytes;
-  static constexpr int kSmemBytes = kCtlOffset + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 struct Control {
@@ -91,7 +87,6 @@ struct Control {
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
   uint64_t drain;
-  uint64_t raw_full[4];      // packed kernels: packed codes of a stage have landed
   uint32_t tmem_base;
   int abort;
 };
@@ -248,17 +243,12 @@ __global__ void __launch_bounds__(Cfg<BN, MT, PACKED>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const GemmParams p) {
   using C = Cfg<BN, MT, PACKED>;
-  // Packed codes reach shared memory by TMA (tmap_b then describes the packed matrix as bytes) unless a
-  // stage's codes of one row are not a multiple of 16 bytes (3-bit codes of a K-major tile: 24 bytes).
-  constexpr bool kRawTma = PACKED && !(BITS == 3 && !B_MN);
-  constexpr int kRawRowBytes = B_MN ? BN * BITS / 8 : BK * BITS / 8;     // bytes per row of the raw tile
-  constexpr int kRawTileBytes = 2048 * BITS;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_addr(smem_raw);
   const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;                                  // 1024-byte aligned stages
   const uint32_t smem_base = raw_addr + pad;
-  Control* ctl = reinterpret_cast<Control*>(smem + C::kCtlOffset);
+  Control* ctl = reinterpret_cast<Control*>(smem + C::kStages * C::kStageBytes);
   volatile int* abort_flag = &ctl->abort;
 
   const int warp = threadIdx.x >> 5;
@@ -278,11 +268,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[a]), 4);
     }
     ptx::mbar_init(ptx::smem_addr(&ctl->drain), 1);
-    for (int s = 0; s < C::kStages && s < 4; ++s) ptx::mbar_init(ptx::smem_addr(&ctl->raw_full[s]), 1);
     ctl->abort = 0;
     ptx::fence_mbar_init();
     ptx::tma_prefetch_desc(&tmap_a);
-    if (!PACKED || kRawTma) ptx::tma_prefetch_desc(&tmap_b);
+    if (!PACKED) ptx::tma_prefetch_desc(&tmap_b);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_base), C::kTmemCols);
@@ -407,13 +396,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             } else {
               ptx::tma_load_2d(b_dst, &tmap_b, kb * BK, n_blk * BN, full);
             }
-          } else if (kRawTma) {
-            // byte coordinates in the packed matrix: K-major tile = rows n, 64 codes of K block kb;
-            // MN-major tile = rows kb*64.., the BN codes of column block n_blk
-            const uint32_t raw_bar = ptx::smem_addr(&ctl->raw_full[stage]);
-            ptx::mbar_expect_tx(raw_bar, kRawTileBytes);
-            if (B_MN) ptx::tma_load_2d(smem_base + C::kRawOffset + stage * C::kRawBytes, &tmap_b, n_blk * kRawRowBytes, kb * BK, raw_bar);
-            else      ptx::tma_load_2d(smem_base + C::kRawOffset + stage * C::kRawBytes, &tmap_b, kb * kRawRowBytes, n_blk * BN, raw_bar);
           }
           ++issued;
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
@@ -423,16 +405,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         // Drain: every copy this thread started must land before the CTA exits.
         const long first = issued > C::kStages ? issued - C::kStages : 0;
         for (long i = first; i < issued; ++i) {
+          const uint32_t bar = ptx::smem_addr(&ctl->full[i % C::kStages]);
           const uint32_t par = (uint32_t)((i / C::kStages) & 1);
-          const uint32_t bars[2] = {ptx::smem_addr(&ctl->full[i % C::kStages]),
-                                    ptx::smem_addr(&ctl->raw_full[(i % C::kStages) & 3])};
-          for (int b = 0; b < (kRawTma ? 2 : 1); ++b) {
-            const uint64_t t0 = ptx::globaltimer_ns();
-            while (!ptx::mbar_try_wait(bars[b], par)) {
-              if (ptx::globaltimer_ns() - t0 > kDrainLimitNs) {
-                atomicExch(&g_device_status[1], (int)WAIT_TEARDOWN);
-                break;
-              }
+          const uint64_t t0 = ptx::globaltimer_ns();
+          while (!ptx::mbar_try_wait(bar, par)) {
+            if (ptx::globaltimer_ns() - t0 > kDrainLimitNs) {
+              atomicExch(&g_device_status[1], (int)WAIT_TEARDOWN);
+              break;
             }
           }
         }
@@ -513,8 +492,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       const int box = (t >> 4) & 3;                               // MN-major: 64-column box 0..3
       const int smem_row_off = B_MN ? (box * (BK * 128) + kr * 128) : n_row * 128;
       const int rx = B_MN ? (kr & 7) : (n_row & 7);
-      // this thread's 32 codes inside the TMA-delivered tile of packed bytes
-      const int raw_off = (B_MN ? kr * kRawRowBytes + box * (8 * BITS) : n_row * kRawRowBytes) + h * (4 * BITS);
       struct Unit {
         uint32_t w[BITS];
         float s, z;
@@ -546,7 +523,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         const int unit = B_MN ? n_blk * (BN / 64) + box : kb;
         u.valid = wrow < p.out_features && unit < chunks_in;
         if (u.valid) {
-          if (!kRawTma) load_codes32<BITS>(p.Wq + (size_t)wrow * pitch + (size_t)(2 * unit + h) * (4 * BITS), u.w);
+          load_codes32<BITS>(p.Wq + (size_t)wrow * pitch + (size_t)(2 * unit + h) * (4 * BITS), u.w);
           if (!sz_blocks) {
             const size_t gi = (size_t)wrow * groups_per_row + ((unit << 6) >> p.group_shift);
             u.s = __half2float(__ushort_as_half(__ldg(p.s16 + gi)));
@@ -584,27 +561,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           for (int j = 0; j < kRing; ++j) {
             const int kb = kb0 + j;
             if (ok && kb < num_kb) {
-              // With TMA-delivered codes the stage's codes landing implies the stage was free.
-              const bool ready = kRawTma
-                  ? wait_bounded(ptx::smem_addr(&ctl->raw_full[stage]), phase, abort_flag, WAIT_DEQ_OPERAND_EMPTY)
-                  : wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_DEQ_OPERAND_EMPTY);
-              if (!ready) {
+              if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_DEQ_OPERAND_EMPTY)) {
                 ok = false;
               } else {
                 uint8_t* row = smem + stage * C::kStageBytes + C::kABytes + smem_row_off;
-                if (kRawTma) {
-                  const uint32_t* rp = reinterpret_cast<const uint32_t*>(smem + C::kRawOffset + stage * C::kRawBytes + raw_off);
-                  if constexpr (BITS == 2) {
-                    const uint2 t2 = *reinterpret_cast<const uint2*>(rp);
-                    ring[j].w[0] = t2.x; ring[j].w[1] = t2.y;
-                  } else if constexpr (BITS == 4) {
-                    const uint4 t4 = *reinterpret_cast<const uint4*>(rp);
-                    ring[j].w[0] = t4.x; ring[j].w[1] = t4.y; ring[j].w[2] = t4.z; ring[j].w[3] = t4.w;
-                  } else {
-#pragma unroll
-                    for (int i = 0; i < BITS; ++i) ring[j].w[i] = rp[i];
-                  }
-                }
                 if (ring[j].valid) {
                   float sv = ring[j].s, zv = ring[j].z;
                   if (sz_blocks) {
@@ -672,20 +632,6 @@ bool make_tmap(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer
   const cuuint32_t estr[2] = {1, 1};
   return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// Packed codes as a byte matrix [rows, pitch]; box = box_bytes x box_rows, no swizzle.
-bool make_tmap_bytes(CUtensorMap* tm, const void* base, uint64_t pitch, uint64_t rows, uint32_t box_bytes,
-                     uint32_t box_rows) {
-  EncodeFn enc = encode_fn();
-  if (enc == nullptr) return false;
-  const cuuint64_t dims[2] = {pitch, rows};
-  const cuuint64_t strides[1] = {pitch};
-  const cuuint32_t box[2] = {box_bytes, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -783,36 +729,29 @@ int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X,
 
 int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
                       const uint8_t* z8, eqat_bf16* Y, cudaStream_t st) {
-  CUtensorMap ta, tb;
+  CUtensorMap ta;
   if (!make_tmap(&ta, X, d.in_features, d.tokens, 2 * BM)) return EQAT_ERR_CUDA;
-  // packed codes as bytes: one box = the 64 codes of a K block for 256 weight rows (3-bit rows of 24 bytes
-  // cannot be a TMA box; that kernel loads its codes itself and never touches this map)
-  const uint64_t pitch = (uint64_t)d.in_features * d.bits / 8;
-  if (!make_tmap_bytes(&tb, Wq, pitch, d.out_features, d.bits == 3 ? 48 : BK * d.bits / 8, 256)) return EQAT_ERR_CUDA;
   GemmParams p = base_params((int)d.tokens, d.out_features, d.in_features);
   p.D = Y;
   set_weight(p, d, Wq, s16, z8);
   switch (d.bits) {
-    case 2: return launch<256, 2, false, false, true, EPI_STORE, 2>(ta, tb, p, st);
-    case 3: return launch<256, 2, false, false, true, EPI_STORE, 3>(ta, tb, p, st);
-    default: return launch<256, 2, false, false, true, EPI_STORE, 4>(ta, tb, p, st);
+    case 2: return launch<256, 2, false, false, true, EPI_STORE, 2>(ta, ta, p, st);
+    case 3: return launch<256, 2, false, false, true, EPI_STORE, 3>(ta, ta, p, st);
+    default: return launch<256, 2, false, false, true, EPI_STORE, 4>(ta, ta, p, st);
   }
 }
 
 int launch_packed_dx(const eqat_desc& d, const eqat_bf16* dY, const uint8_t* Wq, const eqat_fp16* s16,
                      const uint8_t* z8, eqat_bf16* dX, cudaStream_t st) {
-  CUtensorMap ta, tb;
+  CUtensorMap ta;
   if (!make_tmap(&ta, dY, d.out_features, d.tokens, 2 * BM)) return EQAT_ERR_CUDA;
-  // packed codes as bytes: one box = 64 weight rows (a K block) x the 256 codes of a column block
-  const uint64_t pitch = (uint64_t)d.in_features * d.bits / 8;
-  if (!make_tmap_bytes(&tb, Wq, pitch, d.out_features, 256 * d.bits / 8, BK)) return EQAT_ERR_CUDA;
   GemmParams p = base_params((int)d.tokens, d.in_features, d.out_features);
   p.D = dX;
   set_weight(p, d, Wq, s16, z8);
   switch (d.bits) {
-    case 2: return launch<256, 2, false, true, true, EPI_STORE, 2>(ta, tb, p, st);
-    case 3: return launch<256, 2, false, true, true, EPI_STORE, 3>(ta, tb, p, st);
-    default: return launch<256, 2, false, true, true, EPI_STORE, 4>(ta, tb, p, st);
+    case 2: return launch<256, 2, false, true, true, EPI_STORE, 2>(ta, ta, p, st);
+    case 3: return launch<256, 2, false, true, true, EPI_STORE, 3>(ta, ta, p, st);
+    default: return launch<256, 2, false, true, true, EPI_STORE, 4>(ta, ta, p, st);
   }
 }
 
