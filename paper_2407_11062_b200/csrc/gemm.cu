@@ -492,11 +492,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       const int box = (t >> 4) & 3;                               // MN-major: 64-column box 0..3
       const int smem_row_off = B_MN ? (box * (BK * 128) + kr * 128) : n_row * 128;
       const int rx = B_MN ? (kr & 7) : (n_row & 7);
-      struct Unit {
-        uint32_t w[BITS];
-        float s, z;
-        bool valid;
-      };
       // Step sizes and zero points.  With a K-major B operand a thread stays on one
       // weight row for a whole tile and walks its groups in order, so it reads
       // them four groups at a time (one 8-byte and one 4-byte load per four
@@ -510,42 +505,65 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       };
       SzBlock sz_cur = {make_uint2(0u, 0u), 0u}, sz_nxt = {make_uint2(0u, 0u), 0u};
       int sz_blk = -1;
-      auto fetch_sz = [&](SzBlock& b, int n_blk, int blk) {
-        const int wrow = n_blk * BN + n_row;
-        if (wrow < p.out_features && blk * 4 < groups_per_row) {
-          const size_t gi = (size_t)wrow * groups_per_row + (size_t)blk * 4;
-          b.s4 = __ldg(reinterpret_cast<const uint2*>(p.s16 + gi));
-          b.z4 = __ldg(reinterpret_cast<const uint32_t*>(p.z8 + gi));
-        }
-      };
-      auto fetch = [&](Unit& u, int n_blk, int kb) {
-        const int wrow = B_MN ? kb * BK + kr : n_blk * BN + n_row;
-        const int unit = B_MN ? n_blk * (BN / 64) + box : kb;
-        u.valid = wrow < p.out_features && unit < chunks_in;
-        if (u.valid) {
-          load_codes32<BITS>(p.Wq + (size_t)wrow * pitch + (size_t)(2 * unit + h) * (4 * BITS), u.w);
-          if (!sz_blocks) {
-            const size_t gi = (size_t)wrow * groups_per_row + ((unit << 6) >> p.group_shift);
-            u.s = __half2float(__ushort_as_half(__ldg(p.s16 + gi)));
-            u.z = (float)__ldg(p.z8 + gi);
-          }
-        }
-      };
-      // Register ring of units: the loads for K block kb + kRing are issued as soon
-      // as block kb has been expanded, so they have kRing - 1 whole stages to land.
+      // Register ring: the loads for K block kb + kRing are issued as soon as block
+      // kb has been expanded, so they have kRing - 1 whole stages to land.  All
+      // addresses advance by a constant per K block, and whether the thread's unit
+      // lies inside the weight is a per-tile fact (out_features % 64 == 0).
       constexpr int kRing = 4;
-      Unit ring[kRing];
+      uint32_t ring_w[kRing][BITS];
+      float ring_s[kRing], ring_z[kRing];
+      const size_t code_step = B_MN ? (size_t)BK * pitch : (size_t)(8 * BITS);      // bytes per K block
+      const size_t sz_step = B_MN ? (size_t)BK * groups_per_row : 0;                // groups per K block (MN-major)
       int acc = 0;
       uint32_t acc_phase = 0;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
         tile_coords(tile, num_m, num_n, m_blk, n_blk);
+        const int wrow0 = B_MN ? kr : n_blk * BN + n_row;                           // weight row at K block 0
+        const int unit0 = B_MN ? n_blk * (BN / 64) + box : 0;                       // 64-code unit at K block 0
+        const bool valid = B_MN ? (unit0 < chunks_in) : (wrow0 < p.out_features);
+        const uint8_t* code_ptr = p.Wq + (valid ? (size_t)wrow0 * pitch + (size_t)(2 * unit0 + h) * (4 * BITS) : 0);
+        const size_t g0 = valid ? (size_t)wrow0 * groups_per_row + (B_MN ? ((unit0 << 6) >> p.group_shift) : 0) : 0;
+        const eqat_fp16* s_ptr = p.s16 + g0;
+        const uint8_t* z_ptr = p.z8 + g0;
+        auto fetch = [&](int j) {
+          if (valid) {
+            load_codes32<BITS>(code_ptr, ring_w[j]);
+            code_ptr += code_step;
+            if (!sz_blocks) {
+              // K-major without block loads: the group advances every (group / 64) K blocks
+              ring_s[j] = __half2float(__ushort_as_half(__ldg(s_ptr)));
+              ring_z[j] = (float)__ldg(z_ptr);
+            }
+          }
+        };
+        auto fetch_sz = [&](SzBlock& b, int blk) {
+          if (valid && blk * 4 < groups_per_row) {
+            b.s4 = __ldg(reinterpret_cast<const uint2*>(s_ptr + blk * 4));
+            b.z4 = __ldg(reinterpret_cast<const uint32_t*>(z_ptr + blk * 4));
+          }
+        };
+        // s/z pointer advance for the scalar path: MN-major moves 64 rows per K block; K-major moves to the
+        // next group whenever the K block crosses a group boundary
+        auto advance_sz = [&](int kb_next) {
+          if (B_MN) {
+            s_ptr += sz_step;
+            z_ptr += sz_step;
+          } else if (!sz_blocks && ((kb_next << 6) & ((1 << p.group_shift) - 1)) == 0) {
+            ++s_ptr;
+            ++z_ptr;
+          }
+        };
 #pragma unroll
-        for (int j = 0; j < kRing; ++j)
-          if (j < num_kb) fetch(ring[j], n_blk, j);
+        for (int j = 0; j < kRing; ++j) {
+          if (j < num_kb) {
+            fetch(j);
+            if (!sz_blocks) advance_sz(j + 1);
+          }
+        }
         if (sz_blocks) {
-          fetch_sz(sz_cur, n_blk, 0);
-          fetch_sz(sz_nxt, n_blk, 1);
+          fetch_sz(sz_cur, 0);
+          fetch_sz(sz_nxt, 1);
           sz_blk = 0;
         }
         for (int kb0 = 0; kb0 < num_kb && ok; kb0 += kRing) {
@@ -554,7 +572,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             if (blk != sz_blk) {
               sz_cur = sz_nxt;
               sz_blk = blk;
-              fetch_sz(sz_nxt, n_blk, blk + 1);
+              fetch_sz(sz_nxt, blk + 1);
             }
           }
 #pragma unroll
@@ -565,21 +583,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 ok = false;
               } else {
                 uint8_t* row = smem + stage * C::kStageBytes + C::kABytes + smem_row_off;
-                if (ring[j].valid) {
-                  float sv = ring[j].s, zv = ring[j].z;
+                if (valid) {
+                  float sv = ring_s[j], zv = ring_z[j];
                   if (sz_blocks) {
                     const int sub = ((kb << 6) >> p.group_shift) & 3;
                     const uint32_t sw = (sub & 2) ? sz_cur.s4.y : sz_cur.s4.x;
                     sv = __half2float(__ushort_as_half((unsigned short)((sub & 1) ? (sw >> 16) : (sw & 0xFFFFu))));
                     zv = (float)((sz_cur.z4 >> (8 * sub)) & 0xFFu);
                   }
-                  dequant_half32<BITS>(ring[j].w, sv, zv, row, rx, h);
+                  dequant_half32<BITS>(ring_w[j], sv, zv, row, rx, h);
                 } else {
 #pragma unroll
                   for (int c = 0; c < 4; ++c)
                     *reinterpret_cast<uint4*>(row + (((4 * h + c) ^ rx) << 4)) = make_uint4(0u, 0u, 0u, 0u);
                 }
-                if (kb + kRing < num_kb) fetch(ring[j], n_blk, kb + kRing);
+                if (kb + kRing < num_kb) {
+                  fetch(j);
+                  if (!sz_blocks) advance_sz(kb + kRing + 1);
+                }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full[stage]));
