@@ -187,37 +187,79 @@ class BlockWorkload:
 
 
 class HostStaging:
-    """Pinned host copies of each shape's activations and gradient outputs for the end-to-end leg."""
+    """End-to-end leg: every step's X and dY come from pinned host memory and the weight-side
+    gradients (dW, ds, dz of Block-AP, ds of E2E-QP) go back to pinned host memory, all inside the
+    timed region.  Copies run on their own streams and are double-buffered per linear shape, so the
+    upload of the next linear and the download of the previous one overlap the kernels of the
+    current one (the step is then bound by whichever of PCIe and the GPU is slower)."""
+
+    OUT = ("dW", "ds", "dz", "ds2")
 
     def __init__(self, wl: BlockWorkload):
         self.wl = wl
-        self.host = {}
+        self.host, self.sets, self.uses = {}, {}, {}
         for name, S in wl.shapes.items():
             self.host[name] = dict(
                 X=S["X"].cpu().pin_memory(), dY=S["dY"].cpu().pin_memory(),
-                dW=torch.empty(S["dW"].shape, dtype=S["dW"].dtype).pin_memory(),
-                ds=torch.empty(S["ds"].shape).pin_memory(), dz=torch.empty(S["dz"].shape).pin_memory(),
-                ds2=torch.empty(S["ds2"].shape).pin_memory())
+                **{k: torch.empty(S[k].shape, dtype=S[k].dtype).pin_memory() for k in self.OUT})
+            second = {k: torch.empty_like(S[k]) for k in ("X", "dY") + self.OUT}
+            self.sets[name] = [{k: S[k] for k in ("X", "dY") + self.OUT}, second]
+            self.uses[name] = 0
         self.h2d = sum(self.host[L["shape"]]["X"].nbytes + self.host[L["shape"]]["dY"].nbytes for L in wl.layers)
-        self.d2h = sum(sum(self.host[L["shape"]][k].nbytes for k in ("dW", "ds", "dz", "ds2")) for L in wl.layers)
+        self.d2h = sum(sum(self.host[L["shape"]][k].nbytes for k in self.OUT) for L in wl.layers)
+        self.up, self.down = torch.cuda.Stream(), torch.cuda.Stream()
+        self.last_done = {}        # (shape, set) -> event: kernels that read/wrote this set have finished
+        self.last_down = {}        # (shape, set) -> event: its gradients have been downloaded
 
     def step(self):
         wl, e = self.wl, self.wl.eqat
-        for L in wl.layers:
-            S, H = wl.shapes[L["shape"]], self.host[L["shape"]]
-            S["X"].copy_(H["X"], non_blocking=True)
-            S["dY"].copy_(H["dY"], non_blocking=True)
-            Xa, dYa, Ya, dXa = S["X"][: wl.t_ap], S["dY"][: wl.t_ap], S["Y"][: wl.t_ap], S["dX"][: wl.t_ap]
+        main = torch.cuda.current_stream()
+        start = torch.cuda.Event(); start.record(main)
+        self.up.wait_event(start)                       # copies of this step start inside the timed region
+        def upload(L):
+            """Enqueue the upload of one linear's X and dY into the free buffer set of its shape."""
+            name = L["shape"]
+            k = self.uses[name] % 2
+            self.uses[name] += 1
+            D, H = self.sets[name][k], self.host[name]
+            if (name, k) in self.last_done:             # the kernels that last read this set must be done
+                self.up.wait_event(self.last_done[(name, k)])
+            with torch.cuda.stream(self.up):
+                D["X"].copy_(H["X"], non_blocking=True)
+                D["dY"].copy_(H["dY"], non_blocking=True)
+                ev = torch.cuda.Event(); ev.record(self.up)
+            return k, ev
+
+        nxt = upload(wl.layers[0])
+        for i, L in enumerate(wl.layers):
+            k, ev = nxt
+            if i + 1 < len(wl.layers):
+                nxt = upload(wl.layers[i + 1])          # one linear ahead: overlaps this linear's kernels
+            name = L["shape"]
+            S, D, H = wl.shapes[name], self.sets[name][k], self.host[name]
+            main.wait_event(ev)
+            if (name, k) in self.last_down:
+                main.wait_event(self.last_down[(name, k)])
+            X, dY = D["X"], D["dY"]
+            Xa, dYa, Ya, dXa = X[: wl.t_ap], dY[: wl.t_ap], S["Y"][: wl.t_ap], S["dX"][: wl.t_ap]
             e.eqat_minmax_init(S["d_ap"], L["W"], L["s"], L["z"])
             e.qlinear_fakequant_fwd(S["d_ap"], Xa, L["W"], L["s"], L["z"], Ya, S["What"])
-            e.qlinear_fakequant_bwd(S["d_ap"], Xa, dYa, L["W"], L["s"], L["z"], S["What"], dXa, S["dW"], S["ds"], S["dz"], S["ws"])
+            e.qlinear_fakequant_bwd(S["d_ap"], Xa, dYa, L["W"], L["s"], L["z"], S["What"], dXa, D["dW"], D["ds"], D["dz"], S["ws"])
             e.eqat_quantize_pack(S["d_ap"], L["W"], L["s"], L["z"], L["P"], L["z8"], L["s16"])
             e.eqat_unpack(S["d_ap"], L["P"], S["codes"])
-            e.qlinear_packed_fwd(S["d_e2e"], S["X"], L["P"], L["s16"], L["z8"], S["Y"])
-            e.qlinear_packed_bwd_dx(S["d_e2e"], S["dY"], L["P"], L["s16"], L["z8"], S["dX"])
-            e.qlinear_packed_bwd_ds(S["d_e2e"], S["X"], S["dY"], L["P"], L["z8"], L["s16"], S["ds2"])
-            for k in ("dW", "ds", "dz", "ds2"):
-                H[k].copy_(S[k], non_blocking=True)
+            e.qlinear_packed_fwd(S["d_e2e"], X, L["P"], L["s16"], L["z8"], S["Y"])
+            e.qlinear_packed_bwd_dx(S["d_e2e"], dY, L["P"], L["s16"], L["z8"], S["dX"])
+            e.qlinear_packed_bwd_ds(S["d_e2e"], X, dY, L["P"], L["z8"], L["s16"], D["ds2"])
+            done = torch.cuda.Event(); done.record(main)
+            self.last_done[(name, k)] = done
+            self.down.wait_event(done)
+            with torch.cuda.stream(self.down):
+                for o in self.OUT:
+                    H[o].copy_(D[o], non_blocking=True)
+                dn = torch.cuda.Event(); dn.record(self.down)
+            self.last_down[(name, k)] = dn
+        main.wait_stream(self.up)
+        main.wait_stream(self.down)                     # the step ends when its last gradient is on the host
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
