@@ -139,25 +139,7 @@ __device__ __forceinline__ void minmax_finish(float mx, float mn, float Q, float
   z[g] = zv;
 }
 
-template <int LPG>
-__global__ void __launch_bounds__(kThreads)
-minmax_kernel(const eqat_bf16* __restrict__ W, float* __restrict__ s, float* __restrict__ z, size_t n_vec, float Q) {
-  const size_t v = (size_t)blockIdx.x * kThreads + threadIdx.x;
-  const bool live = v < n_vec;
-  float mx = -INFINITY, mn = INFINITY;
-  if (live) {
-    const Vec8 w = load_bf16x8(W, v);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) { mx = fmaxf(mx, w.v[i]); mn = fminf(mn, w.v[i]); }
-  }
-#pragma unroll
-  for (int d = LPG / 2; d >= 1; d >>= 1) {
-    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
-    mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, d));
-  }
-  if (live && (v % LPG) == 0) minmax_finish(mx, mn, Q, s, z, v / LPG);
-}
-
+// (groups of at most 256 elements are handled by the staged kernel in stream.cu)
 __global__ void __launch_bounds__(kThreads)
 minmax_long_group_kernel(const eqat_bf16* __restrict__ W, float* __restrict__ s, float* __restrict__ z,
                          int vec_per_group, float Q) {
@@ -327,24 +309,16 @@ int launch_ste_bwd(const eqat_desc& d, const eqat_bf16* dWhat, const eqat_bf16* 
 }
 
 int launch_minmax(const eqat_desc& d, const eqat_bf16* W, float* s, float* z, cudaStream_t st) {
-  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
+  if (d.group <= 256) return launch_minmax_stream(d, W, s, z, st);
   const float Q = (float)((1 << d.bits) - 1);
-  const unsigned nb = blocks_for(n_vec, kThreads);
-  switch (d.group) {
-    case 32:  minmax_kernel<4><<<nb, kThreads, 0, st>>>(W, s, z, n_vec, Q); break;
-    case 64:  minmax_kernel<8><<<nb, kThreads, 0, st>>>(W, s, z, n_vec, Q); break;
-    case 128: minmax_kernel<16><<<nb, kThreads, 0, st>>>(W, s, z, n_vec, Q); break;
-    case 256: minmax_kernel<32><<<nb, kThreads, 0, st>>>(W, s, z, n_vec, Q); break;
-    default: {
-      const size_t n_groups = (size_t)d.out_features * d.in_features / d.group;
-      minmax_long_group_kernel<<<(unsigned)n_groups, kThreads, 0, st>>>(W, s, z, d.group / 8, Q);
-    }
-  }
+  const size_t n_groups = (size_t)d.out_features * d.in_features / d.group;
+  minmax_long_group_kernel<<<(unsigned)n_groups, kThreads, 0, st>>>(W, s, z, d.group / 8, Q);
   return launch_status();
 }
 
 int launch_quantize_pack(const eqat_desc& d, const eqat_bf16* W, const float* s, const float* z, uint8_t* packed,
                          uint8_t* z8, eqat_fp16* s16, cudaStream_t st) {
+  if (d.group <= 256) return launch_quantize_pack_stream(d, W, s, z, packed, z8, s16, st);
   const size_t n_chunk = (size_t)d.out_features * d.in_features / 32;
   const unsigned nb = blocks_for(n_chunk, kThreads);
   const uint32_t cpg = (uint32_t)d.group / 32;

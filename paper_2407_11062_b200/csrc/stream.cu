@@ -1,5 +1,6 @@
-// Streaming kernels with TMA-staged inputs: fake quantiser (Eq. 1 + Eq. 2) and
-// its straight-through backward (Eqs. 3-5) for groups of at most 256 elements.
+// Streaming kernels with TMA-staged inputs: fake quantiser (Eq. 1 + Eq. 2), its
+// straight-through backward (Eqs. 3-5), min/max initialisation and quantise +
+// pack, for groups of at most 256 elements.
 //
 // These kernels are bound by HBM bandwidth, and what decides how close they
 // get to it is the number of bytes in flight per SM.  A plain "load, compute,
@@ -227,7 +228,7 @@ __device__ __forceinline__ void quotient_round8(const float (&w)[8], float s, fl
   }
 }
 
-constexpr int kFakequantVpt = 4, kSteVpt = 2;
+constexpr int kFakequantVpt = 4, kSteVpt = 2, kMinmaxVpt = 4, kPackVpt = 4;
 
 // Step size and zero point of the groups of a thread's vectors.
 template <int VPT>
@@ -335,6 +336,124 @@ ste_bwd_stream_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __re
   });
 }
 
+// ------------------------------------------------------------------ min/max initialisation
+struct NoParams {};
+
+__device__ __forceinline__ uint32_t bf162_max(uint32_t a, uint32_t b) {
+  const __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+  return *reinterpret_cast<const uint32_t*>(&r);
+}
+__device__ __forceinline__ uint32_t bf162_min(uint32_t a, uint32_t b) {
+  const __nv_bfloat162 r = __hmin2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+  return *reinterpret_cast<const uint32_t*>(&r);
+}
+
+template <int LPG>
+__global__ void __launch_bounds__(kThreadsS)
+minmax_stream_kernel(const eqat_bf16* __restrict__ W, float* __restrict__ s, float* __restrict__ z, size_t n_vec,
+                     float Q) {
+  const uint8_t* const src[1] = {reinterpret_cast<const uint8_t*>(W)};
+  constexpr int VPT = kMinmaxVpt;
+  static_assert(kMinmaxVpt <= 4 && LPG >= 4, "one lane of a group finishes one of the thread's vectors");
+  stream_chunks<1, VPT, NoParams>(src, n_vec, [](size_t) { return NoParams{}; },
+      [&](size_t v0, const uint4 (&raw)[1][VPT], const NoParams&) {
+    // Reduce each of the thread's VPT vectors over the lanes of its group (every lane ends up with the
+    // group's extrema), then let lane u of the group finish vector u: one pass of the division code for
+    // all VPT groups instead of VPT passes with one active lane per group.
+    float mx_sel = 0.0f, mn_sel = 0.0f;
+    const int sub = threadIdx.x % LPG;
+#pragma unroll
+    for (int u = 0; u < VPT; ++u) {
+      const size_t v = v0 + (size_t)u * kConsumers;
+      // extrema on packed bf16 pairs (exact: comparisons only), widened to fp32 at the end
+      uint32_t mx2 = 0xFF80FF80u, mn2 = 0x7F807F80u;    // (-inf, -inf) and (+inf, +inf) as bf16 pairs
+      if (v < n_vec) {                                  // uniform over the lanes of a group
+        const uint4 r4 = raw[0][u];
+        mx2 = bf162_max(bf162_max(r4.x, r4.y), bf162_max(r4.z, r4.w));
+        mn2 = bf162_min(bf162_min(r4.x, r4.y), bf162_min(r4.z, r4.w));
+      }
+#pragma unroll
+      for (int d = LPG / 2; d >= 1; d >>= 1) {
+        mx2 = bf162_max(mx2, __shfl_xor_sync(0xFFFFFFFFu, mx2, d));
+        mn2 = bf162_min(mn2, __shfl_xor_sync(0xFFFFFFFFu, mn2, d));
+      }
+      if (sub == u) {
+        mx_sel = fmaxf(__uint_as_float(mx2 << 16), __uint_as_float(mx2 & 0xFFFF0000u));
+        mn_sel = fminf(__uint_as_float(mn2 << 16), __uint_as_float(mn2 & 0xFFFF0000u));
+      }
+    }
+    const size_t v = v0 - sub + (size_t)sub * kConsumers;          // first vector of the group this lane finishes
+    if (sub < VPT && v < n_vec) {
+      // s = max((max - min) / Q, 2^-14), z = clamp(-round(min / s), 0, Q), all in binary32
+      float sv = __fdiv_rn(mx_sel - mn_sel, Q);
+      sv = fmaxf(sv, 6.103515625e-05f);
+      float zv = -rintf(__fdiv_rn(mn_sel, sv));
+      zv = fminf(fmaxf(zv, 0.0f), Q) + 0.0f;
+      s[v / LPG] = sv;
+      z[v / LPG] = zv;
+    }
+  });
+}
+
+// ------------------------------------------------------------------ quantise + pack (hand-off)
+// A thread turns one vector (8 weights) into 8*BITS bits; four adjacent lanes
+// hold 32 consecutive codes, which lane 0 of the four assembles into BITS
+// 32-bit words of the little-endian stream and stores.
+template <int BITS>
+__global__ void __launch_bounds__(kThreadsS)
+quantize_pack_stream_kernel(const eqat_bf16* __restrict__ W, const float* __restrict__ s, const float* __restrict__ z,
+                            uint8_t* __restrict__ packed, uint8_t* __restrict__ z8, eqat_fp16* __restrict__ s16,
+                            size_t n_vec, int vec_shift) {
+  const uint8_t* const src[1] = {reinterpret_cast<const uint8_t*>(W)};
+  constexpr int VPT = kPackVpt;
+  constexpr float Q = (float)((1 << BITS) - 1);
+  stream_chunks<1, VPT, GroupParams<VPT>>(src, n_vec,
+      [&](size_t v0) { return fetch_groups<VPT>(s, z, v0, n_vec, vec_shift); },
+      [&](size_t v0, const uint4 (&raw)[1][VPT], const GroupParams<VPT>& gp) {
+#pragma unroll
+    for (int u = 0; u < VPT; ++u) {
+      const size_t v = v0 + (size_t)u * kConsumers;
+      const bool live = v < n_vec;                      // uniform over each 4 adjacent lanes (n_vec % 4 == 0)
+      uint32_t piece = 0u;                              // this vector's 8 codes, code i at bits [BITS*i, BITS*i+BITS)
+      if (live) {
+        const float sv = gp.s[u];
+        const float zr = rintf(gp.z[u]);
+        const float rs = group_rcp(sv);
+        float w[8], r[8], rt[8];
+        unpack8(raw[0][u], w);
+        quotient_round8(w, sv, rs, r, rt);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float q = fminf(fmaxf(r[i] + zr, 0.0f), Q);
+          piece |= (__float_as_uint(q + 8388608.0f) & 0xFFu) << (BITS * i);     // integer-valued float -> integer
+        }
+        if ((v & (((size_t)1 << vec_shift) - 1)) == 0) {
+          const size_t g = v >> vec_shift;
+          z8[g] = (uint8_t)(__float_as_uint(fminf(fmaxf(zr, 0.0f), Q) + 8388608.0f) & 0xFFu);
+          s16[g] = __half_as_ushort(__float2half_rn(sv));
+        }
+      }
+      if constexpr (BITS == 4) {
+        if (live) reinterpret_cast<uint32_t*>(packed)[v] = piece;                // 32 bits per vector: store directly
+      } else {
+        const uint32_t p1 = __shfl_down_sync(0xFFFFFFFFu, piece, 1);
+        const uint32_t p2 = __shfl_down_sync(0xFFFFFFFFu, piece, 2);
+        const uint32_t p3 = __shfl_down_sync(0xFFFFFFFFu, piece, 3);
+        if (live && (threadIdx.x & 3) == 0) {
+          if constexpr (BITS == 2) {
+            reinterpret_cast<uint2*>(packed)[v >> 2] = make_uint2(piece | (p1 << 16), p2 | (p3 << 16));
+          } else {
+            uint32_t* dst = reinterpret_cast<uint32_t*>(packed) + (v >> 2) * 3;
+            dst[0] = piece | (p1 << 24);
+            dst[1] = (p1 >> 8) | (p2 << 16);
+            dst[2] = (p2 >> 16) | (p3 << 8);
+          }
+        }
+      }
+    }
+  });
+}
+
 // Persistent grid: every CTA resident at once, never more CTAs than chunks.
 template <typename K>
 unsigned stream_grid(K kernel, int smem_bytes, size_t n_vec, int chunk_vec) {
@@ -385,6 +504,33 @@ int launch_ste_bwd_stream(const eqat_desc& d, const eqat_bf16* dWhat, const eqat
     case 64:  return launch_stream(ste_bwd_stream_kernel<8>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
     case 128: return launch_stream(ste_bwd_stream_kernel<16>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
     default:  return launch_stream(ste_bwd_stream_kernel<32>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+  }
+}
+
+int launch_minmax_stream(const eqat_desc& d, const eqat_bf16* W, float* s, float* z, cudaStream_t st) {
+  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
+  const float Q = (float)((1 << d.bits) - 1);
+  using R = Ring<1, kMinmaxVpt>;
+  constexpr int smem = R::kSmemBytes, cv = R::kChunkVec;
+  switch (d.group) {
+    case 32:  return launch_stream(minmax_stream_kernel<4>, smem, cv, n_vec, st, W, s, z, n_vec, Q);
+    case 64:  return launch_stream(minmax_stream_kernel<8>, smem, cv, n_vec, st, W, s, z, n_vec, Q);
+    case 128: return launch_stream(minmax_stream_kernel<16>, smem, cv, n_vec, st, W, s, z, n_vec, Q);
+    default:  return launch_stream(minmax_stream_kernel<32>, smem, cv, n_vec, st, W, s, z, n_vec, Q);
+  }
+}
+
+int launch_quantize_pack_stream(const eqat_desc& d, const eqat_bf16* W, const float* s, const float* z,
+                                uint8_t* packed, uint8_t* z8, eqat_fp16* s16, cudaStream_t st) {
+  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
+  int vec_shift = 0;
+  while ((8 << vec_shift) < d.group) ++vec_shift;
+  using R = Ring<1, kPackVpt>;
+  constexpr int smem = R::kSmemBytes, cv = R::kChunkVec;
+  switch (d.bits) {
+    case 2:  return launch_stream(quantize_pack_stream_kernel<2>, smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
+    case 3:  return launch_stream(quantize_pack_stream_kernel<3>, smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
+    default: return launch_stream(quantize_pack_stream_kernel<4>, smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
   }
 }
 
