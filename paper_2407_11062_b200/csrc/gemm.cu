@@ -19,11 +19,12 @@
 //               quadrant each); with MT = 1 the next tile is already being
 //               multiplied meanwhile
 //   warps 2-17  (packed-weight kernels only) expand N-bit codes into the bf16 B
-//               operand stage, (q - z) * s exactly, rounded once to bf16; sixteen
-//               warps because the expansion is latency-bound per warp.  Warps
-//               2-5 then run the epilogue of the tile (MT = 2: nothing overlaps it
-//               anyway, and the other twelve warps meanwhile pre-expand the next
-//               tile's first stages up to the point where they need these four)
+//               operand stage, (q - z) * s exactly, rounded once to bf16: two
+//               groups of eight warps take alternate K blocks, one 64-code row per
+//               thread, so two stages are being expanded at any time.  Warps 2-5
+//               then run the epilogue of the tile (MT = 2: nothing overlaps it
+//               anyway, and the other warps meanwhile pre-expand the next tile's
+//               first stages up to the point where they need these four)
 // The epilogue either stores the tile as bf16 or, for the E2E-QP step-size
 // gradient, multiplies each accumulator row by (q - z) of the matching packed
 // codes and reduces runs of `group` columns, so the [out,in] weight gradient
@@ -221,18 +222,24 @@ __device__ __forceinline__ void dequant_half32(const uint32_t (&w)[BITS], float 
   }
 }
 
-// 32 codes = BITS consecutive 32-bit words, at a multiple of 4*BITS bytes.
+// 64 codes = 2*BITS consecutive 32-bit words, at a multiple of 8*BITS bytes.
 template <int BITS>
-__device__ __forceinline__ void load_codes32(const uint8_t* p, uint32_t (&w)[BITS]) {
+__device__ __forceinline__ void load_codes64(const uint8_t* p, uint32_t (&w)[2 * BITS]) {
   if constexpr (BITS == 2) {
-    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
-    w[0] = t.x; w[1] = t.y;
-  } else if constexpr (BITS == 3) {
-#pragma unroll
-    for (int i = 0; i < 3; ++i) w[i] = __ldg(reinterpret_cast<const uint32_t*>(p) + i);
-  } else {
     const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
     w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+  } else if constexpr (BITS == 3) {
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+      const uint2 t = __ldg(reinterpret_cast<const uint2*>(p) + i);
+      w[2 * i] = t.x; w[2 * i + 1] = t.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const uint4 t = __ldg(reinterpret_cast<const uint4*>(p) + i);
+      w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
+    }
   }
 }
 
@@ -260,7 +267,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
-      ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), PACKED ? 1 + kDeqWarps : 1);
+      ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), PACKED ? 1 + kDeqWarps / 2 : 1);
       ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), 1);
     }
     for (int a = 0; a < C::kAccSets; ++a) {
@@ -474,24 +481,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   } else {
     // ------------------------------------------------------------ dequantisers (+ epilogue on warps 2-5)
     if constexpr (PACKED) {
-      const int t = threadIdx.x - 64;                             // 0..511, one 32-code half unit per stage
+      // Sixteen warps in two groups of eight: group 0 expands the even K blocks (counted over all tiles of
+      // this CTA), group 1 the odd ones, each thread one whole 64-code unit (one 128-byte operand row) of
+      // its K blocks.  Two stages are thus being expanded at any time, and the per-K-block bookkeeping
+      // (wait, fence, arrive, addresses, step size) is paid once per 64 codes.
+      const int t = (threadIdx.x - 64) & 255;                     // unit within the stage
+      const int grp = (threadIdx.x - 64) >> 8;                    // 0 or 1
       const size_t pitch = (size_t)p.in_features * BITS / 8;      // bytes per packed row
       const int groups_per_row = p.in_features >> p.group_shift;
       const int chunks_in = p.in_features >> 6;                   // 64-code units per row
-      int stage = 0;
-      uint32_t phase = 0;
       bool ok = true;
-      // A 64-code unit is one 128-byte shared-memory row; a thread expands half h of it.
-      //   B K-major  (Y):  tile row n is weight row n0 + n, unit = kb
+      //   B K-major  (Y):  tile row t is weight row n0 + t, unit = kb
       //   B MN-major (dX): k-row kr is weight row kb*64 + kr, unit = n0/64 + box (64-column box)
-      // The 8 lanes of a quarter-warp (one 16-byte store wavefront) own the same
-      // half of 8 consecutive rows, whose swizzled chunks fall in 8 different bank groups.
-      const int h = (t >> 3) & 1;
-      const int n_row = (t & 7) | ((t >> 4) << 3);                // K-major: tile row 0..255
-      const int kr = (t & 7) | ((t >> 6) << 3);                   // MN-major: k-row 0..63
-      const int box = (t >> 4) & 3;                               // MN-major: 64-column box 0..3
-      const int smem_row_off = B_MN ? (box * (BK * 128) + kr * 128) : n_row * 128;
-      const int rx = B_MN ? (kr & 7) : (n_row & 7);
+      // The 8 lanes of a quarter-warp (one 16-byte store wavefront) own 8 consecutive
+      // rows, whose swizzled chunks fall in 8 different bank groups.
+      const int kr = (t & 7) | ((t >> 5) << 3);                   // MN-major: k-row 0..63
+      const int box = (t >> 3) & 3;                               // MN-major: 64-column box 0..3
+      const int smem_row_off = B_MN ? (box * (BK * 128) + kr * 128) : t * 128;
+      const int rx = B_MN ? (kr & 7) : (t & 7);
       // Step sizes and zero points.  With a K-major B operand a thread stays on one
       // weight row for a whole tile and walks its groups in order, so it reads
       // them four groups at a time (one 8-byte and one 4-byte load per four
@@ -505,35 +512,35 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       };
       SzBlock sz_cur = {make_uint2(0u, 0u), 0u}, sz_nxt = {make_uint2(0u, 0u), 0u};
       int sz_blk = -1;
-      // Register ring: the loads for K block kb + kRing are issued as soon as block
-      // kb has been expanded, so they have kRing - 1 whole stages to land.  All
-      // addresses advance by a constant per K block, and whether the thread's unit
-      // lies inside the weight is a per-tile fact (out_features % 64 == 0).
-      constexpr int kRing = 4;
-      uint32_t ring_w[kRing][BITS];
-      float ring_s[kRing], ring_z[kRing];
-      const size_t code_step = B_MN ? (size_t)BK * pitch : (size_t)(8 * BITS);      // bytes per K block
-      const size_t sz_step = B_MN ? (size_t)BK * groups_per_row : 0;                // groups per K block (MN-major)
+      // Register ring of two units: the loads for the thread's next-but-one K block
+      // (four K blocks ahead) are issued as soon as the current one has been expanded.
+      uint32_t ring_w[2][2 * BITS];
+      float ring_s[2], ring_z[2];
+      const size_t code_step = 2 * (B_MN ? (size_t)BK * pitch : (size_t)(8 * BITS));   // bytes per two K blocks
+      const size_t sz_step = B_MN ? (size_t)2 * BK * groups_per_row : 0;               // groups per two K blocks
+      long gk = 0;                                                // global index of the tile's K block 0
       int acc = 0;
       uint32_t acc_phase = 0;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
         tile_coords(tile, num_m, num_n, m_blk, n_blk);
-        const int wrow0 = B_MN ? kr : n_blk * BN + n_row;                           // weight row at K block 0
-        const int unit0 = B_MN ? n_blk * (BN / 64) + box : 0;                       // 64-code unit at K block 0
+        const int kb_first = (int)((grp - gk) & 1);               // this group's first K block of the tile
+        const int wrow0 = B_MN ? kb_first * BK + kr : n_blk * BN + t;
+        const int unit0 = B_MN ? n_blk * (BN / 64) + box : kb_first;
         const bool valid = B_MN ? (unit0 < chunks_in) : (wrow0 < p.out_features);
-        const uint8_t* code_ptr = p.Wq + (valid ? (size_t)wrow0 * pitch + (size_t)(2 * unit0 + h) * (4 * BITS) : 0);
+        const uint8_t* code_ptr = p.Wq + (valid ? (size_t)wrow0 * pitch + (size_t)unit0 * (8 * BITS) : 0);
         const size_t g0 = valid ? (size_t)wrow0 * groups_per_row + (B_MN ? ((unit0 << 6) >> p.group_shift) : 0) : 0;
-        const eqat_fp16* s_ptr = p.s16 + g0;
+        const eqat_fp16* s_ptr = p.s16 + g0;                      // K-major: group 0 of the row
         const uint8_t* z_ptr = p.z8 + g0;
-        auto fetch = [&](int j) {
+        auto fetch = [&](int j, int kb) {                         // kb: the K block being fetched
           if (valid) {
-            load_codes32<BITS>(code_ptr, ring_w[j]);
+            load_codes64<BITS>(code_ptr, ring_w[j]);
             code_ptr += code_step;
             if (!sz_blocks) {
-              // K-major without block loads: the group advances every (group / 64) K blocks
-              ring_s[j] = __half2float(__ushort_as_half(__ldg(s_ptr)));
-              ring_z[j] = (float)__ldg(z_ptr);
+              const size_t gi = B_MN ? 0 : (size_t)((kb << 6) >> p.group_shift);
+              ring_s[j] = __half2float(__ushort_as_half(__ldg(s_ptr + gi)));
+              ring_z[j] = (float)__ldg(z_ptr + gi);
+              if (B_MN) { s_ptr += sz_step; z_ptr += sz_step; }
             }
           }
         };
@@ -543,42 +550,29 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             b.z4 = __ldg(reinterpret_cast<const uint32_t*>(z_ptr + blk * 4));
           }
         };
-        // s/z pointer advance for the scalar path: MN-major moves 64 rows per K block; K-major moves to the
-        // next group whenever the K block crosses a group boundary
-        auto advance_sz = [&](int kb_next) {
-          if (B_MN) {
-            s_ptr += sz_step;
-            z_ptr += sz_step;
-          } else if (!sz_blocks && ((kb_next << 6) & ((1 << p.group_shift) - 1)) == 0) {
-            ++s_ptr;
-            ++z_ptr;
-          }
-        };
 #pragma unroll
-        for (int j = 0; j < kRing; ++j) {
-          if (j < num_kb) {
-            fetch(j);
-            if (!sz_blocks) advance_sz(j + 1);
-          }
-        }
+        for (int j = 0; j < 2; ++j)
+          if (kb_first + 2 * j < num_kb) fetch(j, kb_first + 2 * j);
         if (sz_blocks) {
           fetch_sz(sz_cur, 0);
           fetch_sz(sz_nxt, 1);
           sz_blk = 0;
         }
-        for (int kb0 = 0; kb0 < num_kb && ok; kb0 += kRing) {
-          if (sz_blocks) {
-            const int blk = ((kb0 << 6) >> p.group_shift) >> 2;      // constant over the kRing blocks below
-            if (blk != sz_blk) {
-              sz_cur = sz_nxt;
-              sz_blk = blk;
-              fetch_sz(sz_nxt, blk + 1);
-            }
-          }
+        int stage = (int)((gk + kb_first) % C::kStages);
+        uint32_t phase = (uint32_t)(((gk + kb_first) / C::kStages) & 1);
+        for (int kb0 = kb_first; kb0 < num_kb && ok; kb0 += 4) {
 #pragma unroll
-          for (int j = 0; j < kRing; ++j) {
-            const int kb = kb0 + j;
+          for (int j = 0; j < 2; ++j) {
+            const int kb = kb0 + 2 * j;
             if (ok && kb < num_kb) {
+              if (sz_blocks) {
+                const int blk = ((kb << 6) >> p.group_shift) >> 2;
+                if (blk != sz_blk) {
+                  sz_cur = sz_nxt;
+                  sz_blk = blk;
+                  fetch_sz(sz_nxt, blk + 1);
+                }
+              }
               if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_DEQ_OPERAND_EMPTY)) {
                 ok = false;
               } else {
@@ -591,24 +585,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     sv = __half2float(__ushort_as_half((unsigned short)((sub & 1) ? (sw >> 16) : (sw & 0xFFFFu))));
                     zv = (float)((sz_cur.z4 >> (8 * sub)) & 0xFFu);
                   }
-                  dequant_half32<BITS>(ring_w[j], sv, zv, row, rx, h);
+                  dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][0]), sv, zv, row, rx, 0);
+                  dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][BITS]), sv, zv, row, rx, 1);
                 } else {
 #pragma unroll
-                  for (int c = 0; c < 4; ++c)
-                    *reinterpret_cast<uint4*>(row + (((4 * h + c) ^ rx) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                  for (int c = 0; c < 8; ++c) reinterpret_cast<uint4*>(row)[c] = make_uint4(0u, 0u, 0u, 0u);
                 }
-                if (kb + kRing < num_kb) {
-                  fetch(j);
-                  if (!sz_blocks) advance_sz(kb + kRing + 1);
-                }
+                if (kb + 4 < num_kb) fetch(j, kb + 4);
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full[stage]));
-                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                stage += 2;                                       // this group's next K block is two further
+                if (stage >= C::kStages) { stage -= C::kStages; phase ^= 1u; }
               }
             }
           }
         }
+        gk += num_kb;
         if (warp < 2 + kEpiWarps && ok) {
           ok = epilogue_tile(m_blk, n_blk, acc, acc_phase);
           if (++acc == C::kAccSets) { acc = 0; acc_phase ^= 1u; }
