@@ -19,9 +19,12 @@
 //               quadrant each); with MT = 1 the next tile is already being
 //               multiplied meanwhile
 //   warps 2-17  (packed-weight kernels only) expand N-bit codes into the bf16 B
-//               operand stage, (q - z) * s exactly, rounded once to bf16: two
-//               groups of eight warps take alternate K blocks, one 64-code row per
-//               thread, so two stages are being expanded at any time.  Warps 2-5
+//               operand, (q - z) * s exactly, rounded once to bf16.  That operand
+//               has a ring of four stages of its own (the TMA-fed A ring has
+//               three), and two groups of eight warps take alternate runs of one
+//               or two K blocks, one 64-code row per thread and K block, so two
+//               stages are being expanded at any time and each group owns two of
+//               the four.  Warps 2-5
 //               then run the epilogue of the tile (MT = 2: nothing overlaps it
 //               anyway, and the other warps meanwhile pre-expand the next tile's
 //               first stages up to the point where they need these four)
@@ -74,17 +77,29 @@ struct Cfg {
   static constexpr int kTileM = MT * BM;                 // output rows per CTA tile
   static constexpr int kAccSets = MT == 1 ? 2 : 1;       // TMEM holds kAccSets * MT accumulators of BN columns
   static constexpr int kStages = MT == 2 ? 3 : (BN == 256 ? 4 : 6);
+  // Packed kernels keep the expanded B operand in a ring of its own, one stage deeper than the TMA-fed A
+  // ring: an expansion takes longer than a copy, and the extra B stage is what lets it run a K block further
+  // ahead of the tensor core.  Dense kernels keep A and B of a stage side by side.
+  static constexpr int kStagesB = PACKED ? kStages + 1 : kStages;
   static constexpr int kABytes = kTileM * BK * 2;
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kRingBytes = kStages * kABytes + kStagesB * kBBytes;
+  __host__ __device__ static constexpr int a_offset(int stage) { return PACKED ? stage * kABytes : stage * kStageBytes; }
+  __host__ __device__ static constexpr int b_offset(int stage_b) {
+    return PACKED ? kStages * kABytes + stage_b * kBBytes : stage_b * kStageBytes + kABytes;
+  }
   static constexpr int kThreads = (2 + (PACKED ? kDeqWarps : kEpiWarps)) * 32;
   static constexpr int kTmemCols = kAccSets * MT * BN;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static_assert(kSmemBytes <= 232448, "stage rings exceed the shared memory of one CTA");
 };
 
 struct Control {
-  uint64_t full[8];
+  uint64_t full[8];          // A (and, dense kernels, B) stage filled by TMA
   uint64_t empty[8];
+  uint64_t full_b[4];        // packed kernels: B stage expanded
+  uint64_t empty_b[4];
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
   uint64_t drain;
@@ -255,7 +270,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;                                  // 1024-byte aligned stages
   const uint32_t smem_base = raw_addr + pad;
-  Control* ctl = reinterpret_cast<Control*>(smem + C::kStages * C::kStageBytes);
+  Control* ctl = reinterpret_cast<Control*>(smem + C::kRingBytes);
   volatile int* abort_flag = &ctl->abort;
 
   const int warp = threadIdx.x >> 5;
@@ -267,8 +282,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
-      ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), PACKED ? 1 + kDeqWarps / 2 : 1);
+      ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), 1);
       ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), 1);
+    }
+    if (PACKED) {
+      for (int s = 0; s < C::kStagesB; ++s) {
+        ptx::mbar_init(ptx::smem_addr(&ctl->full_b[s]), kDeqWarps / 2);
+        ptx::mbar_init(ptx::smem_addr(&ctl->empty_b[s]), 1);
+      }
     }
     for (int a = 0; a < C::kAccSets; ++a) {
       ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[a]), 1);
@@ -385,8 +406,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             break;
           }
           const uint32_t full = ptx::smem_addr(&ctl->full[stage]);
-          const uint32_t a_dst = smem_base + stage * C::kStageBytes;
-          const uint32_t b_dst = a_dst + C::kABytes;
+          const uint32_t a_dst = smem_base + C::a_offset(stage);
+          const uint32_t b_dst = smem_base + C::b_offset(stage);
           ptx::mbar_expect_tx(full, PACKED ? C::kABytes : C::kStageBytes);
           if (A_MN) {
 #pragma unroll
@@ -432,8 +453,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       constexpr uint32_t a_lbo = A_MN ? BK * 128 : 16, b_lbo = B_MN ? BK * 128 : 16;
       constexpr uint32_t a_step = A_MN ? UMMA_K * 128 : UMMA_K * 2, b_step = B_MN ? UMMA_K * 128 : UMMA_K * 2;
       constexpr uint32_t a_half = BM * BK * 2;        // second 128-row half of the A stage (either major)
-      int stage = 0;
-      uint32_t phase = 0;
+      int stage = 0, stage_b = 0;
+      uint32_t phase = 0, phase_b = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
@@ -442,13 +463,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MT * BN);
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!wait_bounded(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL, PACKED ? 32 : 0)) {
+          if (!wait_bounded(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL, PACKED ? 32 : 0) ||
+              (PACKED &&
+               !wait_bounded(ptx::smem_addr(&ctl->full_b[stage_b]), phase_b, abort_flag, WAIT_MMA_FULL, 32))) {
             ok = false;
             break;
           }
           ptx::tc_fence_after();
-          const uint32_t a_addr = smem_base + stage * C::kStageBytes;
-          const uint32_t b_addr = a_addr + C::kABytes;
+          const uint32_t a_addr = smem_base + C::a_offset(stage);
+          const uint32_t b_addr = smem_base + C::b_offset(PACKED ? stage_b : stage);
 #pragma unroll
           for (int kk = 0; kk < BK / UMMA_K; ++kk) {
             const uint64_t b_desc = smem_desc(b_addr + kk * b_step, b_lbo);
@@ -459,6 +482,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
           ptx::mma_commit(ptx::smem_addr(&ctl->empty[stage]));
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+          if (PACKED) {
+            ptx::mma_commit(ptx::smem_addr(&ctl->empty_b[stage_b]));
+            if (++stage_b == C::kStagesB) { stage_b = 0; phase_b ^= 1u; }
+          }
         }
         if (!ok) break;
         ptx::mma_commit(ptx::smem_addr(&ctl->acc_full[acc]));
@@ -512,19 +539,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       };
       SzBlock sz_cur = {make_uint2(0u, 0u), 0u}, sz_nxt = {make_uint2(0u, 0u), 0u};
       int sz_blk = -1;
-      // Register ring of two units: the loads for the thread's next-but-one K block
-      // (four K blocks ahead) are issued as soon as the current one has been expanded.
-      uint32_t ring_w[2][2 * BITS];
-      float ring_s[2], ring_z[2];
-      const size_t code_step = 2 * (B_MN ? (size_t)BK * pitch : (size_t)(8 * BITS));   // bytes per two K blocks
-      const size_t sz_step = B_MN ? (size_t)2 * BK * groups_per_row : 0;               // groups per two K blocks
+      // Each group takes alternate runs of R consecutive K blocks (counted over all tiles of this CTA).  R = 2
+      // for 2-bit codes with a K-major operand: the 2 x 16 bytes of a run are one 32-byte sector of the packed
+      // row, fetched by one thread with one load, instead of by two warps at unrelated times.
+      // Register ring of two runs: the loads for the thread's next-but-one run (4R K blocks ahead) are issued
+      // as soon as the current run has been expanded.
+      constexpr int R = (!B_MN && BITS == 2) ? 2 : 1;
+      static_assert(C::kStagesB == 4, "stage and phase of a K block are taken from its index mod 4");
+      uint32_t ring_w[2][R][2 * BITS];
+      float ring_s[2][R], ring_z[2][R];
+      const size_t code_step = 2 * R * (B_MN ? (size_t)BK * pitch : (size_t)(8 * BITS));   // bytes per two runs
+      const size_t sz_step = B_MN ? (size_t)2 * BK * groups_per_row : 0;                   // groups per two runs
       long gk = 0;                                                // global index of the tile's K block 0
       int acc = 0;
       uint32_t acc_phase = 0;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
         tile_coords(tile, num_m, num_n, m_blk, n_blk);
-        const int kb_first = (int)((grp - gk) & 1);               // this group's first K block of the tile
+        // this group's first K block of the tile (R = 2: K is a multiple of 128, so gk is even)
+        const int kb_first = R * (int)((grp - gk / R) & 1);
         const int wrow0 = B_MN ? kb_first * BK + kr : n_blk * BN + t;
         const int unit0 = B_MN ? n_blk * (BN / 64) + box : kb_first;
         const bool valid = B_MN ? (unit0 < chunks_in) : (wrow0 < p.out_features);
@@ -532,14 +565,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         const size_t g0 = valid ? (size_t)wrow0 * groups_per_row + (B_MN ? ((unit0 << 6) >> p.group_shift) : 0) : 0;
         const eqat_fp16* s_ptr = p.s16 + g0;                      // K-major: group 0 of the row
         const uint8_t* z_ptr = p.z8 + g0;
-        auto fetch = [&](int j, int kb) {                         // kb: the K block being fetched
+        auto fetch = [&](int j, int kb) {                         // kb: first K block of the run being fetched
           if (valid) {
-            load_codes64<BITS>(code_ptr, ring_w[j]);
+            if constexpr (R == 2) {
+              ptx::ldg_256(code_ptr, reinterpret_cast<uint32_t(&)[8]>(ring_w[j][0][0]));
+            } else {
+              load_codes64<BITS>(code_ptr, ring_w[j][0]);
+            }
             code_ptr += code_step;
             if (!sz_blocks) {
-              const size_t gi = B_MN ? 0 : (size_t)((kb << 6) >> p.group_shift);
-              ring_s[j] = __half2float(__ushort_as_half(__ldg(s_ptr + gi)));
-              ring_z[j] = (float)__ldg(z_ptr + gi);
+#pragma unroll
+              for (int u = 0; u < R; ++u) {
+                const size_t gi = B_MN ? 0 : (size_t)(((kb + u) << 6) >> p.group_shift);
+                ring_s[j][u] = __half2float(__ushort_as_half(__ldg(s_ptr + gi)));
+                ring_z[j][u] = (float)__ldg(z_ptr + gi);
+              }
               if (B_MN) { s_ptr += sz_step; z_ptr += sz_step; }
             }
           }
@@ -552,51 +592,55 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         };
 #pragma unroll
         for (int j = 0; j < 2; ++j)
-          if (kb_first + 2 * j < num_kb) fetch(j, kb_first + 2 * j);
+          if (kb_first + 2 * R * j < num_kb) fetch(j, kb_first + 2 * R * j);
         if (sz_blocks) {
-          fetch_sz(sz_cur, 0);
-          fetch_sz(sz_nxt, 1);
-          sz_blk = 0;
+          const int blk0 = ((kb_first << 6) >> p.group_shift) >> 2;
+          fetch_sz(sz_cur, blk0);
+          fetch_sz(sz_nxt, blk0 + 1);
+          sz_blk = blk0;
         }
-        int stage = (int)((gk + kb_first) % C::kStages);
-        uint32_t phase = (uint32_t)(((gk + kb_first) / C::kStages) & 1);
-        for (int kb0 = kb_first; kb0 < num_kb && ok; kb0 += 4) {
+        for (int kb0 = kb_first; kb0 < num_kb && ok; kb0 += 4 * R) {
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
-            const int kb = kb0 + 2 * j;
-            if (ok && kb < num_kb) {
-              if (sz_blocks) {
-                const int blk = ((kb << 6) >> p.group_shift) >> 2;
-                if (blk != sz_blk) {
-                  sz_cur = sz_nxt;
-                  sz_blk = blk;
-                  fetch_sz(sz_nxt, blk + 1);
-                }
-              }
-              if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_DEQ_OPERAND_EMPTY)) {
-                ok = false;
-              } else {
-                uint8_t* row = smem + stage * C::kStageBytes + C::kABytes + smem_row_off;
-                if (valid) {
-                  float sv = ring_s[j], zv = ring_z[j];
-                  if (sz_blocks) {
-                    const int sub = ((kb << 6) >> p.group_shift) & 3;
-                    const uint32_t sw = (sub & 2) ? sz_cur.s4.y : sz_cur.s4.x;
-                    sv = __half2float(__ushort_as_half((unsigned short)((sub & 1) ? (sw >> 16) : (sw & 0xFFFFu))));
-                    zv = (float)((sz_cur.z4 >> (8 * sub)) & 0xFFu);
-                  }
-                  dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][0]), sv, zv, row, rx, 0);
-                  dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][BITS]), sv, zv, row, rx, 1);
-                } else {
 #pragma unroll
-                  for (int c = 0; c < 8; ++c) reinterpret_cast<uint4*>(row)[c] = make_uint4(0u, 0u, 0u, 0u);
+            for (int u = 0; u < R; ++u) {
+              const int kb = kb0 + 2 * R * j + u;
+              if (ok && kb < num_kb) {
+                if (sz_blocks) {
+                  const int blk = ((kb << 6) >> p.group_shift) >> 2;
+                  if (blk != sz_blk) {
+                    sz_cur = sz_nxt;
+                    sz_blk = blk;
+                    fetch_sz(sz_nxt, blk + 1);
+                  }
                 }
-                if (kb + 4 < num_kb) fetch(j, kb + 4);
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full[stage]));
-                stage += 2;                                       // this group's next K block is two further
-                if (stage >= C::kStages) { stage -= C::kStages; phase ^= 1u; }
+                const int stage = (int)((gk + kb) & 3);
+                const uint32_t phase = (uint32_t)(((gk + kb) >> 2) & 1);
+                if (!wait_bounded(ptx::smem_addr(&ctl->empty_b[stage]), phase ^ 1u, abort_flag,
+                                  WAIT_DEQ_OPERAND_EMPTY)) {
+                  ok = false;
+                } else {
+                  uint8_t* row = smem + C::b_offset(stage) + smem_row_off;
+                  if (valid) {
+                    float sv = ring_s[j][u], zv = ring_z[j][u];
+                    if (sz_blocks) {
+                      const int sub = ((kb << 6) >> p.group_shift) & 3;
+                      const uint32_t sw = (sub & 2) ? sz_cur.s4.y : sz_cur.s4.x;
+                      sv = __half2float(__ushort_as_half((unsigned short)((sub & 1) ? (sw >> 16) : (sw & 0xFFFFu))));
+                      zv = (float)((sz_cur.z4 >> (8 * sub)) & 0xFFu);
+                    }
+                    dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][u][0]), sv, zv, row, rx, 0);
+                    dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][u][BITS]), sv, zv, row, rx,
+                                         1);
+                  } else {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) reinterpret_cast<uint4*>(row)[c] = make_uint4(0u, 0u, 0u, 0u);
+                  }
+                  if (u == R - 1 && kb - (R - 1) + 4 * R < num_kb) fetch(j, kb - (R - 1) + 4 * R);
+                  ptx::fence_proxy_async_smem();
+                  __syncwarp();
+                  if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full_b[stage]));
+                }
               }
             }
           }
