@@ -166,16 +166,17 @@ struct DequantScale {
   __device__ __forceinline__ float operator()(uint32_t xbits) const { return fmaf(__uint_as_float(xbits), sp, cz); }
 };
 
-__device__ __forceinline__ void store_chunk(uint8_t* row, int chunk, int rx, const float (&v)[8]) {
-  const uint4 o = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
-                             pack_bf16x2(v[6], v[7]));
-  *reinterpret_cast<uint4*>(row + ((chunk ^ rx) << 4)) = o;
+//
+// `row_sx` is the shared-memory address of the row XOR (rx << 4): the row is 128-byte aligned, so chunk c
+// lies at row_sx ^ (c << 4), one logic operation per store.
+__device__ __forceinline__ void store_chunk(uint32_t row_sx, int chunk, const float (&v)[8]) {
+  ptx::sts_128(row_sx ^ ((uint32_t)chunk << 4), pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+               pack_bf16x2(v[6], v[7]));
 }
 
 // Expands 32 consecutive codes (half h of a 64-code row) into chunks 4h .. 4h+3.
 template <int BITS>
-__device__ __forceinline__ void dequant_half32(const uint32_t (&w)[BITS], float s, float z, uint8_t* row, int rx,
-                                               int h) {
+__device__ __forceinline__ void dequant_half32(const uint32_t (&w)[BITS], float s, float z, uint32_t row_sx, int h) {
   constexpr uint32_t kMagic = 0x4B000000u;
   if constexpr (BITS == 2) {
     // Four possible values per group: build them once, exactly, as bf16
@@ -201,7 +202,7 @@ __device__ __forceinline__ void dequant_half32(const uint32_t (&w)[BITS], float 
           const uint32_t pair_sel = __byte_perm(sel[r], sel[r + 1], b | ((4u + b) << 4));
           o[pr] = __byte_perm(lut01, lut23, pair_sel);
         }
-        *reinterpret_cast<uint4*>(row + (((4 * h + 2 * i + c) ^ rx) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+        ptx::sts_128(row_sx ^ ((uint32_t)(4 * h + 2 * i + c) << 4), o[0], o[1], o[2], o[3]);
       }
     }
   } else if constexpr (BITS == 4) {
@@ -213,7 +214,7 @@ __device__ __forceinline__ void dequant_half32(const uint32_t (&w)[BITS], float 
 #pragma unroll
       for (int e = 0; e < 8; ++e)
         v[e] = f(__byte_perm((e & 1) ? m1 : m0, kMagic, 0x7044u | ((uint32_t)(e >> 1) << 8)));
-      store_chunk(row, 4 * h + i, rx, v);
+      store_chunk(row_sx, 4 * h + i, v);
     }
   } else {
     const DequantScale f(s, z);
@@ -232,7 +233,7 @@ __device__ __forceinline__ void dequant_half32(const uint32_t (&w)[BITS], float 
         }
         v[e] = f((t & 0x00070000u) | kMagic);
       }
-      store_chunk(row, 4 * h + c, rx, v);
+      store_chunk(row_sx, 4 * h + c, v);
     }
   }
 }
@@ -526,6 +527,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       const int box = (t >> 3) & 3;                               // MN-major: 64-column box 0..3
       const int smem_row_off = B_MN ? (box * (BK * 128) + kr * 128) : t * 128;
       const int rx = B_MN ? (kr & 7) : (t & 7);
+      const uint32_t smem_row_sx = (uint32_t)smem_row_off ^ ((uint32_t)rx << 4);   // stage bases are 1024-byte aligned
       // Step sizes and zero points.  With a K-major B operand a thread stays on one
       // weight row for a whole tile and walks its groups in order, so it reads
       // them four groups at a time (one 8-byte and one 4-byte load per four
@@ -620,7 +622,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                                   WAIT_DEQ_OPERAND_EMPTY)) {
                   ok = false;
                 } else {
-                  uint8_t* row = smem + C::b_offset(stage) + smem_row_off;
+                  const uint32_t row_sx = smem_base + C::b_offset(stage) + smem_row_sx;
                   if (valid) {
                     float sv = ring_s[j][u], zv = ring_z[j][u];
                     if (sz_blocks) {
@@ -629,12 +631,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                       sv = __half2float(__ushort_as_half((unsigned short)((sub & 1) ? (sw >> 16) : (sw & 0xFFFFu))));
                       zv = (float)((sz_cur.z4 >> (8 * sub)) & 0xFFu);
                     }
-                    dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][u][0]), sv, zv, row, rx, 0);
-                    dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][u][BITS]), sv, zv, row, rx,
-                                         1);
+                    dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][u][0]), sv, zv, row_sx, 0);
+                    dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][u][BITS]), sv, zv, row_sx, 1);
                   } else {
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) reinterpret_cast<uint4*>(row)[c] = make_uint4(0u, 0u, 0u, 0u);
+                    for (int c = 0; c < 8; ++c) ptx::sts_128(row_sx ^ ((uint32_t)c << 4), 0u, 0u, 0u, 0u);
                   }
                   if (u == R - 1 && kb - (R - 1) + 4 * R < num_kb) fetch(j, kb - (R - 1) + 4 * R);
                   ptx::fence_proxy_async_smem();

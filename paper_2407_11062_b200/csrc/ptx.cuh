@@ -110,5 +110,10 @@ __device__ __forceinline__ void ldg_256(const void* p, uint32_t (&r)[8]) {
                : "l"(p));
 }
 
+// 16-byte store to a 32-bit shared-memory address.
+__device__ __forceinline__ void sts_128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 }  // namespace ptx
 }  // namespace eqat
