@@ -161,7 +161,7 @@ class BlockWorkload:
                                         z8=torch.empty(out, ng, dtype=torch.uint8, device=dev),
                                         s16=torch.empty(out, ng, dtype=torch.float16, device=dev)))
         self.calls_per_step = 8 * len(self.layers)
-        self.kernels_per_step = 11 * len(self.layers)     # fwd = 2 kernels, bwd = 3, the other six calls 1 each
+        self.kernels_per_step = 10 * len(self.layers)     # fwd = 2 kernels, bwd = 2 (group <= 256), the other six calls 1 each
 
     def step(self, timers=None):
         e = self.eqat

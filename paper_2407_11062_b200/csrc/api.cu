@@ -138,6 +138,9 @@ int qlinear_fakequant_bwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf1
   eqat_bf16* dW_hat = static_cast<eqat_bf16*>(workspace);
   cudaStream_t st = as_stream(stream);
   EQAT_TRY(launch_dense_dx(*d, dY, W_hat, dX, st));
+  // A group that fits inside one output tile is reduced in the weight-gradient GEMM's epilogue; a longer one
+  // (channel-wise quantisation) spans tiles, so its gradient goes through the workspace and a second kernel.
+  if (d->group <= 256) return launch_dense_dw_ste(*d, dY, X, W, s, z, dW, ds, dz, st);
   EQAT_TRY(launch_dense_dw(*d, dY, X, dW_hat, st));
   return launch_ste_bwd(*d, dW_hat, W, s, z, dW, ds, dz, st);
 }

@@ -42,6 +42,7 @@
 #include "codec.cuh"
 #include "gemm.cuh"
 #include "ptx.cuh"
+#include "quant_math.cuh"
 
 namespace eqat {
 
@@ -57,7 +58,7 @@ constexpr int kDeqWarps = 16;      // packed kernels: warps 2-17 expand codes; w
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s per wait
 constexpr uint64_t kDrainLimitNs = 50000000ull;    // 50 ms per stage at teardown
 
-enum Epilogue : int { EPI_STORE = 0, EPI_DS = 1 };
+enum Epilogue : int { EPI_STORE = 0, EPI_DS = 1, EPI_STE = 2 };
 
 struct GemmParams {
   int M, N, K;
@@ -68,8 +69,14 @@ struct GemmParams {
   const uint8_t* z8;         // [out, in/group]
   int out_features, in_features;
   int group_shift;           // log2(group)
-  float* ds;                 // EPI_DS outputs [out, in/group]
+  float* ds;                 // EPI_DS / EPI_STE outputs [out, in/group]
   float* dz;                 // may be null
+  // EPI_STE: latent weight and Block-AP quantiser parameters of the [out,in] tile rows
+  const eqat_bf16* W;        // [out, in]
+  const float* s32;          // [out, in/group]
+  const float* z32;          // [out, in/group]
+  float Q;                   // 2^N - 1
+  int dz_literal;            // Eq. 4 clamped branch: -1 instead of -s
 };
 
 template <int BN, int MT, bool PACKED>
@@ -343,6 +350,59 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])));
                 *reinterpret_cast<uint4*>(drow + col0 + v * 8) = o;
               }
+            }
+          }
+        }
+      } else if constexpr (EPI == EPI_STE) {
+        // Block-AP: the accumulator row is the gradient of row m of W_hat.  Eqs. 3-5 are applied to it here,
+        // in fp32, next to the matching latent weights: dW = G where the code is in range, ds and dz are the
+        // group sums of G times the partials.  G itself is never written.
+        const int groups_per_row = p.N >> p.group_shift;
+        const int chunks_per_group = 1 << (p.group_shift - 5);
+        const eqat_bf16* wrow = p.W + (size_t)m * p.N;
+        eqat_bf16* drow = p.D + (size_t)m * p.N;
+        float acc_s = 0.0f, acc_g = 0.0f;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          const int col0 = n_blk * BN + c * 32;
+          const bool live = m < p.M && col0 < p.N;
+          uint4 wraw[4];
+          float sv = 1.0f, zr = 0.0f;
+          if (live) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) wraw[v] = __ldg(reinterpret_cast<const uint4*>(wrow + col0) + v);
+            const size_t gi = (size_t)m * groups_per_row + (col0 >> p.group_shift);
+            sv = __ldg(p.s32 + gi);
+            zr = rintf(__ldg(p.z32 + gi));
+          }
+          uint32_t r32[32];
+          ptx::tmem_ld_32x32(t_row + c * 32, r32);
+          ptx::tmem_ld_wait();
+          if (live) {
+            const float rs = group_rcp(sv);
+            const float lo = -zr, hi = p.Q - zr;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              float w[8], r[8], rt[8];
+              unpack8(wraw[v], w);
+              quotient_round8(w, sv, rs, r, rt);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float gr = __uint_as_float(r32[8 * v + i]);
+                const float cl = fminf(fmaxf(r[i], lo), hi);
+                const bool inside = (cl == r[i]);
+                acc_s = fmaf(gr, inside ? rt[i] : cl, acc_s);     // Eq. 3
+                acc_g += inside ? 0.0f : gr;                      // Eq. 4
+                w[i] = inside ? gr : 0.0f;                        // Eq. 5
+              }
+              reinterpret_cast<uint4*>(drow + col0)[v] = pack8(w);
+            }
+            if (((c + 1) & (chunks_per_group - 1)) == 0) {
+              const size_t gi = (size_t)m * groups_per_row + (col0 >> p.group_shift);
+              p.ds[gi] = acc_s;
+              if (p.dz != nullptr) p.dz[gi] = (p.dz_literal ? -1.0f : -sv) * acc_g;
+              acc_s = 0.0f;
+              acc_g = 0.0f;
             }
           }
         }
@@ -784,6 +844,22 @@ int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X,
   p.D = dWhat;
   return dense_row_tiles(p.M, p.N) == 2 ? launch<256, 2, true, true, false, EPI_STORE, 2>(ta, tb, p, st)
                                         : launch<256, 1, true, true, false, EPI_STORE, 2>(ta, tb, p, st);
+}
+
+int launch_dense_dw_ste(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X, const eqat_bf16* W, const float* s,
+                        const float* z, eqat_bf16* dW, float* ds, float* dz, cudaStream_t st) {
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, dY, d.out_features, d.tokens, BK) || !make_tmap(&tb, X, d.in_features, d.tokens, BK))
+    return EQAT_ERR_CUDA;
+  GemmParams p = base_params(d.out_features, d.in_features, (int)d.tokens);
+  p.D = dW;
+  p.W = W; p.s32 = s; p.z32 = z;
+  p.ds = ds; p.dz = dz;
+  p.group_shift = log2_exact(d.group);
+  p.Q = (float)((1 << d.bits) - 1);
+  p.dz_literal = d.dz_mode;
+  // 128-row tiles: with two accumulator sets this epilogue, the longest of the three, runs under the next tile
+  return launch<256, 1, true, true, false, EPI_STE, 2>(ta, tb, p, st);
 }
 
 int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,

@@ -11,6 +11,10 @@ int launch_dense_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* Wh
 int launch_dense_dx(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* What, eqat_bf16* dX, cudaStream_t st);
 // dWhat[out,in] = dY[T,out]^T * X[T,in]
 int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X, eqat_bf16* dWhat, cudaStream_t st);
+// The same contraction with Eqs. 3-5 applied in its epilogue (group <= 256): writes dW, ds and optionally dz;
+// the gradient of W_hat is never stored.
+int launch_dense_dw_ste(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X, const eqat_bf16* W, const float* s,
+                        const float* z, eqat_bf16* dW, float* ds, float* dz, cudaStream_t st);
 // Y = X * dequant(Wq)^T and dX = dY * dequant(Wq), codes expanded in shared memory
 int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
                       const uint8_t* z8, eqat_bf16* Y, cudaStream_t st);

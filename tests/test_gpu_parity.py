@@ -242,6 +242,9 @@ def test_block_ap_config1(eqat):
     (64, 128, 1, 2, 64),            # a single token, a single K block pair
     (320, 640, 129, 3, 128),        # one row past a tile boundary
     (1024, 256, 520, 2, 256),
+    (128, 256, 200, 4, 32),         # one 32-column accumulator chunk per group
+    (128, 1024, 260, 3, 512),       # groups longer than an output tile: gradient goes through the workspace
+    (192, 1024, 64, 2, 1024),       # channel-wise
 ])
 def test_block_ap_ragged(eqat, out, in_f, tokens, bits, group):
     cfg = small_cfg(f"rag_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens, "student_t4", 0.02, 0.01)

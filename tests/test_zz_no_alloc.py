@@ -37,9 +37,13 @@ def test_rejects_problems_larger_than_the_builtin_scratch(eqat):
 
 
 @pytest.mark.gpu
-def test_matches_the_workspace_variant_twice_in_a_row(eqat):
+@pytest.mark.parametrize("channel_wise", [True, False])
+def test_matches_the_workspace_variant_twice_in_a_row(eqat, channel_wise):
+    """Channel-wise groups are the case that uses the scratch (a group longer than an output tile sends the
+    gradient of W_hat through memory); the short-group case checks that the entry point agrees there too."""
     cfg = get_config("c1"); lin = cfg.linears[0]
-    out, in_f, T, bits, g = lin.out_features, lin.in_features, cfg.tokens, cfg.bits, cfg.group
+    out, in_f, T, bits = lin.out_features, lin.in_features, cfg.tokens, cfg.bits
+    g = in_f if channel_wise else cfg.group
     ng = in_f // g
     Wb = weight_for(cfg, lin); Xb, dYb = activations_for(cfg, lin)
     s, z = O.minmax_init(f32(Wb), bits, g)
