@@ -63,6 +63,7 @@ enum Epilogue : int { EPI_STORE = 0, EPI_DS = 1, EPI_STE = 2 };
 struct GemmParams {
   int M, N, K;
   eqat_bf16* D;              // EPI_STORE: [M,N] row-major
+  int wide_store;            // D is 32-byte aligned: rows can be written a sector per lane
   // packed weight (B operand of the packed kernels, epilogue operand of EPI_DS)
   const uint8_t* Wq;         // [out, in*bits/8]
   const eqat_fp16* s16;      // [out, in/group]
@@ -340,15 +341,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           ptx::tmem_ld_wait();
           const int col0 = n_blk * BN + c * 32;
           if (m < p.M) {
+            // A lane owns a row, so the lanes of a store instruction hit 32 different lines and the stores,
+            // not the TMEM loads, set the pace of this epilogue: write whole 32-byte sectors where the
+            // output is aligned for it (N is a multiple of 16 for every shape the library accepts).
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              if (col0 + v * 8 < p.N) {
-                const uint4 o = make_uint4(
-                    pack_bf16x2(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1])),
-                    pack_bf16x2(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3])),
-                    pack_bf16x2(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5])),
-                    pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])));
-                *reinterpret_cast<uint4*>(drow + col0 + v * 8) = o;
+            for (int v = 0; v < 2; ++v) {
+              if (col0 + v * 16 < p.N) {
+                uint32_t o[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                  o[i] = pack_bf16x2(__uint_as_float(r[16 * v + 2 * i]), __uint_as_float(r[16 * v + 2 * i + 1]));
+                if (p.wide_store) {
+                  ptx::stg_256(drow + col0 + v * 16, o);
+                } else {
+                  reinterpret_cast<uint4*>(drow + col0 + v * 16)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                  reinterpret_cast<uint4*>(drow + col0 + v * 16)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                }
               }
             }
           }
@@ -805,6 +813,11 @@ GemmParams base_params(int M, int N, int K) {
   return p;
 }
 
+void set_output(GemmParams& p, eqat_bf16* D) {
+  p.D = D;
+  p.wide_store = (reinterpret_cast<uintptr_t>(D) & 31u) == 0 && (p.N & 15) == 0;
+}
+
 void set_weight(GemmParams& p, const eqat_desc& d, const uint8_t* Wq, const eqat_fp16* s16, const uint8_t* z8) {
   p.Wq = Wq; p.s16 = s16; p.z8 = z8;
   p.out_features = d.out_features;
@@ -817,7 +830,7 @@ void set_weight(GemmParams& p, const eqat_desc& d, const uint8_t* Wq, const eqat
 int launch_dense_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* What, eqat_bf16* Y, cudaStream_t st) {
   CUtensorMap ta, tb;
   GemmParams p = base_params((int)d.tokens, d.out_features, d.in_features);
-  p.D = Y;
+  set_output(p, Y);
   const int mt = dense_row_tiles(p.M, p.N);
   if (!make_tmap(&ta, X, d.in_features, d.tokens, mt * BM) || !make_tmap(&tb, What, d.in_features, d.out_features, 256))
     return EQAT_ERR_CUDA;
@@ -828,7 +841,7 @@ int launch_dense_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* Wh
 int launch_dense_dx(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* What, eqat_bf16* dX, cudaStream_t st) {
   CUtensorMap ta, tb;
   GemmParams p = base_params((int)d.tokens, d.in_features, d.out_features);
-  p.D = dX;
+  set_output(p, dX);
   const int mt = dense_row_tiles(p.M, p.N);
   if (!make_tmap(&ta, dY, d.out_features, d.tokens, mt * BM) || !make_tmap(&tb, What, d.in_features, d.out_features, BK))
     return EQAT_ERR_CUDA;
@@ -841,7 +854,7 @@ int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X,
   if (!make_tmap(&ta, dY, d.out_features, d.tokens, BK) || !make_tmap(&tb, X, d.in_features, d.tokens, BK))
     return EQAT_ERR_CUDA;
   GemmParams p = base_params(d.out_features, d.in_features, (int)d.tokens);
-  p.D = dWhat;
+  set_output(p, dWhat);
   return dense_row_tiles(p.M, p.N) == 2 ? launch<256, 2, true, true, false, EPI_STORE, 2>(ta, tb, p, st)
                                         : launch<256, 1, true, true, false, EPI_STORE, 2>(ta, tb, p, st);
 }
@@ -852,7 +865,7 @@ int launch_dense_dw_ste(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16
   if (!make_tmap(&ta, dY, d.out_features, d.tokens, BK) || !make_tmap(&tb, X, d.in_features, d.tokens, BK))
     return EQAT_ERR_CUDA;
   GemmParams p = base_params(d.out_features, d.in_features, (int)d.tokens);
-  p.D = dW;
+  set_output(p, dW);
   p.W = W; p.s32 = s; p.z32 = z;
   p.ds = ds; p.dz = dz;
   p.group_shift = log2_exact(d.group);
@@ -867,7 +880,7 @@ int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq,
   CUtensorMap ta;
   if (!make_tmap(&ta, X, d.in_features, d.tokens, 2 * BM)) return EQAT_ERR_CUDA;
   GemmParams p = base_params((int)d.tokens, d.out_features, d.in_features);
-  p.D = Y;
+  set_output(p, Y);
   set_weight(p, d, Wq, s16, z8);
   switch (d.bits) {
     case 2: return launch<256, 2, false, false, true, EPI_STORE, 2>(ta, ta, p, st);
@@ -881,7 +894,7 @@ int launch_packed_dx(const eqat_desc& d, const eqat_bf16* dY, const uint8_t* Wq,
   CUtensorMap ta;
   if (!make_tmap(&ta, dY, d.out_features, d.tokens, 2 * BM)) return EQAT_ERR_CUDA;
   GemmParams p = base_params((int)d.tokens, d.in_features, d.out_features);
-  p.D = dX;
+  set_output(p, dX);
   set_weight(p, d, Wq, s16, z8);
   switch (d.bits) {
     case 2: return launch<256, 2, false, true, true, EPI_STORE, 2>(ta, ta, p, st);

@@ -255,6 +255,31 @@ def test_block_ap_ragged(eqat, out, in_f, tokens, bits, group):
     check_block_ap(r, s, z, bits, group)
 
 
+def test_outputs_aligned_to_16_bytes_only(eqat):
+    """Outputs that are 16- but not 32-byte aligned take the narrower store path: same bits."""
+    cfg = get_config("c1"); lin = cfg.linears[0]
+    out, in_f, T = lin.out_features, lin.in_features, cfg.tokens
+    s, z = O.minmax_init(f32(weight_for(cfg, lin)), cfg.bits, cfg.group)
+    Wd = bits_to_torch(weight_for(cfg, lin)); Xb, dYb = activations_for(cfg, lin, T)
+    Xd, dYd, sd, zd = bits_to_torch(Xb), bits_to_torch(dYb), dev(s), dev(z)
+    d = eqat.make_desc(cfg.bits, cfg.group, out, in_f, T)
+    What = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD), dtype=torch.uint8, device="cuda")
+    res = []
+    for shift in (0, 8):                                         # elements: 0 or 16 bytes past a 512-byte boundary
+        Y = torch.zeros(T * out + 16, dtype=torch.bfloat16, device="cuda")[shift:shift + T * out].view(T, out)
+        dX = torch.zeros(T * in_f + 16, dtype=torch.bfloat16, device="cuda")[shift:shift + T * in_f].view(T, in_f)
+        dW = torch.zeros(out * in_f + 16, dtype=torch.bfloat16, device="cuda")[shift:shift + out * in_f].view(out, in_f)
+        assert Y.data_ptr() % 32 == 2 * shift
+        ds = torch.empty(out, in_f // cfg.group, device="cuda"); dz = torch.empty_like(ds)
+        eqat.qlinear_fakequant_fwd(d, Xd, Wd, sd, zd, Y, What)
+        eqat.qlinear_fakequant_bwd(d, Xd, dYd, Wd, sd, zd, What, dX, dW, ds, dz, ws)
+        torch.cuda.synchronize()
+        res.append((Y.clone(), dX.clone(), dW.clone()))
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
+
+
 def test_block_ap_is_deterministic(eqat):
     cfg = get_config("c1"); lin = cfg.linears[0]
     s, z = O.minmax_init(f32(weight_for(cfg, lin)), cfg.bits, cfg.group)
