@@ -146,7 +146,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes)
          (1ull << 46) | (2ull << 61);
 }
 
+template <bool ROW_ORDER>
 __device__ __forceinline__ void tile_coords(int tile, int num_m, int num_n, int& m_blk, int& n_blk) {
+  if (ROW_ORDER) {
+    // Packed kernels: the B operand (N-bit codes, a few MB) lives in L2 whatever the order, so tiles run along
+    // a row of tiles first and each A panel is fetched by one wave of CTAs only.
+    m_blk = tile / num_n;
+    n_blk = tile - m_blk * num_n;
+    return;
+  }
   // Bands of 16 row-tiles, row-tile fastest inside a band: the ~148 tiles in
   // flight share 16 A panels and ~9 B panels in L2.
   const int band_tiles = 16 * num_n;
@@ -468,7 +476,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
-        tile_coords(tile, num_m, num_n, m_blk, n_blk);
+        tile_coords<PACKED>(tile, num_m, num_n, m_blk, n_blk);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!wait_bounded(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_PRODUCER_EMPTY, 64)) {
             ok = false;
@@ -570,7 +578,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
       int m_blk, n_blk;
-      tile_coords(tile, num_m, num_n, m_blk, n_blk);
+      tile_coords<PACKED>(tile, num_m, num_n, m_blk, n_blk);
       if (!epilogue_tile(m_blk, n_blk, acc, acc_phase)) break;
       if (++acc == C::kAccSets) { acc = 0; acc_phase ^= 1u; }
     }
@@ -625,7 +633,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       uint32_t acc_phase = 0;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
-        tile_coords(tile, num_m, num_n, m_blk, n_blk);
+        tile_coords<PACKED>(tile, num_m, num_n, m_blk, n_blk);
         // this group's first K block of the tile (R = 2: K is a multiple of 128, so gk is even)
         const int kb_first = R * (int)((grp - gk / R) & 1);
         const int wrow0 = B_MN ? kb_first * BK + kr : n_blk * BN + t;
