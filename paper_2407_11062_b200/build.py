@@ -13,7 +13,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libeqat_b200.so")
-SOURCES = ("api.cu", "elementwise.cu", "gemm.cu", "noalloc.cu", "stream.cu")
+SOURCES = ("api.cu", "elementwise.cu", "gemm.cu", "gemv.cu", "noalloc.cu", "stream.cu")
 
 
 def _nvcc() -> str:

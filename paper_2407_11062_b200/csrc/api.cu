@@ -4,6 +4,7 @@
 #include "common.cuh"
 #include "elementwise.cuh"
 #include "gemm.cuh"
+#include "gemv.cuh"
 
 namespace {
 
@@ -182,6 +183,8 @@ int qlinear_packed_fwd(const eqat_desc* d, const eqat_bf16* X, const uint8_t* Wq
                        const uint8_t* z8, eqat_bf16* Y, void* stream) {
   EQAT_TRY(check_gemm_desc(d, true));
   EQAT_TRY(check_ptrs(X, Wq_packed, s16, z8, Y));
+  // a handful of tokens (decoding): one pass over the packed weight instead of near-empty tensor-core tiles
+  if (packed_gemv_applies(*d)) return launch_packed_gemv(*d, X, Wq_packed, s16, z8, Y, as_stream(stream));
   return launch_packed_fwd(*d, X, Wq_packed, s16, z8, Y, as_stream(stream));
 }
 

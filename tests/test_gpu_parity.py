@@ -332,6 +332,33 @@ def test_e2e_small(eqat, bits, group):
     check_e2e(run_e2e(eqat, cfg, cfg.linears[0], 256), group)
 
 
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("tokens", [1, 2, 3, 4, 5])
+def test_e2e_few_tokens(eqat, bits, tokens):
+    """Decode-sized batches: up to four tokens take the matrix-vector forward kernel, five the tiled one.
+    640 = 10 units of 64 columns, fewer than the sixteen warps of a CTA (some get none); 1408 = 22 (one or two each)."""
+    group = 64 if bits == 2 else 128
+    cfg = small_cfg(f"gemv_{bits}_{tokens}", 448, 640 if group == 64 else 1408, bits, group, tokens, "student_t4", 0.02, 0.01)
+    check_e2e(run_e2e(eqat, cfg, cfg.linears[0], tokens), group)
+
+
+def test_few_token_forward_agrees_with_tiled_forward(eqat):
+    """The same rows through both forward kernels (4 tokens alone, and as the first rows of a 5-token batch)."""
+    cfg = small_cfg("gemv_vs_gemm", 512, 1024, 2, 64, 5)
+    r5 = run_e2e(eqat, cfg, cfg.linears[0], 5)
+    cfg4 = small_cfg("gemv_vs_gemm", 512, 1024, 2, 64, 4)
+    Wb = weight_for(cfg4, cfg4.linears[0])
+    assert np.array_equal(Wb, weight_for(cfg, cfg.linears[0]))
+    P_o, z8_o, s16_o = O.quantize_pack(r5["W"], r5["s"], r5["z"], 2, 64)
+    X4 = torch.from_numpy(bf16_round(r5["X"][:4]).astype(np.float32)).to(torch.bfloat16).cuda()
+    d = eqat.make_desc(2, 64, 512, 1024, 4)
+    Y4 = torch.empty(4, 512, dtype=torch.bfloat16, device="cuda")
+    s16d = torch.from_numpy(s16_o.view(np.int16)).view(torch.float16).cuda()
+    eqat.qlinear_packed_fwd(d, X4, dev(P_o), s16d, dev(z8_o), Y4)
+    torch.cuda.synchronize()
+    assert rel_err(torch_to_f64(Y4), torch_to_f64(r5["Y"][:4])) <= TOL
+
+
 @pytest.mark.parametrize("out,in_f,tokens,bits,group", [
     (192, 384, 300, 2, 64),
     (64, 128, 1, 4, 128),
