@@ -38,6 +38,34 @@ WORKLOAD = "llama2-7b decoder-block linears, w2g64: Block-AP fwd+bwd @4096 tok, 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+# DRAM bytes (read + write) per launch of the packed-weight GEMMs at 16384 tokens, w2g64, by linear shape: ncu
+# `dram__bytes_read.sum + dram__bytes_write.sum`, one capture per shape with `bench.py --kernel-case` (the summaries
+# under profiles/ give the command).  They describe the kernels whose sources hash to `sources_sha256`; once those
+# files change the figures are stale and `roofline.traffic` is reported as null.
+NCU_TRAFFIC = {
+    "sources": ("gemm.cu", "ptx.cuh"),
+    "sources_sha256": "cf228092eebbfc5e320ed3f8d3cd152718e108f4cbf03b584874890ddd5fbe36",
+    "packed_fwd": {"qkvo": 139.27e6 + 97.46e6, "gate_up": 147.76e6 + 314.98e6, "down": 442.55e6 + 114.84e6},
+    "packed_bwd_dx": {"qkvo": 139.26e6 + 98.08e6, "gate_up": 451.88e6 + 114.70e6, "down": 148.39e6 + 315.95e6},
+    "packed_bwd_ds": {"qkvo": 416.51e6 + 4.73e6, "gate_up": 1306.28e6 + 2.74e6, "down": 1073.37e6 + 3.04e6},
+}
+
+
+def traffic_per_launch(kernel_class):
+    """Launch-weighted mean of the captured DRAM bytes over the class's launches in one step, or None if the
+    kernel sources have changed since the capture."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in NCU_TRAFFIC["sources"]:
+        with open(os.path.join(ROOT, "paper_2407_11062_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    table = NCU_TRAFFIC.get(kernel_class)
+    if table is None or h.hexdigest() != NCU_TRAFFIC["sources_sha256"]:
+        return None
+    n = sum(l.count for l in LINEARS["7b"])
+    return sum(table[l.name] * l.count for l in LINEARS["7b"]) / n
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -408,7 +436,11 @@ def run_ours(args):
             ach = tot_f / (tot_ms * 1e-3) / 1e12
             peak = peaks["bf16_tflops_sustained"]
             roof = {"kernel": "gemm_kernel (" + top_class + ")", "bound": "tensor", "achieved": ach, "peak": peak,
-                    "unit": "TFLOP/s", "frac": ach / peak, "peak_source": peaks["source"] + " (sustained)", "traffic": None}
+                    "unit": "TFLOP/s", "frac": ach / peak, "peak_source": peaks["source"] + " (sustained)", "traffic": traffic_per_launch(top_class),
+                    "traffic_unit": "DRAM bytes per launch (ncu, launch-weighted mean over the class)",
+                    "algorithmic_bytes": sum((T_E2E * (l.in_features + l.out_features) * 2
+                                              + l.in_features * l.out_features * BITS // 8) * l.count
+                                             for l in LINEARS["7b"]) / sum(l.count for l in LINEARS["7b"])}
         classes = {c: {"total_ms_per_step": t / args.steps, "share": t / sum(by_class.values())} for c, t in by_class.items()}
         out = {"metric": "QLinear fwd+bwd TFLOP/s", "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": world,
                "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -452,9 +484,60 @@ def run_kernel_case(args):
     print(json.dumps({k: v for k, v in summarise(timers).items()}), flush=True)
 
 
+def run_decode_case(args):
+    """Few-token packed forward (the matrix-vector kernel) on the block's three linear shapes: device time per
+    launch from a CUDA graph of launches over rotating weight copies (more than L2 in total), and the bandwidth that
+    time means for the bytes one launch must read."""
+    torch.cuda.set_device(0)
+    from paper_2407_11062_b200.build import build_library
+    build_library()
+    from paper_2407_11062_b200 import binding as eqat
+    peaks = load_peaks()
+    dev = torch.device("cuda", 0)
+    out = {"metric": "packed forward, few tokens", "unit": "us per launch", "bits": BITS, "group": GROUP,
+           "hbm_gbs_peak": peaks["hbm_gbs"], "cases": {}}
+    for lin in LINEARS["7b"]:
+        o, i = lin.out_features, lin.in_features
+        ng = i // GROUP
+        wbytes = o * i * BITS // 8
+        copies = max(4, int(320e6 // wbytes))
+        Ps = [torch.randint(0, 256, (o, i * BITS // 8), dtype=torch.uint8, device=dev) for _ in range(copies)]
+        z8 = torch.randint(0, 1 << BITS, (o, ng), dtype=torch.uint8, device=dev)
+        s16 = (torch.rand(o, ng, device=dev) * 0.01 + 0.001).half()
+        for T in (1, 4):
+            X = torch.randn(T, i, device=dev).to(torch.bfloat16)
+            Y = torch.empty(T, o, dtype=torch.bfloat16, device=dev)
+            d = eqat.make_desc(BITS, GROUP, o, i, T)
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                for P in Ps[:3]:
+                    eqat.qlinear_packed_fwd(d, X, P, s16, z8, Y)       # warm-up, outside the capture
+                side.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    for P in Ps:
+                        eqat.qlinear_packed_fwd(d, X, P, s16, z8, Y)
+                g.replay(); side.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(side)
+                for _ in range(args.case_iters):
+                    g.replay()
+                e1.record(side)
+                side.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / (args.case_iters * copies)
+            nbytes = wbytes + o * ng * 3 + T * (i + o) * 2
+            out["cases"][f"{lin.name}/T{T}"] = {"us": us, "bytes": nbytes, "gbs": nbytes / us / 1e3,
+                                                 "frac_of_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+        del Ps
+    assert eqat.device_status() == (0, 0)
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--kernel-case", action="store_true", help="run one linear shape a few times (for profilers)")
+    ap.add_argument("--decode-case", action="store_true",
+                    help="time the few-token packed forward on the block's linear shapes (uses --case-iters)")
     ap.add_argument("--case-shape", default="qkvo", choices=[l.name for l in LINEARS["7b"]])
     ap.add_argument("--case-tokens", type=int, default=16384)
     ap.add_argument("--case-iters", type=int, default=2)
@@ -466,6 +549,8 @@ def main():
     args = ap.parse_args()
     if args.kernel_case:
         run_kernel_case(args)
+    elif args.decode_case:
+        run_decode_case(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
