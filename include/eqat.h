@@ -125,9 +125,13 @@ int qlinear_fakequant_fwd(const eqat_desc* desc, const eqat_bf16* X, const eqat_
 int eqat_ste_bwd(const eqat_desc* desc, const eqat_bf16* dW_hat, const eqat_bf16* W, const float* s,
                  const float* z, eqat_bf16* dW, float* ds, float* dz, void* stream);
 
-/* Block-AP backward: dX = dY * W_hat, dW_hat = dY^T * X (kept in bf16 in the
- * workspace), then eqat_ste_bwd.  Needs eqat_workspace_bytes(desc,
- * EQAT_OP_FAKEQUANT_BWD) bytes of scratch.
+/* Block-AP backward: dX = dY * W_hat, dW_hat = dY^T * X, then Eqs. 3-5 as in
+ * eqat_ste_bwd.  With groups of up to 256 elements Eqs. 3-5 are applied to the
+ * fp32 accumulators of dW_hat inside the same kernel and dW_hat is never
+ * stored; longer groups (channel-wise) keep dW_hat in bf16 in the workspace and
+ * run eqat_ste_bwd on it.  Needs eqat_workspace_bytes(desc,
+ * EQAT_OP_FAKEQUANT_BWD) bytes of scratch in both cases (touched only in the
+ * second).
  *   X [T,in], dY [T,out], W, W_hat [out,in] bf16, s, z (in)
  *   dX [T,in] bf16, dW [out,in] bf16, ds, dz [out,in/g] fp32 (out) */
 int qlinear_fakequant_bwd(const eqat_desc* desc, const eqat_bf16* X, const eqat_bf16* dY, const eqat_bf16* W,
@@ -185,7 +189,9 @@ int eqat_unpack_zeros(const eqat_desc* desc, const uint8_t* z_packed, uint8_t* z
 /* ------------------------------------------------------------------ E2E-QP */
 
 /* Y = X * ((W_int - z) * s)^T, the packed codes expanded tile by tile in
- * shared memory inside the GEMM (Eq. 2; Sec. 3.3).
+ * shared memory inside the GEMM (Eq. 2; Sec. 3.3).  With one to four tokens
+ * (decoding) a matrix-vector kernel streams the packed weight instead and
+ * keeps (W_int - z) * s in fp32.
  *   X [T,in] bf16, Wq_packed, s16, z8 (in)   Y [T,out] bf16 (out) */
 int qlinear_packed_fwd(const eqat_desc* desc, const eqat_bf16* X, const uint8_t* Wq_packed,
                        const eqat_fp16* s16, const uint8_t* z8, eqat_bf16* Y, void* stream);
