@@ -63,7 +63,6 @@ enum Epilogue : int { EPI_STORE = 0, EPI_DS = 1, EPI_STE = 2 };
 struct GemmParams {
   int M, N, K;
   eqat_bf16* D;              // EPI_STORE: [M,N] row-major
-  int wide_store;            // D is 32-byte aligned: rows can be written a sector per lane
   // packed weight (B operand of the packed kernels, epilogue operand of EPI_DS)
   const uint8_t* Wq;         // [out, in*bits/8]
   const eqat_fp16* s16;      // [out, in/group]
@@ -275,6 +274,26 @@ __device__ __forceinline__ void load_codes64(const uint8_t* p, uint32_t (&w)[2 *
   }
 }
 
+// 4 x 4 transpose of 16-byte pieces inside each quad of lanes.  In: o[4p .. 4p+3] = piece p (8 bf16 columns) of the
+// lane's own row.  Out: o[4k .. 4k+3] = piece (lane & 3) of the row owned by lane k of the quad.  Two butterfly
+// rounds; in round b the pieces whose index differs from the lane's in bit b change lane and slot.
+__device__ __forceinline__ void quad_transpose(uint32_t (&o)[16], int lane) {
+#pragma unroll
+  for (int b = 1; b >= 0; --b) {
+    const bool up = (lane >> b) & 1;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int s0 = b == 1 ? j : 2 * j, s1 = s0 + (1 << b);        // slots that differ in bit b only
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const uint32_t send = up ? o[4 * s0 + w] : o[4 * s1 + w];
+        const uint32_t recv = __shfl_xor_sync(0xFFFFFFFFu, send, 1 << b);
+        if (up) o[4 * s0 + w] = recv; else o[4 * s1 + w] = recv;
+      }
+    }
+  }
+}
+
 // A_MN / B_MN: operand is MN-major.  PACKED: B is expanded from N-bit codes.
 // BITS is used by PACKED and by EPI_DS.
 template <int BN, int MT, bool A_MN, bool B_MN, bool PACKED, int EPI, int BITS>
@@ -341,31 +360,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MT + h) * BN);
       const int m = m_blk * C::kTileM + h * BM + row_in_tile;
       if constexpr (EPI == EPI_STORE) {
-        eqat_bf16* drow = p.D + (size_t)m * p.N;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           uint32_t r[32];
           ptx::tmem_ld_32x32(t_row + c * 32, r);
           ptx::tmem_ld_wait();
           const int col0 = n_blk * BN + c * 32;
-          if (m < p.M) {
-            // A lane owns a row, so the lanes of a store instruction hit 32 different lines and the stores,
-            // not the TMEM loads, set the pace of this epilogue: write whole 32-byte sectors where the
-            // output is aligned for it (N is a multiple of 16 for every shape the library accepts).
+          // A lane owns a row, so a plain store instruction would hit 32 different lines, and it is the stores, not
+          // the TMEM loads, that set the pace of this epilogue.  The four lanes of a quad therefore trade 16-byte
+          // pieces so that each store instruction writes 64 contiguous bytes of one row per quad: 8 lines instead
+          // of 32.  (N is a multiple of 16 for every shape the library accepts, so a piece is never ragged.)
+          uint32_t o[16];
 #pragma unroll
-            for (int v = 0; v < 2; ++v) {
-              if (col0 + v * 16 < p.N) {
-                uint32_t o[8];
+          for (int i = 0; i < 16; ++i) o[i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+          quad_transpose(o, lane);
+          const int q = lane & 3;
+          if (col0 + q * 8 < p.N) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                  o[i] = pack_bf16x2(__uint_as_float(r[16 * v + 2 * i]), __uint_as_float(r[16 * v + 2 * i + 1]));
-                if (p.wide_store) {
-                  ptx::stg_256(drow + col0 + v * 16, o);
-                } else {
-                  reinterpret_cast<uint4*>(drow + col0 + v * 16)[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                  reinterpret_cast<uint4*>(drow + col0 + v * 16)[1] = make_uint4(o[4], o[5], o[6], o[7]);
-                }
-              }
+            for (int k = 0; k < 4; ++k) {
+              const int mk = m - q + k;
+              if (mk < p.M)
+                *reinterpret_cast<uint4*>(p.D + (size_t)mk * p.N + col0 + q * 8) =
+                    make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
             }
           }
         }
@@ -821,10 +837,7 @@ GemmParams base_params(int M, int N, int K) {
   return p;
 }
 
-void set_output(GemmParams& p, eqat_bf16* D) {
-  p.D = D;
-  p.wide_store = (reinterpret_cast<uintptr_t>(D) & 31u) == 0 && (p.N & 15) == 0;
-}
+void set_output(GemmParams& p, eqat_bf16* D) { p.D = D; }
 
 void set_weight(GemmParams& p, const eqat_desc& d, const uint8_t* Wq, const eqat_fp16* s16, const uint8_t* z8) {
   p.Wq = Wq; p.s16 = s16; p.z8 = z8;

@@ -256,7 +256,7 @@ def test_block_ap_ragged(eqat, out, in_f, tokens, bits, group):
 
 
 def test_outputs_aligned_to_16_bytes_only(eqat):
-    """Outputs that are 16- but not 32-byte aligned take the narrower store path: same bits."""
+    """Outputs need 16-byte alignment only: the same bits at a 16-byte offset from a 512-byte boundary."""
     cfg = get_config("c1"); lin = cfg.linears[0]
     out, in_f, T = lin.out_features, lin.in_features, cfg.tokens
     s, z = O.minmax_init(f32(weight_for(cfg, lin)), cfg.bits, cfg.group)
