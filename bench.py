@@ -44,10 +44,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # files change the figures are stale and `roofline.traffic` is reported as null.
 NCU_TRAFFIC = {
     "sources": ("gemm.cu", "ptx.cuh"),
-    "sources_sha256": "cf228092eebbfc5e320ed3f8d3cd152718e108f4cbf03b584874890ddd5fbe36",
-    "packed_fwd": {"qkvo": 139.27e6 + 97.46e6, "gate_up": 147.76e6 + 314.98e6, "down": 442.55e6 + 114.84e6},
-    "packed_bwd_dx": {"qkvo": 139.26e6 + 98.08e6, "gate_up": 451.88e6 + 114.70e6, "down": 148.39e6 + 315.95e6},
-    "packed_bwd_ds": {"qkvo": 416.51e6 + 4.73e6, "gate_up": 1306.28e6 + 2.74e6, "down": 1073.37e6 + 3.04e6},
+    "sources_sha256": "4f1b17a7d3d3c5a1612b28492de8c8fbe3d7f2c6a1f74837f8c93d8d050d03df",
+    "packed_fwd": {"qkvo": 139.67e6 + 93.95e6, "gate_up": 147.84e6 + 315.90e6, "down": 438.26e6 + 113.95e6},
+    "packed_bwd_dx": {"qkvo": 139.26e6 + 93.87e6, "gate_up": 443.92e6 + 114.00e6, "down": 148.44e6 + 316.33e6},
+    "packed_bwd_ds": {"qkvo": 416.39e6 + 0.99e6, "gate_up": 1339.70e6 + 3.08e6, "down": 1077.48e6 + 2.81e6},
 }
 
 

@@ -351,9 +351,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const int quad = warp & 3;
   const int row_in_tile = quad * 32 + lane;
   auto epilogue_tile = [&](int m_blk, int n_blk, int acc, uint32_t acc_phase) -> bool {
-    if (!wait_bounded(ptx::smem_addr(&ctl->acc_full[acc]), acc_phase, abort_flag, WAIT_EPI_ACC_FULL,
-                      PACKED ? 0 : (MT == 2 ? 512 : 128)))
-      return false;
+    // The lanes of a warp must leave together: the store epilogue below shuffles across the whole warp.
+    const bool got = wait_bounded(ptx::smem_addr(&ctl->acc_full[acc]), acc_phase, abort_flag, WAIT_EPI_ACC_FULL,
+                                  PACKED ? 0 : (MT == 2 ? 512 : 128));
+    if (!__all_sync(0xFFFFFFFFu, got)) return false;
     ptx::tc_fence_after();
 #pragma unroll 1
     for (int h = 0; h < MT; ++h) {
@@ -739,6 +740,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
         }
         gk += num_kb;
+        ok = __all_sync(0xFFFFFFFFu, ok);                          // a warp gives up as a whole
         if (warp < 2 + kEpiWarps && ok) {
           ok = epilogue_tile(m_blk, n_blk, acc, acc_phase);
           if (++acc == C::kAccSets) { acc = 0; acc_phase ^= 1u; }
