@@ -29,6 +29,19 @@ def test_peaks_have_a_source():
     assert p["hbm_gbs"] > 1000 and p["bf16_tflops_sustained"] > 100
 
 
+def test_traffic_figures_follow_the_kernel_sources(monkeypatch):
+    """The ncu DRAM figures are reported only for the kernel sources they were captured from."""
+    t = bench.traffic_per_launch("packed_fwd")
+    if t is None:
+        pytest.skip("gemm.cu or ptx.cuh changed since the last ncu capture (bench.py then reports traffic: null)")
+    table = bench.NCU_TRAFFIC["packed_fwd"]
+    assert t == pytest.approx((4 * table["qkvo"] + 2 * table["gate_up"] + table["down"]) / 7)
+    assert 0.5 < t / 372.7e6 < 1.5                       # near the algorithmic bytes of a forward launch
+    assert bench.traffic_per_launch("fakequant_fwd") is None
+    monkeypatch.setitem(bench.NCU_TRAFFIC, "sources_sha256", "0" * 64)
+    assert bench.traffic_per_launch("packed_fwd") is None
+
+
 def _rank_main(rank, world, port, q):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
                       LOCAL_RANK=str(rank))
