@@ -697,6 +697,65 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         for (int kb0 = kb_first; kb0 < num_kb && ok; kb0 += 4 * R) {
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
+            if constexpr (R == 2) {
+              // Both K blocks of a run as one straight-line piece of code (their two stages belong to this group and
+              // share a phase): twice the independent work for the scheduler to interleave, one fence and one warp
+              // synchronisation for the two stages.
+              const int kb = kb0 + 4 * j;                           // even; kb + 1 < num_kb since num_kb is even
+              if (ok && kb < num_kb) {
+                if (sz_blocks) {
+                  const int blk = ((kb << 6) >> p.group_shift) >> 2;
+                  if (blk != sz_blk) {
+                    sz_cur = sz_nxt;
+                    sz_blk = blk;
+                    fetch_sz(sz_nxt, blk + 1);
+                  }
+                }
+                const int stage = (int)((gk + kb) & 3);             // 0 or 2; the run's second block is stage + 1
+                const uint32_t phase = (uint32_t)(((gk + kb) >> 2) & 1);
+                if (!wait_bounded(ptx::smem_addr(&ctl->empty_b[stage]), phase ^ 1u, abort_flag,
+                                  WAIT_DEQ_OPERAND_EMPTY) ||
+                    !wait_bounded(ptx::smem_addr(&ctl->empty_b[stage + 1]), phase ^ 1u, abort_flag,
+                                  WAIT_DEQ_OPERAND_EMPTY)) {
+                  ok = false;
+                } else {
+                  const uint32_t row_sx = smem_base + C::b_offset(stage) + smem_row_sx;
+                  if (valid) {
+                    float sv[2], zv[2];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                      sv[u] = ring_s[j][u];
+                      zv[u] = ring_z[j][u];
+                      if (sz_blocks) {
+                        const int sub = (((kb + u) << 6) >> p.group_shift) & 3;
+                        const uint32_t sw = (sub & 2) ? sz_cur.s4.y : sz_cur.s4.x;
+                        sv[u] = __half2float(__ushort_as_half((unsigned short)((sub & 1) ? (sw >> 16) : (sw & 0xFFFFu))));
+                        zv[u] = (float)((sz_cur.z4 >> (8 * sub)) & 0xFFu);
+                      }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                      const uint32_t rs = row_sx + (uint32_t)u * C::kBBytes;
+                      dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][u][0]), sv[u], zv[u], rs, 0);
+                      dequant_half32<BITS>(reinterpret_cast<const uint32_t(&)[BITS]>(ring_w[j][u][BITS]), sv[u], zv[u], rs, 1);
+                    }
+                  } else {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                      ptx::sts_128(row_sx ^ ((uint32_t)c << 4), 0u, 0u, 0u, 0u);
+                      ptx::sts_128((row_sx + C::kBBytes) ^ ((uint32_t)c << 4), 0u, 0u, 0u, 0u);
+                    }
+                  }
+                  if (kb + 8 < num_kb) fetch(j, kb + 8);
+                  ptx::fence_proxy_async_smem();
+                  __syncwarp();
+                  if (lane == 0) {
+                    ptx::mbar_arrive(ptx::smem_addr(&ctl->full_b[stage]));
+                    ptx::mbar_arrive(ptx::smem_addr(&ctl->full_b[stage + 1]));
+                  }
+                }
+              }
+            } else {
 #pragma unroll
             for (int u = 0; u < R; ++u) {
               const int kb = kb0 + 2 * R * j + u;
@@ -736,6 +795,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                   if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full_b[stage]));
                 }
               }
+            }
             }
           }
         }
