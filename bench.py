@@ -44,10 +44,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # files change the figures are stale and `roofline.traffic` is reported as null.
 NCU_TRAFFIC = {
     "sources": ("gemm.cu", "ptx.cuh"),
-    "sources_sha256": "4f1b17a7d3d3c5a1612b28492de8c8fbe3d7f2c6a1f74837f8c93d8d050d03df",
-    "packed_fwd": {"qkvo": 139.67e6 + 93.95e6, "gate_up": 147.84e6 + 315.90e6, "down": 438.26e6 + 113.95e6},
-    "packed_bwd_dx": {"qkvo": 139.26e6 + 93.87e6, "gate_up": 443.92e6 + 114.00e6, "down": 148.44e6 + 316.33e6},
-    "packed_bwd_ds": {"qkvo": 416.39e6 + 0.99e6, "gate_up": 1339.70e6 + 3.08e6, "down": 1077.48e6 + 2.81e6},
+    "sources_sha256": "0533e4c64057d1a8e9b43ad0fe145a1389847317b4c268b65566fcf7937a2101",
+    "packed_fwd": {"qkvo": 139.40e6 + 93.30e6, "gate_up": 148.25e6 + 314.49e6, "down": 446.58e6 + 114.28e6},
+    "packed_bwd_dx": {"qkvo": 139.33e6 + 93.68e6, "gate_up": 447.84e6 + 113.75e6, "down": 147.86e6 + 315.66e6},
+    "packed_bwd_ds": {"qkvo": 416.30e6 + 0.81e6, "gate_up": 1344.16e6 + 3.39e6, "down": 1074.86e6 + 3.15e6},
 }
 
 
