@@ -364,6 +364,8 @@ def test_few_token_forward_agrees_with_tiled_forward(eqat):
     (64, 128, 1, 4, 128),
     (320, 640, 129, 3, 128),
     (1024, 256, 520, 2, 64),
+    (64, 11008, 4, 2, 64),          # few-token kernel with more than 48 KB of staged activations
+    (64, 28672, 2, 4, 128),         # activations too large to stage: two tokens through the tiled kernel
 ])
 def test_e2e_ragged(eqat, out, in_f, tokens, bits, group):
     cfg = small_cfg(f"e2er_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens)
