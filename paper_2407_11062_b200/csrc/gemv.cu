@@ -7,8 +7,8 @@
 // Mapping: a CTA owns 32 consecutive weight rows, lane = row, and its 16 warps
 // split the row into contiguous runs of 64-code units.  All lanes of a warp are
 // on the same columns, so the activations are read from shared memory as
-// broadcasts (one wavefront per 16-byte load) and are staged there once per CTA
-// as fp32, together with their sum over every 64-column unit.
+// broadcasts (one wavefront per 16-byte load); each warp stages the columns of
+// its own units there as fp32, together with their sum over every 64-column unit.
 //
 // Arithmetic: a code q is dropped into the top mantissa bits of the float 1.0,
 // giving 1 + q/2^N with two logic operations and no int-to-float conversion.
@@ -44,7 +44,11 @@ __device__ __forceinline__ float code_as_float(const uint32_t (&w)[2 * BITS], in
   } else {
     t = __funnelshift_r(w[word], w[word + 1], off - pos);      // 3-bit codes that straddle two words
   }
-  return __uint_as_float((t & (((1u << BITS) - 1u) << pos)) | 0x3F800000u);
+  // (t & mask) | 1.0f as one three-input logic operation: both constants are passed in registers, which the
+  // compiler otherwise folds into two instructions with one immediate each.
+  uint32_t r;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(t), "r"(((1u << BITS) - 1u) << pos), "r"(0x3F800000u));
+  return __uint_as_float(r);
 }
 
 template <int BITS>
@@ -75,28 +79,6 @@ packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ 
   float* xsum = xs + (size_t)T * in_features;           // [T][units]
   float* part = xsum + (size_t)T * units;               // [warps][T][32]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  // activations -> fp32 (X is [T,in] row-major, i.e. T*in contiguous elements)
-  for (int i = threadIdx.x; i < T * in_features / 8; i += kThreads) {
-    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(X) + i);
-    const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
-    float4 lo, hi;
-    lo.x = __uint_as_float(r[0] << 16); lo.y = __uint_as_float(r[0] & 0xFFFF0000u);
-    lo.z = __uint_as_float(r[1] << 16); lo.w = __uint_as_float(r[1] & 0xFFFF0000u);
-    hi.x = __uint_as_float(r[2] << 16); hi.y = __uint_as_float(r[2] & 0xFFFF0000u);
-    hi.z = __uint_as_float(r[3] << 16); hi.w = __uint_as_float(r[3] & 0xFFFF0000u);
-    reinterpret_cast<float4*>(xs)[2 * i] = lo;
-    reinterpret_cast<float4*>(xs)[2 * i + 1] = hi;
-  }
-  __syncthreads();
-  // per-unit sums: a warp per (token, unit), two elements per lane, fixed-order tree
-  for (int i = warp; i < T * units; i += kWarps) {
-    float v = xs[(size_t)i * 64 + lane] + xs[(size_t)i * 64 + 32 + lane];
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
-    if (lane == 0) xsum[i] = v;
-  }
-  __syncthreads();
 
   const int row = blockIdx.x * kRows + lane;
   const bool live = row < out_features;
@@ -144,7 +126,36 @@ packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ 
         }
       }
   };
-  fetch(u_begin);
+  fetch(u_begin);                                       // in flight while this warp stages its activations
+
+  // A warp reads only the columns of its own units, so it stages just those (bf16 -> fp32) and their per-unit
+  // sums itself: no CTA-wide barrier before the main loop.
+  {
+    const int nu = u_end - u_begin;
+    for (int i = lane; i < T * nu * 8; i += 32) {       // one 16-byte piece (8 bf16) per iteration
+      const int t = i / (nu * 8), r8 = i - t * (nu * 8);
+      const size_t e0 = (size_t)t * in_features + (size_t)u_begin * 64 + (size_t)r8 * 8;
+      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(X + e0));
+      const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+      float4 lo, hi;
+      lo.x = __uint_as_float(r[0] << 16); lo.y = __uint_as_float(r[0] & 0xFFFF0000u);
+      lo.z = __uint_as_float(r[1] << 16); lo.w = __uint_as_float(r[1] & 0xFFFF0000u);
+      hi.x = __uint_as_float(r[2] << 16); hi.y = __uint_as_float(r[2] & 0xFFFF0000u);
+      hi.z = __uint_as_float(r[3] << 16); hi.w = __uint_as_float(r[3] & 0xFFFF0000u);
+      reinterpret_cast<float4*>(xs + e0)[0] = lo;
+      reinterpret_cast<float4*>(xs + e0)[1] = hi;
+    }
+    __syncwarp();
+    for (int i = 0; i < T * nu; ++i) {                  // two elements per lane, fixed-order tree
+      const int t = i / nu, u = u_begin + (i - t * nu);
+      const float* xu = xs + (size_t)t * in_features + (size_t)u * 64;
+      float v = xu[lane] + xu[32 + lane];
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+      if (lane == 0) xsum[t * units + u] = v;
+    }
+    __syncwarp();
+  }
 #pragma unroll 1
   for (int u0 = u_begin; u0 < u_end; u0 += kBatch) {
     uint32_t w[kBatch][2 * BITS], sz[kBatch];
