@@ -412,7 +412,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           ptx::tmem_ld_32x32(t_row + c * 32, r32);
           ptx::tmem_ld_wait();
           if (live) {
-            const float rs = group_rcp(sv);
+            const float rs = group_rcp(sv, zr);
             const float lo = -zr, hi = p.Q - zr;
 #pragma unroll
             for (int v = 0; v < 4; ++v) {

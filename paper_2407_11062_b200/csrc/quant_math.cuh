@@ -22,12 +22,14 @@ __device__ __forceinline__ uint4 pack8(const float (&v)[8]) {
                     pack_bf16x2(v[6], v[7]));
 }
 
-// 1/s to within 1 ulp (rcp.approx.f32); NaN, which forces the exact path below,
-// when the reciprocal is subnormal or not finite and the error bound would not hold.
-__device__ __forceinline__ float group_rcp(float s) {
+// 1/s to within 1 ulp (rcp.approx.f32); NaN, which forces the exact path below for the whole group, when the
+// reciprocal is subnormal or not finite and the error bound would not hold, or when the rounded zero point zr lies
+// outside [-16, 16] (the shortcut relies on the clamp range [-zr, Q - zr] lying within [-16, 31], see below).
+__device__ __forceinline__ float group_rcp(float s, float zr) {
   float rs;
   asm("rcp.approx.f32 %0, %1;" : "=f"(rs) : "f"(s));
-  return (fabsf(rs) >= 1.17549435e-38f && fabsf(rs) <= 3.402823466e+38f) ? rs : __int_as_float(0x7FC00000);
+  const bool ok = fabsf(rs) >= 1.17549435e-38f && fabsf(rs) <= 3.402823466e+38f && fabsf(zr) <= 16.0f;
+  return ok ? rs : __int_as_float(0x7FC00000);
 }
 
 // Eq. 1 for the eight elements of a vector: r = round(w/s) and the STE term
@@ -43,14 +45,18 @@ __device__ __forceinline__ float group_rcp(float s) {
 //   from rint(rn(w/s)) only if a half-integer lies between the two values; for
 //   |q| <= 32.5 that needs w*rs within 1.5 * 2^-23 * 32.5 < 2^-17 of a half-integer.
 //   d = w*rs - r0 (one more fused multiply-add) is the distance to the integer.
-//   Unless every element of the vector has |d| < 0.5 - 2^-17 and |r0| <= 32,
-//   the whole vector is redone with the exact sequence (about one vector in
-//   eight thousand on in-range weights; always for quotients far out of range).
+//   An element with |d| >= 0.5 - 2^-17 (or NaN) is redone with the exact
+//   sequence: a few elements per thousand on min/max-initialised bf16 weights,
+//   whose quotients are ratios of small integers and hit exact half-integers.
+//   Quotients beyond 32.5 in magnitude need no care: every caller clamps r to
+//   [-zr, Q - zr], which group_rcp keeps inside [-16, 31]; there r >= 33 or
+//   r <= -33, r0 is within 1 of r (or as huge, or as infinite), and both clamp to
+//   the same end.  (r itself is then not the defined value; only its clamp is.)
 // The STE term r - w/s is returned as -d in the common case (2^-23 relative away
 // from the exact one, immaterial for a gradient).
 __device__ __forceinline__ void quotient_round8(const float (&w)[8], float s, float rs, float (&r)[8],
                                                 float (&r_minus_t)[8]) {
-  float dmax = 0.0f, rmax = 0.0f;
+  float dmax = 0.0f;
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const float r0 = fmaf(w[i], rs, 12582912.0f) - 12582912.0f;
@@ -58,14 +64,19 @@ __device__ __forceinline__ void quotient_round8(const float (&w)[8], float s, fl
     r[i] = r0;
     r_minus_t[i] = -d;
     dmax = fmaxf(dmax, fabsf(d));
-    rmax = fmaxf(rmax, fabsf(r0));
   }
-  if (!(dmax < 0.49999237060546875f && rmax <= 32.0f)) {   // also taken when anything is NaN
+  // fmaxf drops NaNs, so a NaN reciprocal (group_rcp's way of asking for the exact path) is tested by itself; a NaN
+  // weight makes r NaN on either path
+  if (!(dmax < 0.49999237060546875f) || rs != rs) {
+    // Some lane of nearly every warp lands here (bf16 weights over a min/max grid hit exact half-integer quotients
+    // in a few elements per thousand), so the whole warp walks this path: redo only the elements that need it.
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const float q = __fdiv_rn(w[i], s);
-      r[i] = rintf(q);
-      r_minus_t[i] = r[i] - q;
+      if (!(fabsf(r_minus_t[i]) < 0.49999237060546875f)) {
+        const float q = __fdiv_rn(w[i], s);
+        r[i] = rintf(q);
+        r_minus_t[i] = r[i] - q;
+      }
     }
   }
 }

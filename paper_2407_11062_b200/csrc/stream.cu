@@ -208,7 +208,7 @@ fakequant_stream_kernel(const eqat_bf16* __restrict__ W, const float* __restrict
       if (v < n_vec) {
         const float sv = gp.s[u];
         const float zr = rintf(gp.z[u]);
-        const float rs = group_rcp(sv);
+        const float rs = group_rcp(sv, zr);
         const float lo = -zr, hi = Q - zr;
         float w[8], r[8], rt[8];
         unpack8(raw[0][u], w);
@@ -246,7 +246,7 @@ ste_bwd_stream_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __re
       const float sv = gp.s[u];
       if (live) {
         const float zr = rintf(gp.z[u]);
-        const float rs = group_rcp(sv);
+        const float rs = group_rcp(sv, zr);
         const float lo = -zr, hi = Q - zr;
         float gr[8], w[8], r[8], rt[8];
         unpack8(raw[0][u], gr);
@@ -357,7 +357,7 @@ quantize_pack_stream_kernel(const eqat_bf16* __restrict__ W, const float* __rest
       if (live) {
         const float sv = gp.s[u];
         const float zr = rintf(gp.z[u]);
-        const float rs = group_rcp(sv);
+        const float rs = group_rcp(sv, zr);
         float w[8], r[8], rt[8];
         unpack8(raw[0][u], w);
         quotient_round8(w, sv, rs, r, rt);

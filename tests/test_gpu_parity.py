@@ -195,6 +195,50 @@ def test_codes_on_exact_and_near_ties(eqat):
     assert np.array_equal(torch_to_f64(dW), dW_o)
 
 
+def test_quotients_far_out_of_range_and_zero_points_off_the_grid(eqat):
+    """Quotients of magnitude 30 .. 1e30 (and infinite), on and next to half-integers, and zero points far
+    outside [0, Q]: the fake-quantised weight and the STE mask must still be the oracle's, element for
+    element.  (With a zero point of +-20 or +-40 the in-range window lies around quotients of that size.)"""
+    bits, group, in_f = 4, 32, 128
+    base = np.float32(0.0234375)
+    hs = np.concatenate([np.arange(-45.0, 45.5, 0.5), [31.5, 32.5, 33.5, -32.5, 1e3 + 0.5, -1e4, 3e7, -2e9, 1e30, -1e30]]
+                        ).astype(np.float32)
+    rows, s_rows, z_rows = [], [], []
+    for ulps in range(-2, 3):
+        sv = base
+        for _ in range(abs(ulps)):
+            sv = np.nextafter(sv, np.float32(np.inf if ulps > 0 else -np.inf), dtype=np.float32)
+        for zz in (0.0, 15.0, 16.0, 17.0, 20.0, -20.0, 40.0, -40.0):
+            for shift in (0, 7, 19):
+                rows.append(np.resize(np.roll(hs, shift) * base, in_f).astype(np.float32))
+                s_rows.append(np.full(in_f // group, sv, np.float32))
+                z_rows.append(np.full(in_f // group, zz, np.float32))
+    for big_s, zz in ((1e38, 0.0), (3e38, 7.0)):                           # 1/s is subnormal: no usable reciprocal
+        rows.append(np.resize(hs[:181] * np.float32(2e36), in_f).astype(np.float32))   # quotients up to +-0.9 / +-0.3
+        s_rows.append(np.full(in_f // group, big_s, np.float32))
+        z_rows.append(np.full(in_f // group, zz, np.float32))
+    while len(rows) % 64:
+        rows.append(rows[0]); s_rows.append(s_rows[0]); z_rows.append(z_rows[0])
+    W32 = np.stack(rows); s = np.stack(s_rows); z = np.stack(z_rows)
+    Wb = to_bf16_bits(W32); W32 = f32(Wb)                                  # whatever bf16 makes of them
+    out = W32.shape[0]
+    d = eqat.make_desc(bits, group, out, in_f)
+    What = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
+    eqat.eqat_fakequant_weight(d, bits_to_torch(Wb), dev(s), dev(z), What)
+    # Eq. 2 on the oracle's codes, the product taken in binary32 as the kernel does: with |q - z| up to 40 the
+    # product is not exact in binary32, and rounding it to bf16 from binary64 instead could differ in the last bit
+    q_o, _, _ = O.quantize_codes(W32, s, z, bits, group)                  # the zero points here are integers
+    What_o = bf16_round(((q_o - np.repeat(z, group, 1)).astype(np.float32) * np.repeat(s, group, 1)).astype(np.float32))
+    bad = np.argwhere(torch_to_f64(What) != What_o.astype(np.float64))
+    assert bad.size == 0, (bad[:5], [(W32[i, j], s[i, j // group], z[i, j // group]) for i, j in bad[:5]])
+    G = np.ones_like(W32); dW = torch.empty_like(What)
+    ds = torch.empty(out, in_f // group, device="cuda")
+    eqat.eqat_ste_bwd(d, bits_to_torch(to_bf16_bits(G)), bits_to_torch(Wb), dev(s), dev(z), dW, ds, None)
+    dW_o, _, _ = O.ste_bwd(G, W32, s, z, bits, group)
+    assert np.array_equal(torch_to_f64(dW), dW_o)
+    assert dW_o.sum() > 1000 and (dW_o == 0).sum() > 1000                  # both branches well populated
+
+
 # --------------------------------------------------------------------------- Block-AP layer
 def run_block_ap(eqat, cfg, lin, tokens, s, z, dz_mode=0):
     Wb = weight_for(cfg, lin); Xb, dYb = activations_for(cfg, lin, tokens)
