@@ -44,10 +44,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # files change the figures are stale and `roofline.traffic` is reported as null.
 NCU_TRAFFIC = {
     "sources": ("gemm.cu", "ptx.cuh"),
-    "sources_sha256": "0533e4c64057d1a8e9b43ad0fe145a1389847317b4c268b65566fcf7937a2101",
-    "packed_fwd": {"qkvo": 139.40e6 + 93.30e6, "gate_up": 148.25e6 + 314.49e6, "down": 446.58e6 + 114.28e6},
-    "packed_bwd_dx": {"qkvo": 139.33e6 + 93.68e6, "gate_up": 447.84e6 + 113.75e6, "down": 147.86e6 + 315.66e6},
-    "packed_bwd_ds": {"qkvo": 416.30e6 + 0.81e6, "gate_up": 1344.16e6 + 3.39e6, "down": 1074.86e6 + 3.15e6},
+    "sources_sha256": "3c1167f2e2956794ea01cf8312af7c9515346679e3a6707d70e99a3cc3cfec0f",
+    "packed_fwd": {"qkvo": 139.26e6 + 93.10e6, "gate_up": 147.72e6 + 314.19e6, "down": 448.65e6 + 114.63e6},
+    "packed_bwd_dx": {"qkvo": 139.26e6 + 93.85e6, "gate_up": 449.56e6 + 114.69e6, "down": 147.73e6 + 315.56e6},
+    "packed_bwd_ds": {"qkvo": 416.23e6 + 0.85e6, "gate_up": 1306.73e6 + 3.00e6, "down": 1073.39e6 + 2.82e6},
 }
 
 
