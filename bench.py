@@ -41,26 +41,33 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) per launch of the packed-weight GEMMs at 16384 tokens, w2g64, by linear shape: ncu
 # `dram__bytes_read.sum + dram__bytes_write.sum`, one capture per shape with `bench.py --kernel-case` (the summaries
 # under profiles/ give the command).  They describe the kernels whose sources hash to `sources_sha256`; once those
-# files change the figures are stale and `roofline.traffic` is reported as null.
+# files change (comments and white space aside) the figures are stale and `roofline.traffic` is reported as null.
 NCU_TRAFFIC = {
     "sources": ("gemm.cu", "ptx.cuh"),
-    "sources_sha256": "3c1167f2e2956794ea01cf8312af7c9515346679e3a6707d70e99a3cc3cfec0f",
+    "sources_sha256": "3b2106bc3b7354efc28822654a030b5243cf54848a42562f6390b2b582091a92",
     "packed_fwd": {"qkvo": 139.26e6 + 93.10e6, "gate_up": 147.72e6 + 314.19e6, "down": 448.65e6 + 114.63e6},
     "packed_bwd_dx": {"qkvo": 139.26e6 + 93.85e6, "gate_up": 449.56e6 + 114.69e6, "down": 147.73e6 + 315.56e6},
     "packed_bwd_ds": {"qkvo": 416.23e6 + 0.85e6, "gate_up": 1306.73e6 + 3.00e6, "down": 1073.39e6 + 2.82e6},
 }
 
 
+def sources_fingerprint():
+    """SHA-256 of the kernel sources with // comments and white space removed: what the compiler sees."""
+    import hashlib
+    import re
+    h = hashlib.sha256()
+    for f in NCU_TRAFFIC["sources"]:
+        with open(os.path.join(ROOT, "paper_2407_11062_b200", "csrc", f), "r") as fh:
+            text = re.sub(r"//[^\n]*", "", fh.read())
+        h.update("".join(text.split()).encode())
+    return h.hexdigest()
+
+
 def traffic_per_launch(kernel_class):
     """Launch-weighted mean of the captured DRAM bytes over the class's launches in one step, or None if the
     kernel sources have changed since the capture."""
-    import hashlib
-    h = hashlib.sha256()
-    for f in NCU_TRAFFIC["sources"]:
-        with open(os.path.join(ROOT, "paper_2407_11062_b200", "csrc", f), "rb") as fh:
-            h.update(fh.read())
     table = NCU_TRAFFIC.get(kernel_class)
-    if table is None or h.hexdigest() != NCU_TRAFFIC["sources_sha256"]:
+    if table is None or sources_fingerprint() != NCU_TRAFFIC["sources_sha256"]:
         return None
     n = sum(l.count for l in LINEARS["7b"])
     return sum(table[l.name] * l.count for l in LINEARS["7b"]) / n

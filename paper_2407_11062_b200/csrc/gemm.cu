@@ -28,10 +28,13 @@
 //               then run the epilogue of the tile (MT = 2: nothing overlaps it
 //               anyway, and the other warps meanwhile pre-expand the next tile's
 //               first stages up to the point where they need these four)
-// The epilogue either stores the tile as bf16 or, for the E2E-QP step-size
+// The epilogue either stores the tile as bf16; or, for the E2E-QP step-size
 // gradient, multiplies each accumulator row by (q - z) of the matching packed
 // codes and reduces runs of `group` columns, so the [out,in] weight gradient
-// never leaves the chip.
+// never leaves the chip; or, for the Block-AP weight gradient, applies Eqs. 3-5
+// to the accumulators next to the latent weights and writes dW, ds and dz.
+// Packed kernels walk their tiles row by row (the few MB of codes stay in L2,
+// each activation panel is fetched once); dense kernels in bands of 16 row-tiles.
 //
 // Every wait on an mbarrier is bounded in time; a role that gives up raises a
 // CTA-wide abort flag, records the site in a device status word and all roles

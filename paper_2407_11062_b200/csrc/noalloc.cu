@@ -1,8 +1,10 @@
 // Block-AP backward for callers that must not allocate device memory.
 //
 // qlinear_fakequant_bwd needs out*in bf16 values of scratch for the weight
-// gradient between its GEMM and its STE kernel, and normally the caller
-// allocates that.  Some callers cannot: code that runs after another framework
+// gradient between its GEMM and its STE kernel when a quantisation group is
+// longer than 256 elements (channel-wise quantisation; shorter groups are
+// reduced inside the GEMM and leave the scratch untouched), and normally the
+// caller allocates that.  Some callers cannot: code that runs after another framework
 // has claimed the whole device for its own pool, or inside a section where the
 // implicit device-wide synchronisation that cudaMalloc / cudaFree may perform is
 // not acceptable.  For them this file keeps the scratch in a fixed array that is
