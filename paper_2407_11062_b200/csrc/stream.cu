@@ -361,10 +361,17 @@ quantize_pack_stream_kernel(const eqat_bf16* __restrict__ W, const float* __rest
         float w[8], r[8], rt[8];
         unpack8(raw[0][u], w);
         quotient_round8(w, sv, rs, r, rt);
+        // The piece is sum_i code_i * 2^(BITS*i) with code_i = clamp(r_i + zr, 0, Q): evaluated by Horner's rule on the
+        // integer-valued floats (exact: below 2^24), with one conversion per 16 or 24 bits instead of an add, a mask,
+        // a shift and an or per code.
+        constexpr float kRadix = (float)(1 << BITS);
+        constexpr int kHalf = BITS == 4 ? 4 : 8;                                 // codes per conversion
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float q = fminf(fmaxf(r[i] + zr, 0.0f), Q);
-          piece |= (__float_as_uint(q + 8388608.0f) & 0xFFu) << (BITS * i);     // integer-valued float -> integer
+        for (int h = 0; h < 8 / kHalf; ++h) {
+          float acc = fminf(fmaxf(r[h * kHalf + kHalf - 1] + zr, 0.0f), Q);
+#pragma unroll
+          for (int i = kHalf - 2; i >= 0; --i) acc = fmaf(acc, kRadix, fminf(fmaxf(r[h * kHalf + i] + zr, 0.0f), Q));
+          piece |= __float2uint_rn(acc) << (h * BITS * kHalf);
         }
         if ((v & (((size_t)1 << vec_shift) - 1)) == 0) {
           const size_t g = v >> vec_shift;
