@@ -8,6 +8,7 @@ compared on a seeded sample it can compute directly:
   * codes, packed bytes, zero points and step sizes bit-exactly on those rows,
 and whole-tensor identities that hold at any size tie the rest together:
   <dY, Y> = <dX, X>  (adjoint),  sum s*ds = <dY, Y>  (Y is linear in s).
+The E2E-QP cases also push the first one and four tokens through the forward alone (decoding).
 """
 import numpy as np
 import pytest
@@ -149,5 +150,14 @@ def test_full_size(eqat, cfg_name, lin_name, mode):
         assert abs(a - b) <= tol_abs
         euler = float((s16.double() * ds.double()).sum())
         assert abs(euler - a) <= tol_abs
+        # decoding: the first one and four tokens alone (the matrix-vector kernel where its activations fit in shared
+        # memory, the tiled kernel otherwise), against the oracle and against the same rows of the full batch
+        for t_few in (1, 4):
+            d_few = eqat.make_desc(bits, g, out, in_f, t_few)
+            Y_few = torch.empty(t_few, out, dtype=torch.bfloat16, device="cuda")
+            eqat.qlinear_packed_fwd(d_few, Xd[:t_few].contiguous(), P, s16, z8, Y_few)
+            torch.cuda.synchronize()
+            assert rel_err(torch_to_f64(Y_few[:, rows_y]), O.linear_fwd(f32(Xb[:t_few]), What_rows[iy])) <= TOL
+            assert rel_err(torch_to_f64(Y_few), torch_to_f64(Y[:t_few])) <= TOL
     torch.cuda.synchronize()
     assert eqat.device_status() == (0, 0)
