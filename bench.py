@@ -449,6 +449,25 @@ def run_ours(args):
                                               + l.in_features * l.out_features * BITS // 8) * l.count
                                              for l in LINEARS["7b"]) / sum(l.count for l in LINEARS["7b"])}
         classes = {c: {"total_ms_per_step": t / args.steps, "share": t / sum(by_class.values())} for c, t in by_class.items()}
+        # every class that is exactly one kernel launch per call also gets its own roofline figure:
+        # the contractions against the sustained bf16 peak, the streaming kernels against the copy bandwidth
+        n_elem = sum(l.in_features * l.out_features * l.count for l in LINEARS["7b"])
+        n_grp = n_elem / GROUP
+        hbm_bytes = {"minmax_init": 2 * n_elem + 8 * n_grp,
+                     "quantize_pack": (2 + BITS / 8) * n_elem + 11 * n_grp,
+                     "unpack": (1 + BITS / 8) * n_elem}
+        e2e_flops = sum(2 * T_E2E * l.in_features * l.out_features * l.count for l in LINEARS["7b"])
+        for c, t in by_class.items():
+            sec = t * 1e-3 / args.steps
+            if c in hbm_bytes:
+                ach = hbm_bytes[c] / sec / 1e9
+                classes[c]["roofline"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                          "frac": ach / peaks["hbm_gbs"]}
+            elif c in t_tok:
+                ach = e2e_flops / sec / 1e12
+                classes[c]["roofline"] = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
+                                          "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
+                                          "traffic": traffic_per_launch(c)}
         out = {"metric": "QLinear fwd+bwd TFLOP/s", "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": world,
                "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
