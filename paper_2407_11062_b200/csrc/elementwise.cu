@@ -243,7 +243,9 @@ pack_kernel(const uint8_t* __restrict__ codes8, uint8_t* __restrict__ packed, si
   store_words<BITS>(packed, c, words);
 }
 
-template <int BITS>
+// WIDE: the output is 32-byte aligned, so a thread's 32 codes go out as one store (a whole sector per lane,
+// 1 KB contiguous per warp); otherwise as two 16-byte stores.
+template <int BITS, bool WIDE>
 __global__ void __launch_bounds__(kThreads)
 unpack_kernel(const uint8_t* __restrict__ packed, uint8_t* __restrict__ codes8, size_t n_chunk) {
   const size_t c = (size_t)blockIdx.x * kThreads + threadIdx.x;
@@ -252,15 +254,19 @@ unpack_kernel(const uint8_t* __restrict__ packed, uint8_t* __restrict__ codes8, 
   load_words<BITS>(packed, c, words);
   uint32_t codes[32];
   unpack32<BITS>(words, codes);
+  uint32_t w[8];
 #pragma unroll
-  for (int k = 0; k < 2; ++k) {
-    uint32_t w[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int j = 16 * k + 4 * i;
-      w[i] = codes[j] | (codes[j + 1] << 8) | (codes[j + 2] << 16) | (codes[j + 3] << 24);
-    }
-    reinterpret_cast<uint4*>(codes8)[c * 2 + k] = make_uint4(w[0], w[1], w[2], w[3]);
+  for (int i = 0; i < 8; ++i) {
+    const int j = 4 * i;
+    w[i] = codes[j] | (codes[j + 1] << 8) | (codes[j + 2] << 16) | (codes[j + 3] << 24);
+  }
+  if constexpr (WIDE) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(codes8 + c * 32), "r"(w[0]), "r"(w[1]),
+                 "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+  } else {
+    reinterpret_cast<uint4*>(codes8)[c * 2] = make_uint4(w[0], w[1], w[2], w[3]);
+    reinterpret_cast<uint4*>(codes8)[c * 2 + 1] = make_uint4(w[4], w[5], w[6], w[7]);
   }
 }
 
@@ -344,10 +350,14 @@ int launch_pack(const eqat_desc& d, const uint8_t* codes, uint8_t* packed, cudaS
 int launch_unpack(const eqat_desc& d, const uint8_t* packed, uint8_t* codes, cudaStream_t st) {
   const size_t n_chunk = (size_t)d.out_features * d.in_features / 32;
   const unsigned nb = blocks_for(n_chunk, kThreads);
-  switch (d.bits) {
-    case 2: unpack_kernel<2><<<nb, kThreads, 0, st>>>(packed, codes, n_chunk); break;
-    case 3: unpack_kernel<3><<<nb, kThreads, 0, st>>>(packed, codes, n_chunk); break;
-    default: unpack_kernel<4><<<nb, kThreads, 0, st>>>(packed, codes, n_chunk); break;
+  const bool wide = (reinterpret_cast<uintptr_t>(codes) & 31u) == 0;
+  switch (d.bits * 2 + (wide ? 1 : 0)) {
+    case 4: unpack_kernel<2, false><<<nb, kThreads, 0, st>>>(packed, codes, n_chunk); break;
+    case 5: unpack_kernel<2, true><<<nb, kThreads, 0, st>>>(packed, codes, n_chunk); break;
+    case 6: unpack_kernel<3, false><<<nb, kThreads, 0, st>>>(packed, codes, n_chunk); break;
+    case 7: unpack_kernel<3, true><<<nb, kThreads, 0, st>>>(packed, codes, n_chunk); break;
+    case 8: unpack_kernel<4, false><<<nb, kThreads, 0, st>>>(packed, codes, n_chunk); break;
+    default: unpack_kernel<4, true><<<nb, kThreads, 0, st>>>(packed, codes, n_chunk); break;
   }
   return launch_status();
 }

@@ -135,6 +135,22 @@ def test_zero_point_stream(eqat, bits):
     assert np.array_equal(back.cpu().numpy(), z)
 
 
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_unpack_into_a_buffer_aligned_to_16_bytes_only(eqat, bits):
+    out, in_f, group = 64, 256, 64
+    rng = np.random.default_rng(bits)
+    q = rng.integers(0, 1 << bits, size=(out, in_f), dtype=np.uint8)
+    P = dev(O.pack_rows(q, bits))
+    d = eqat.make_desc(bits, group, out, in_f)
+    for shift in (0, 16):
+        buf = torch.zeros(out * in_f + 32, dtype=torch.uint8, device="cuda")
+        codes = buf[shift:shift + out * in_f].view(out, in_f)
+        assert codes.data_ptr() % 32 == shift
+        eqat.eqat_unpack(d, P, codes)
+        assert np.array_equal(codes.cpu().numpy(), q)
+        assert not buf[:shift].any() and not buf[shift + out * in_f:].any()
+
+
 def test_fractional_zero_point_is_rounded(eqat):
     out, in_f, bits, group = 64, 128, 2, 64
     cfg = small_cfg("fracz", out, in_f, bits, group, 0)
