@@ -21,7 +21,8 @@
  *   - Every tensor pointer is a DEVICE pointer owned by the caller unless its
  *     name starts with `h_` (host).  The library allocates no memory and keeps
  *     no pointer after a call returns.  Device base pointers must be 16-byte
- *     aligned.
+ *     aligned; nothing more is required (where a kernel has a faster path for
+ *     32-byte aligned data it picks it from the pointer).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls enqueue work on `stream` and return without waiting for it.
  *   - Return value: EQAT_OK, or a negative eqat_status decided on the host
@@ -92,6 +93,16 @@ size_t eqat_workspace_bytes(const eqat_desc* desc, int op);
  * NULL) a code naming the wait that was abandoned. */
 int eqat_device_status(int* h_status, int* h_detail);
 
+/* Diagnostic of the bounded waits (no counterpart in the paper).  Every wait of
+ * a kernel on a barrier has a time limit, after which the kernel records
+ * EQAT_ERR_TIMEOUT in the device status word, abandons its work and returns
+ * normally.  This call enqueues one warp that waits, with a limit of 1 ms, on a
+ * barrier that nothing ever signals, through the very wait routine of the GEMM
+ * kernels (which = 0) or of the streaming kernels (which = 1); afterwards
+ * eqat_device_status() must report EQAT_ERR_TIMEOUT once and EQAT_OK from then
+ * on.  It touches no tensor. */
+int eqat_selftest_wait_expiry(int which, void* stream);
+
 /* ------------------------------------------------------------------ helpers */
 
 /* Round-to-nearest initialisation of the quantisation parameters from each
@@ -130,8 +141,8 @@ int eqat_ste_bwd(const eqat_desc* desc, const eqat_bf16* dW_hat, const eqat_bf16
  * fp32 accumulators of dW_hat inside the same kernel and dW_hat is never
  * stored; longer groups (channel-wise) keep dW_hat in bf16 in the workspace and
  * run eqat_ste_bwd on it.  Needs eqat_workspace_bytes(desc,
- * EQAT_OP_FAKEQUANT_BWD) bytes of scratch in both cases (touched only in the
- * second).
+ * EQAT_OP_FAKEQUANT_BWD) bytes of scratch: 0 for groups of up to 256 elements
+ * (workspace may then be NULL), out*in*2 bytes for longer ones.
  *   X [T,in], dY [T,out], W, W_hat [out,in] bf16, s, z (in)
  *   dX [T,in] bf16, dW [out,in] bf16, ds, dz [out,in/g] fp32 (out) */
 int qlinear_fakequant_bwd(const eqat_desc* desc, const eqat_bf16* X, const eqat_bf16* dY, const eqat_bf16* W,
@@ -150,8 +161,12 @@ int qlinear_fakequant_bwd(const eqat_desc* desc, const eqat_bf16* X, const eqat_
  *     (8 MiB of bf16); larger problems return EQAT_ERR_WORKSPACE and launch
  *     nothing.  Every GPU that loads the library holds those 8 MiB until exit;
  *   - the first call on each device looks the array's address up (a runtime
- *     call that is not stream work): make that first call before any stream
- *     capture begins on that device;
+ *     call that is not stream work).  With CUDA's lazy module loading that
+ *     look-up is also the moment the device actually sets the 8 MiB aside, so
+ *     make that first call (any small valid problem will do) early: before
+ *     another framework claims the rest of the device's memory, and before any
+ *     stream capture begins on that device.  EQAT_ERR_CUDA from a first call
+ *     means the array could not be reserved;
  *   - all calls on a device share the one array.  Its previous contents do not
  *     matter (every value read is written earlier in the same call), but two
  *     calls whose kernels overlap on the GPU (different streams) race on it:

@@ -24,7 +24,8 @@ the in-range branch, idempotence and grid membership of the quantiser, textbook
 triple-loop matmuls and adjoint identities for the three contractions,
 brute-force group sums and exact finite differences for the E2E-QP step-size
 gradient, exhaustive round trips, hand-evaluated byte patterns and the paper's
-bits-per-parameter table for the codec.
+bits-per-parameter table for the codec, hand-derived FP16 bit patterns and
+clamped N-bit zero points for the side outputs of the hand-off.
 
 Parity unpinned by the paper (conventions of this library, each exercised by a
 test but fixed by no printed value): the bit layout of the packed stream, the

@@ -44,6 +44,7 @@ def _load():
         "eqat_version": (c_int, []),
         "eqat_workspace_bytes": (c_size_t, [D, c_int]),
         "eqat_device_status": (c_int, [POINTER(c_int), POINTER(c_int)]),
+        "eqat_selftest_wait_expiry": (c_int, [c_int, P]),
         "eqat_minmax_init": (c_int, [D, P, P, P, P]),
         "eqat_fakequant_weight": (c_int, [D, P, P, P, P, P]),
         "qlinear_fakequant_fwd": (c_int, [D, P, P, P, P, P, P, P]),
@@ -105,6 +106,10 @@ def device_status():
     st, det = c_int(0), c_int(0)
     _check(lib.eqat_device_status(ctypes.byref(st), ctypes.byref(det)), "eqat_device_status")
     return st.value, det.value
+
+
+def eqat_selftest_wait_expiry(which):
+    _check(lib.eqat_selftest_wait_expiry(int(which), _stream()), "eqat_selftest_wait_expiry")
 
 
 def eqat_minmax_init(desc, W, s, z):

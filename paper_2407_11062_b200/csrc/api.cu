@@ -10,6 +10,8 @@ namespace {
 
 using namespace eqat;
 
+constexpr int kMaxFusedSteGroup = 256;   // longest group the weight-gradient epilogue reduces by itself
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 
@@ -78,6 +80,8 @@ int eqat_version(void) { return 100; }
 size_t eqat_workspace_bytes(const eqat_desc* d, int op) {
   if (op == EQAT_OP_FAKEQUANT_BWD) {
     if (check_gemm_desc(d, false) != EQAT_OK) return (size_t)-1;
+    // groups that fit an output tile are reduced inside the weight-gradient GEMM: nothing to store
+    if (d->group <= kMaxFusedSteGroup) return 0;
     return (size_t)d->out_features * d->in_features * sizeof(eqat_bf16);   // dW_hat in bf16
   }
   if (op == EQAT_OP_PACKED_BWD_DS) {
@@ -96,6 +100,12 @@ int eqat_device_status(int* h_status, int* h_detail) {
   *h_status = st[k];
   if (h_detail != nullptr) *h_detail = det[k];
   return EQAT_OK;
+}
+
+int eqat_selftest_wait_expiry(int which, void* stream) {
+  if (which == 0) return launch_wait_expiry_gemm(as_stream(stream));
+  if (which == 1) return launch_wait_expiry_stream(as_stream(stream));
+  return EQAT_ERR_UNSUPPORTED;
 }
 
 int eqat_minmax_init(const eqat_desc* d, const eqat_bf16* W, float* s, float* z, void* stream) {
@@ -133,15 +143,19 @@ int qlinear_fakequant_bwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf1
   EQAT_TRY(check_gemm_desc(d, false));
   EQAT_TRY(check_ptrs(X, dY, W, s, z, W_hat, dX, dW, ds));
   if (dz != nullptr && !aligned16(dz)) return EQAT_ERR_ALIGN;
-  const size_t need = (size_t)d->out_features * d->in_features * sizeof(eqat_bf16);
-  if (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
-    return EQAT_ERR_WORKSPACE;
+  // A group that fits inside one output tile is reduced in the weight-gradient GEMM's epilogue and needs no
+  // scratch; a longer one (channel-wise quantisation) spans tiles, so its gradient goes through the workspace
+  // and a second kernel.
+  const bool fused = d->group <= kMaxFusedSteGroup;
+  if (!fused) {
+    const size_t need = (size_t)d->out_features * d->in_features * sizeof(eqat_bf16);
+    if (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+      return EQAT_ERR_WORKSPACE;
+  }
   eqat_bf16* dW_hat = static_cast<eqat_bf16*>(workspace);
   cudaStream_t st = as_stream(stream);
   EQAT_TRY(launch_dense_dx(*d, dY, W_hat, dX, st));
-  // A group that fits inside one output tile is reduced in the weight-gradient GEMM's epilogue; a longer one
-  // (channel-wise quantisation) spans tiles, so its gradient goes through the workspace and a second kernel.
-  if (d->group <= 256) return launch_dense_dw_ste(*d, dY, X, W, s, z, dW, ds, dz, st);
+  if (fused) return launch_dense_dw_ste(*d, dY, X, W, s, z, dW, ds, dz, st);
   EQAT_TRY(launch_dense_dw(*d, dY, X, dW_hat, st));
   return launch_ste_bwd(*d, dW_hat, W, s, z, dW, ds, dz, st);
 }

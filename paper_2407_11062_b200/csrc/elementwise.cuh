@@ -22,6 +22,8 @@ int launch_ste_bwd_stream(const eqat_desc& d, const eqat_bf16* dWhat, const eqat
 int launch_minmax_stream(const eqat_desc& d, const eqat_bf16* W, float* s, float* z, cudaStream_t st);
 int launch_quantize_pack_stream(const eqat_desc& d, const eqat_bf16* W, const float* s, const float* z,
                                 uint8_t* packed, uint8_t* z8, eqat_fp16* s16, cudaStream_t st);
+// Self-test of the streaming kernels' bounded wait (one warp, 1 ms, a barrier nothing signals).
+int launch_wait_expiry_stream(cudaStream_t st);
 // Reads and clears the streaming kernels' status word ({status, wait site}); synchronises.
 int read_stream_status(int* status, int* detail);
 }  // namespace eqat

@@ -72,6 +72,7 @@ struct GemmParams {
   const uint8_t* z8;         // [out, in/group]
   int out_features, in_features;
   int group_shift;           // log2(group)
+  int wq_sectors;            // Wq is 32-byte aligned: a thread may fetch a whole 32-byte sector with one load
   float* ds;                 // EPI_DS / EPI_STE outputs [out, in/group]
   float* dz;                 // may be null
   // EPI_STE: latent weight and Block-AP quantiser parameters of the [out,in] tile rows
@@ -666,7 +667,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         auto fetch = [&](int j, int kb) {                         // kb: first K block of the run being fetched
           if (valid) {
             if constexpr (R == 2) {
-              ptx::ldg_256(code_ptr, reinterpret_cast<uint32_t(&)[8]>(ring_w[j][0][0]));
+              // the run's 32 bytes are one sector of the packed row when the matrix itself starts on a 32-byte
+              // boundary (row pitch and unit offsets are multiples of 32); otherwise two 16-byte loads
+              if (p.wq_sectors) {
+                ptx::ldg_256(code_ptr, reinterpret_cast<uint32_t(&)[8]>(ring_w[j][0][0]));
+              } else {
+                load_codes64<BITS>(code_ptr, ring_w[j][0]);
+                load_codes64<BITS>(code_ptr + 8 * BITS, ring_w[j][1]);
+              }
             } else {
               load_codes64<BITS>(code_ptr, ring_w[j][0]);
             }
@@ -821,6 +829,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   }
 }
 
+// One warp waits, with a short limit, on an mbarrier that nothing ever arrives at: the give-up path of
+// wait_bounded (abort flag, status word, normal return) without any copy or tensor-memory state around it.
+__global__ void wait_expiry_kernel(uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_word;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_addr(&bar), 1);
+    abort_word = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  (void)wait_bounded(ptx::smem_addr(&bar), 0u, &abort_word, WAIT_SELFTEST, 0, limit_ns);
+}
+
 // ------------------------------------------------------------------ host side
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -851,22 +873,12 @@ bool make_tmap(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-  static int n = [] {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    return v;
-  }();
-  return n;
-}
-
 template <int BN, int MT, bool A_MN, bool B_MN, bool PACKED, int EPI, int BITS>
 int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cudaStream_t st) {
   using C = Cfg<BN, MT, PACKED>;
   auto kern = gemm_kernel<BN, MT, A_MN, B_MN, PACKED, EPI, BITS>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-    return EQAT_ERR_CUDA;
+  static SmemOptIn opt_in;
+  if (!opt_in.ensure(kern, C::kSmemBytes)) return EQAT_ERR_CUDA;
   const int sms = sm_count();
   if (sms <= 0) return EQAT_ERR_CUDA;
   const int tiles = ((p.M + C::kTileM - 1) / C::kTileM) * ((p.N + BN - 1) / BN);
@@ -909,6 +921,7 @@ void set_weight(GemmParams& p, const eqat_desc& d, const uint8_t* Wq, const eqat
   p.out_features = d.out_features;
   p.in_features = d.in_features;
   p.group_shift = log2_exact(d.group);
+  p.wq_sectors = (reinterpret_cast<uintptr_t>(Wq) & 31u) == 0 ? 1 : 0;
 }
 
 }  // namespace
@@ -1007,6 +1020,11 @@ int launch_packed_ds(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* dY
     default: return mt == 2 ? launch<256, 2, true, true, false, EPI_DS, 4>(ta, tb, p, st)
                             : launch<256, 1, true, true, false, EPI_DS, 4>(ta, tb, p, st);
   }
+}
+
+int launch_wait_expiry_gemm(cudaStream_t st) {
+  wait_expiry_kernel<<<1, 32, 0, st>>>(1000000ull);   // 1 ms
+  return launch_status();
 }
 
 int read_device_status(int* status, int* detail) {

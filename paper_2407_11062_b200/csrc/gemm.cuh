@@ -24,6 +24,10 @@ int launch_packed_dx(const eqat_desc& d, const eqat_bf16* dY, const uint8_t* Wq,
 int launch_packed_ds(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* dY, const uint8_t* Wq,
                      const uint8_t* z8, const eqat_fp16* s16, float* ds, float* dz, cudaStream_t st);
 
+// Self-test of the bounded wait: one warp waits 1 ms for a barrier that is never signalled, records
+// EQAT_ERR_TIMEOUT / WAIT_SELFTEST in the status word and returns.
+int launch_wait_expiry_gemm(cudaStream_t st);
+
 // Reads and clears the device status word ({status, wait site}); synchronises.
 int read_device_status(int* status, int* detail);
 

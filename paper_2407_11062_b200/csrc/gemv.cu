@@ -15,8 +15,6 @@
 // For a unit with step size s and zero point z
 //     sum_j (q_j - z) s x_j = s (2^N * sum_j (1 + q_j/2^N) x_j - (2^N + z) * sum_j x_j),
 // all in fp32, so the dequantised weight is never rounded to bf16 here.
-#include <atomic>
-
 #include "common.cuh"
 #include "gemv.cuh"
 #include "ptx.cuh"
@@ -72,7 +70,7 @@ template <int BITS, int T>
 __global__ void __launch_bounds__(kThreads)
 packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ Wq, const eqat_fp16* __restrict__ s16,
                    const uint8_t* __restrict__ z8, eqat_bf16* __restrict__ Y, int out_features, int in_features,
-                   int group_shift) {
+                   int group_shift, int sectors) {
   extern __shared__ __align__(16) float smem_f[];
   const int units = in_features >> 6;
   float* xs = smem_f;                                   // [T][in]
@@ -106,14 +104,24 @@ packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ 
     for (int k = 0; k < kBatch; k += 2)
       if (u0 + k < u_end) {
         const uint8_t* src = wrow + (size_t)(u0 + k) * (8 * BITS);
-        if constexpr (BITS == 2) {                      // both units: one 32-byte sector
-          ptx::ldg_256(src, reinterpret_cast<uint32_t(&)[8]>(w_nxt[k][0]));
+        // `sectors`: the packed matrix starts on a 32-byte boundary, so every pair of units does too and is
+        // fetched as whole 32-byte sectors; otherwise with 16-byte (3-bit: 8-byte) loads
+        bool fetched = false;
+        if constexpr (BITS == 2) {
+          if (sectors) {                                // both units: one 32-byte sector
+            ptx::ldg_256(src, reinterpret_cast<uint32_t(&)[8]>(w_nxt[k][0]));
+            fetched = true;
+          }
         } else if constexpr (BITS == 4) {
-          ptx::ldg_256(src, w_nxt[k]);
-          ptx::ldg_256(src + 32, w_nxt[k + 1]);
-        } else {
+          if (sectors) {
+            ptx::ldg_256(src, w_nxt[k]);
+            ptx::ldg_256(src + 32, w_nxt[k + 1]);
+            fetched = true;
+          }
+        }
+        if (!fetched) {
           load_unit<BITS>(src, w_nxt[k]);
-          load_unit<BITS>(src + 24, w_nxt[k + 1]);
+          load_unit<BITS>(src + 8 * BITS, w_nxt[k + 1]);
         }
         const int g = ((u0 + k) << 6) >> group_shift;
         if (group_shift == 6) {
@@ -228,19 +236,12 @@ int launch_one(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const 
   auto kern = packed_gemv_kernel<BITS, T>;
   const size_t smem = smem_floats(T, d.in_features) * sizeof(float);
   if (smem > 48 * 1024) {
-    // raise the kernel's shared-memory limit once per device (the attribute belongs to the device's context)
-    static std::atomic<uint64_t> configured{0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return EQAT_ERR_CUDA;
-    const uint64_t bit = 1ull << (dev & 63);
-    if (dev >= 64 || !(configured.load(std::memory_order_acquire) & bit)) {
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess)
-        return EQAT_ERR_CUDA;
-      if (dev < 64) configured.fetch_or(bit, std::memory_order_release);
-    }
+    static SmemOptIn opt_in;        // raise the kernel's shared-memory limit once per device
+    if (!opt_in.ensure(kern, (int)kMaxSmem)) return EQAT_ERR_CUDA;
   }
   const int grid = (d.out_features + kRows - 1) / kRows;
-  kern<<<grid, kThreads, smem, st>>>(X, Wq, s16, z8, Y, d.out_features, d.in_features, group_shift);
+  const int sectors = (reinterpret_cast<uintptr_t>(Wq) & 31u) == 0 ? 1 : 0;
+  kern<<<grid, kThreads, smem, st>>>(X, Wq, s16, z8, Y, d.out_features, d.in_features, group_shift, sectors);
   return launch_status();
 }
 

@@ -52,7 +52,7 @@ struct RingCtl {
 static_assert(sizeof(RingCtl) <= 256, "ring control block must fit its reservation");
 
 __device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity, volatile int* abort, int site,
-                                          uint32_t sleep_ns) {
+                                          uint32_t sleep_ns, uint64_t limit_ns = kStreamWaitLimitNs) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = ptx::globaltimer_ns();
   uint32_t n = 0;
@@ -60,7 +60,7 @@ __device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity, volatil
     if (sleep_ns != 0) __nanosleep(sleep_ns);
     if ((++n & 31u) == 0u) {
       if (*abort) return false;
-      if (ptx::globaltimer_ns() - t0 > kStreamWaitLimitNs) {
+      if (ptx::globaltimer_ns() - t0 > limit_ns) {
         *abort = 1;
         atomicExch(&g_stream_status[1], site);
         atomicExch(&g_stream_status[0], (int)EQAT_ERR_TIMEOUT);
@@ -113,7 +113,7 @@ __device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], 
       size_t issued = 0;
       bool ok = true;
       for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
-        if (!ring_wait(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_PRODUCER_EMPTY, 32)) {
+        if (!ring_wait(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_STREAM_EMPTY, 32)) {
           ok = false;
           break;
         }
@@ -151,7 +151,9 @@ __device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], 
     for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
       const Params cur = next;
       if (chunk + gridDim.x < n_chunks) next = fetch((chunk + gridDim.x) * kChunkVec + threadIdx.x);
-      if (!ring_wait(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_MMA_FULL, 0)) break;
+      // the lanes of a warp leave together: the bodies shuffle across the whole warp
+      const bool got = ring_wait(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_STREAM_FULL, 0);
+      if (!__all_sync(0xFFFFFFFFu, got)) break;
       uint4 raw[NIN][VPT];
       const uint8_t* st = smem + stage * R::kStageBytes;
 #pragma unroll
@@ -400,28 +402,41 @@ quantize_pack_stream_kernel(const eqat_bf16* __restrict__ W, const float* __rest
   });
 }
 
-// Persistent grid: every CTA resident at once, never more CTAs than chunks.
-template <typename K>
-unsigned stream_grid(K kernel, int smem_bytes, size_t n_vec, int chunk_vec) {
-  int dev = 0, sms = 0, per_sm = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreadsS, smem_bytes) != cudaSuccess ||
-      sms <= 0 || per_sm <= 0) {
-    (void)cudaGetLastError();
-    return 0;
+// The give-up path of ring_wait alone: one warp, a barrier nothing signals, a short limit.
+__global__ void ring_wait_expiry_kernel(uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_word;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_addr(&bar), 1);
+    abort_word = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  (void)ring_wait(ptx::smem_addr(&bar), 0u, &abort_word, WAIT_SELFTEST, 0, limit_ns);
+}
+
+// Persistent grid: every CTA resident at once, never more CTAs than chunks.  The kernel is a template
+// argument so that each kernel has its own per-device state: the shared-memory opt-in and the number of
+// CTAs that fit on an SM (both asked of the runtime once per device).
+template <auto kernel, typename... Args>
+int launch_stream(int smem_bytes, int chunk_vec, size_t n_vec, cudaStream_t st, Args... args) {
+  static SmemOptIn opt_in;
+  static std::atomic<int> ctas_per_sm[kMaxCachedDevices];
+  if (!opt_in.ensure(kernel, smem_bytes)) return EQAT_ERR_CUDA;
+  const int dev = current_device(), sms = sm_count();
+  if (dev < 0 || sms <= 0) return EQAT_ERR_CUDA;
+  int per_sm = dev < kMaxCachedDevices ? ctas_per_sm[dev].load(std::memory_order_relaxed) : 0;
+  if (per_sm <= 0) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreadsS, smem_bytes) != cudaSuccess ||
+        per_sm <= 0) {
+      (void)cudaGetLastError();
+      return EQAT_ERR_CUDA;
+    }
+    if (dev < kMaxCachedDevices) ctas_per_sm[dev].store(per_sm, std::memory_order_relaxed);
   }
   const size_t chunks = (n_vec + chunk_vec - 1) / chunk_vec;
   const size_t resident = (size_t)sms * per_sm;
-  return (unsigned)(chunks < resident ? chunks : resident);
-}
-
-template <typename K, typename... Args>
-int launch_stream(K kernel, int smem_bytes, int chunk_vec, size_t n_vec, cudaStream_t st, Args... args) {
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
-    return EQAT_ERR_CUDA;
-  const unsigned grid = stream_grid(kernel, smem_bytes, n_vec, chunk_vec);
-  if (grid == 0) return EQAT_ERR_CUDA;
+  const unsigned grid = (unsigned)(chunks < resident ? chunks : resident);
   kernel<<<grid, kThreadsS, smem_bytes, st>>>(args...);
   return launch_status();
 }
@@ -435,7 +450,7 @@ int launch_fakequant_stream(const eqat_desc& d, const eqat_bf16* W, const float*
   int vec_shift = 0;
   while ((8 << vec_shift) < d.group) ++vec_shift;
   using R = Ring<1, kFakequantVpt>;
-  return launch_stream(fakequant_stream_kernel, R::kSmemBytes, R::kChunkVec, n_vec, st, W, s, z, What, n_vec, vec_shift, Q);
+  return launch_stream<fakequant_stream_kernel>(R::kSmemBytes, R::kChunkVec, n_vec, st, W, s, z, What, n_vec, vec_shift, Q);
 }
 
 int launch_ste_bwd_stream(const eqat_desc& d, const eqat_bf16* dWhat, const eqat_bf16* W, const float* s,
@@ -446,10 +461,10 @@ int launch_ste_bwd_stream(const eqat_desc& d, const eqat_bf16* dWhat, const eqat
   using R = Ring<2, kSteVpt>;
   constexpr int smem = R::kSmemBytes, cv = R::kChunkVec;
   switch (d.group) {
-    case 32:  return launch_stream(ste_bwd_stream_kernel<4>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
-    case 64:  return launch_stream(ste_bwd_stream_kernel<8>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
-    case 128: return launch_stream(ste_bwd_stream_kernel<16>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
-    default:  return launch_stream(ste_bwd_stream_kernel<32>, smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    case 32:  return launch_stream<ste_bwd_stream_kernel<4>>(smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    case 64:  return launch_stream<ste_bwd_stream_kernel<8>>(smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    case 128: return launch_stream<ste_bwd_stream_kernel<16>>(smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    default:  return launch_stream<ste_bwd_stream_kernel<32>>(smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
   }
 }
 
@@ -459,10 +474,10 @@ int launch_minmax_stream(const eqat_desc& d, const eqat_bf16* W, float* s, float
   using R = Ring<1, kMinmaxVpt>;
   constexpr int smem = R::kSmemBytes, cv = R::kChunkVec;
   switch (d.group) {
-    case 32:  return launch_stream(minmax_stream_kernel<4>, smem, cv, n_vec, st, W, s, z, n_vec, Q);
-    case 64:  return launch_stream(minmax_stream_kernel<8>, smem, cv, n_vec, st, W, s, z, n_vec, Q);
-    case 128: return launch_stream(minmax_stream_kernel<16>, smem, cv, n_vec, st, W, s, z, n_vec, Q);
-    default:  return launch_stream(minmax_stream_kernel<32>, smem, cv, n_vec, st, W, s, z, n_vec, Q);
+    case 32:  return launch_stream<minmax_stream_kernel<4>>(smem, cv, n_vec, st, W, s, z, n_vec, Q);
+    case 64:  return launch_stream<minmax_stream_kernel<8>>(smem, cv, n_vec, st, W, s, z, n_vec, Q);
+    case 128: return launch_stream<minmax_stream_kernel<16>>(smem, cv, n_vec, st, W, s, z, n_vec, Q);
+    default:  return launch_stream<minmax_stream_kernel<32>>(smem, cv, n_vec, st, W, s, z, n_vec, Q);
   }
 }
 
@@ -474,10 +489,15 @@ int launch_quantize_pack_stream(const eqat_desc& d, const eqat_bf16* W, const fl
   using R = Ring<1, kPackVpt>;
   constexpr int smem = R::kSmemBytes, cv = R::kChunkVec;
   switch (d.bits) {
-    case 2:  return launch_stream(quantize_pack_stream_kernel<2>, smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
-    case 3:  return launch_stream(quantize_pack_stream_kernel<3>, smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
-    default: return launch_stream(quantize_pack_stream_kernel<4>, smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
+    case 2:  return launch_stream<quantize_pack_stream_kernel<2>>(smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
+    case 3:  return launch_stream<quantize_pack_stream_kernel<3>>(smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
+    default: return launch_stream<quantize_pack_stream_kernel<4>>(smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
   }
+}
+
+int launch_wait_expiry_stream(cudaStream_t st) {
+  ring_wait_expiry_kernel<<<1, 32, 0, st>>>(1000000ull);   // 1 ms
+  return launch_status();
 }
 
 int read_stream_status(int* status, int* detail) {

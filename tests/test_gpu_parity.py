@@ -8,7 +8,8 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import TOL, bf16_round, bits_to_torch, f32, rel_err, torch_to_f64
+from helpers import (TOL, Guarded, assert_elementwise, bf16_round, bits_to_torch, contraction_bound, f32, rel_err,
+                     torch_to_f64)
 from oracle import eqat_oracle as O
 from workloads import CONFIGS, Config, Linear, activations_for, get_config, normal_bf16, to_bf16_bits, weight_for
 
@@ -65,7 +66,8 @@ def test_minmax_fakequant_ste_pack(eqat, bits, group):
 
     # min/max initialisation: bit-exact (binary32 arithmetic on both sides)
     s_o, z_o = O.minmax_init(W32, bits, group)
-    s_g = torch.empty(out, ng, device="cuda"); z_g = torch.empty(out, ng, device="cuda")
+    guard = Guarded()                                    # every output below sits between guard words
+    s_g = guard.empty(out, ng); z_g = guard.empty(out, ng)
     eqat.eqat_minmax_init(d, Wd, s_g, z_g)
     assert np.array_equal(s_g.cpu().numpy(), s_o)
     assert np.array_equal(z_g.cpu().numpy(), z_o)
@@ -79,23 +81,23 @@ def test_minmax_fakequant_ste_pack(eqat, bits, group):
         if name == "shifted":
             assert (p_o > (1 << bits) - 1).any()
         # quantise + pack: bit-exact codes, zero points, fp16 step sizes
-        P = torch.empty(out, in_f * bits // 8, dtype=torch.uint8, device="cuda")
-        z8 = torch.empty(out, ng, dtype=torch.uint8, device="cuda")
-        s16 = torch.empty(out, ng, dtype=torch.float16, device="cuda")
+        P = guard.empty(out, in_f * bits // 8, dtype=torch.uint8)
+        z8 = guard.empty(out, ng, dtype=torch.uint8)
+        s16 = guard.empty(out, ng, dtype=torch.float16)
         eqat.eqat_quantize_pack(d, Wd, sd, zd, P, z8, s16)
         P_o, z8_o, s16_o = O.quantize_pack(W32, s, z, bits, group)
         assert np.array_equal(P.cpu().numpy(), P_o), name
         assert np.array_equal(z8.cpu().numpy(), z8_o)
         assert np.array_equal(s16.cpu().numpy().view(np.uint16), s16_o.view(np.uint16))
         # unpack / pack round trip against the oracle's codes
-        codes = torch.empty(out, in_f, dtype=torch.uint8, device="cuda")
+        codes = guard.empty(out, in_f, dtype=torch.uint8)
         eqat.eqat_unpack(d, P, codes)
         assert np.array_equal(codes.cpu().numpy(), q_o.astype(np.uint8))
-        P2 = torch.empty_like(P)
+        P2 = guard.empty(out, in_f * bits // 8, dtype=torch.uint8)
         eqat.eqat_pack(d, dev(q_o.astype(np.uint8)), P2)
         assert np.array_equal(P2.cpu().numpy(), P_o)
         # fake quantiser
-        What = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
+        What = guard.empty(out, in_f, dtype=torch.bfloat16)
         eqat.eqat_fakequant_weight(d, Wd, sd, zd, What)
         What_o = O.dequantize(q_o, s, z, group)
         assert rel_err(torch_to_f64(What), What_o) <= TOL
@@ -106,8 +108,8 @@ def test_minmax_fakequant_ste_pack(eqat, bits, group):
         # STE backward, both readings of Eq. 4
         for dz_mode in (0, 1):
             dd = eqat.make_desc(bits, group, out, in_f, 0, dz_mode)
-            dW = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
-            ds = torch.empty(out, ng, device="cuda"); dz = torch.empty(out, ng, device="cuda")
+            dW = guard.empty(out, in_f, dtype=torch.bfloat16)
+            ds = guard.empty(out, ng); dz = guard.empty(out, ng)
             eqat.eqat_ste_bwd(dd, Gd, Wd, sd, zd, dW, ds, dz)
             dW_o, ds_o, dz_o = O.ste_bwd(G32, W32, s, z, bits, group, dz_mode)
             assert np.array_equal(torch_to_f64(dW), dW_o)            # a masked copy: exact
@@ -116,10 +118,11 @@ def test_minmax_fakequant_ste_pack(eqat, bits, group):
                 assert rel_err(torch_to_f64(dz), dz_o) <= TOL, (name, dz_mode)
             else:
                 assert not torch_to_f64(dz).any()
-        ds_only = torch.empty(out, ng, device="cuda")
+        ds_only = guard.empty(out, ng)
         eqat.eqat_ste_bwd(d, Gd, Wd, sd, zd, dW, ds_only, None)      # dz is optional
         _, ds_o, _ = O.ste_bwd(G32, W32, s, z, bits, group, 0)
         assert rel_err(torch_to_f64(ds_only), ds_o) <= TOL
+        guard.check()
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
@@ -256,31 +259,55 @@ def test_quotients_far_out_of_range_and_zero_points_off_the_grid(eqat):
 
 
 # --------------------------------------------------------------------------- Block-AP layer
+def workspace_for(eqat, d):
+    """Scratch of the Block-AP backward: none (NULL) when the group is reduced inside the GEMM."""
+    n = eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD)
+    assert (n == 0) == (d.group <= 256)
+    return torch.empty(n, dtype=torch.uint8, device="cuda") if n else None
+
+
 def run_block_ap(eqat, cfg, lin, tokens, s, z, dz_mode=0):
     Wb = weight_for(cfg, lin); Xb, dYb = activations_for(cfg, lin, tokens)
     out, in_f, ng = lin.out_features, lin.in_features, lin.in_features // cfg.group
     d = eqat.make_desc(cfg.bits, cfg.group, out, in_f, tokens, dz_mode)
     Wd, Xd, dYd, sd, zd = bits_to_torch(Wb), bits_to_torch(Xb), bits_to_torch(dYb), dev(s), dev(z)
-    Y = torch.empty(tokens, out, dtype=torch.bfloat16, device="cuda")
-    What = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
+    guard = Guarded()
+    Y = guard.empty(tokens, out, dtype=torch.bfloat16)
+    What = guard.empty(out, in_f, dtype=torch.bfloat16)
     eqat.qlinear_fakequant_fwd(d, Xd, Wd, sd, zd, Y, What)
-    dX = torch.empty(tokens, in_f, dtype=torch.bfloat16, device="cuda")
-    dW = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
-    ds = torch.empty(out, ng, device="cuda"); dz = torch.empty(out, ng, device="cuda")
-    ws = torch.empty(eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD), dtype=torch.uint8, device="cuda")
+    dX = guard.empty(tokens, in_f, dtype=torch.bfloat16)
+    dW = guard.empty(out, in_f, dtype=torch.bfloat16)
+    ds = guard.empty(out, ng); dz = guard.empty(out, ng)
+    ws = workspace_for(eqat, d)
     eqat.qlinear_fakequant_bwd(d, Xd, dYd, Wd, sd, zd, What, dX, dW, ds, dz, ws)
-    torch.cuda.synchronize()
+    guard.check()
     return dict(W=f32(Wb), X=f32(Xb), dY=f32(dYb), Y=Y, What=What, dX=dX, dW=dW, ds=ds, dz=dz)
+
+
+def check_contractions(r, What_o):
+    """Y and dX element by element: each within the rounding a correct kernel can show (see
+    helpers.contraction_bound), next to the norm criterion."""
+    X, dY = r["X"], r["dY"]
+    Y_o, dX_o = O.linear_fwd(X, What_o), O.linear_bwd_dx(dY, What_o)
+    assert rel_err(torch_to_f64(r["Y"]), Y_o) <= TOL
+    assert rel_err(torch_to_f64(r["dX"]), dX_o) <= TOL
+    aW, W2 = np.abs(What_o), What_o ** 2
+    assert_elementwise(torch_to_f64(r["Y"]), Y_o,
+                       contraction_bound(Y_o, O.linear_fwd(np.abs(X), aW), O.linear_fwd(X ** 2, W2)), "Y")
+    assert_elementwise(torch_to_f64(r["dX"]), dX_o,
+                       contraction_bound(dX_o, O.linear_bwd_dx(np.abs(dY), aW), O.linear_bwd_dx(dY ** 2, W2)), "dX")
 
 
 def check_block_ap(r, s, z, bits, group, dz_mode=0):
     What_o = O.fake_quant_weight(r["W"], s, z, bits, group)
     assert rel_err(torch_to_f64(r["What"]), What_o) <= TOL
-    assert rel_err(torch_to_f64(r["Y"]), O.linear_fwd(r["X"], What_o)) <= TOL
-    assert rel_err(torch_to_f64(r["dX"]), O.linear_bwd_dx(r["dY"], What_o)) <= TOL
+    check_contractions(r, What_o)
     G = O.weight_grad(r["dY"], r["X"])
     dW_o, ds_o, dz_o = O.ste_bwd(G, r["W"], s, z, bits, group, dz_mode)
     assert rel_err(torch_to_f64(r["dW"]), dW_o) <= TOL
+    # dW is the gradient of W_hat, masked, rounded once to bf16 (both operands of its contraction are exact)
+    absG = O.weight_grad(np.abs(r["dY"]), np.abs(r["X"]))
+    assert_elementwise(torch_to_f64(r["dW"]), dW_o, contraction_bound(dW_o, absG, 0.0, 0), "dW")
     assert rel_err(torch_to_f64(r["ds"]), ds_o) <= TOL
     if np.linalg.norm(dz_o) > 0:
         assert rel_err(torch_to_f64(r["dz"]), dz_o) <= TOL
@@ -324,7 +351,7 @@ def test_outputs_aligned_to_16_bytes_only(eqat):
     Xd, dYd, sd, zd = bits_to_torch(Xb), bits_to_torch(dYb), dev(s), dev(z)
     d = eqat.make_desc(cfg.bits, cfg.group, out, in_f, T)
     What = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda")
-    ws = torch.empty(eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD), dtype=torch.uint8, device="cuda")
+    ws = workspace_for(eqat, d)
     res = []
     for shift in (0, 8):                                         # elements: 0 or 16 bytes past a 512-byte boundary
         Y = torch.zeros(T * out + 16, dtype=torch.bfloat16, device="cuda")[shift:shift + T * out].view(T, out)
@@ -363,14 +390,15 @@ def run_e2e(eqat, cfg, lin, tokens, with_dz=True, fp16_steps=False):
     Pd, z8d = dev(P_o), dev(z8_o)
     s16d = torch.from_numpy(s16_o.view(np.int16)).view(torch.float16).cuda()
     Xd, dYd = bits_to_torch(Xb), bits_to_torch(dYb)
-    Y = torch.empty(tokens, out, dtype=torch.bfloat16, device="cuda")
-    dX = torch.empty(tokens, in_f, dtype=torch.bfloat16, device="cuda")
-    ds = torch.empty(out, ng, device="cuda")
-    dz = torch.empty(out, ng, device="cuda") if with_dz else None
+    guard = Guarded()
+    Y = guard.empty(tokens, out, dtype=torch.bfloat16)
+    dX = guard.empty(tokens, in_f, dtype=torch.bfloat16)
+    ds = guard.empty(out, ng)
+    dz = guard.empty(out, ng) if with_dz else None
     eqat.qlinear_packed_fwd(d, Xd, Pd, s16d, z8d, Y)
     eqat.qlinear_packed_bwd_dx(d, dYd, Pd, s16d, z8d, dX)
     eqat.qlinear_packed_bwd_ds(d, Xd, dYd, Pd, z8d, s16d, ds, dz)
-    torch.cuda.synchronize()
+    guard.check()
     q = O.unpack_rows(P_o, cfg.bits, in_f)
     return dict(X=f32(Xb), dY=f32(dYb), q=q, z8=z8_o, s16=s16_o.astype(np.float32), Y=Y, dX=dX, ds=ds, dz=dz,
                 W=W32, s=s, z=z)
@@ -378,8 +406,7 @@ def run_e2e(eqat, cfg, lin, tokens, with_dz=True, fp16_steps=False):
 
 def check_e2e(r, group):
     What_o = O.dequantize(r["q"], r["s16"], r["z8"], group)
-    assert rel_err(torch_to_f64(r["Y"]), O.linear_fwd(r["X"], What_o)) <= TOL
-    assert rel_err(torch_to_f64(r["dX"]), O.linear_bwd_dx(r["dY"], What_o)) <= TOL
+    check_contractions(r, What_o)
     assert rel_err(torch_to_f64(r["ds"]), O.e2e_ds(r["dY"], r["X"], r["q"], r["z8"], group)) <= TOL
     if r["dz"] is not None:
         assert rel_err(torch_to_f64(r["dz"]), O.e2e_dz(r["dY"], r["X"], r["s16"], group)) <= TOL
@@ -444,3 +471,93 @@ def test_e2e_is_deterministic_and_matches_block_ap_forward(eqat):
     r = run_block_ap(eqat, cfg, lin, 256, a["s"], a["z"])
     assert rel_err(torch_to_f64(r["Y"]), torch_to_f64(a["Y"])) <= 2e-3
     assert rel_err(torch_to_f64(r["dX"]), torch_to_f64(a["dX"])) <= 2e-3
+
+
+# --------------------------------------------------------------------------- hand-off side outputs, alignment, waits
+@pytest.mark.parametrize("kind,bits", [("z2", 2), ("z4", 4)])
+def test_handoff_side_outputs_against_hand_values(eqat, kind, bits):
+    """Step sizes that fp16 cannot hold exactly and zero points that are fractional or outside [0, Q]: the fp16
+    bit patterns and the stored bytes are the hand-derived ones of tests/golden/handoff_side_outputs.txt (the
+    same fixture pins the oracle), through both quantise + pack kernels (groups of 32 and channel-wise)."""
+    import os
+    from conftest import GOLDEN
+    rows = [[x.strip() for x in l.split("|")] for l in open(os.path.join(GOLDEN, "handoff_side_outputs.txt"))
+            if l.strip() and not l.startswith("#")]
+    s_rows = [(float(v), int(h, 16)) for k, v, h in rows if k == "s"]
+    z_rows = [(float(v), int(b)) for k, v, b in rows if k == kind]
+    for group, in_f in ((32, 128), (512, 512)):
+        ng, out = in_f // group, 8
+        s = np.array([[s_rows[(o + j) % 4][0] for j in range(ng)] for o in range(out)], np.float32)
+        s_bits = np.array([[s_rows[(o + j) % 4][1] for j in range(ng)] for o in range(out)], np.uint16)
+        z = np.array([[z_rows[(o + j) % len(z_rows)][0] for j in range(ng)] for o in range(out)], np.float32)
+        z_bytes = np.array([[z_rows[(o + j) % len(z_rows)][1] for j in range(ng)] for o in range(out)], np.uint8)
+        Wb = normal_bf16((out, in_f), 0.05, "handoff", kind, group)
+        d = eqat.make_desc(bits, group, out, in_f)
+        guard = Guarded()
+        P = guard.empty(out, in_f * bits // 8, dtype=torch.uint8)
+        z8 = guard.empty(out, ng, dtype=torch.uint8)
+        s16 = guard.empty(out, ng, dtype=torch.float16)
+        eqat.eqat_quantize_pack(d, bits_to_torch(Wb), dev(s), dev(z), P, z8, s16)
+        guard.check()
+        assert np.array_equal(z8.cpu().numpy(), z_bytes)
+        assert np.array_equal(s16.cpu().numpy().view(np.uint16), s_bits)
+        P_o, z8_o, s16_o = O.quantize_pack(f32(Wb), s, z, bits, group)
+        assert np.array_equal(P.cpu().numpy(), P_o)
+        assert np.array_equal(z8_o, z_bytes) and np.array_equal(s16_o.view(np.uint16), s_bits)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("tokens", [1, 4, 300])
+def test_packed_weight_aligned_to_16_bytes_only(eqat, bits, tokens):
+    """The packed matrix (and its step sizes and zero points) 16 bytes past a 256-byte boundary: 16-byte alignment is
+    all the interface asks for, so the kernels must not fetch whole 32-byte sectors from it.  Same bits as the
+    aligned run, through the matrix-vector kernel (1 and 4 tokens) and the tiled one."""
+    group = 64 if bits == 2 else 128
+    cfg = small_cfg(f"wq16_{bits}", 320, 512, bits, group, tokens, "student_t4", 0.02, 0.01)
+    lin = cfg.linears[0]
+    out, in_f, ng = 320, 512, 512 // group
+    W32 = f32(weight_for(cfg, lin))
+    s, z = O.minmax_init(W32, bits, group)
+    P_o, z8_o, s16_o = O.quantize_pack(W32, s, z, bits, group)
+    Xb, dYb = activations_for(cfg, lin, tokens)
+    Xd, dYd = bits_to_torch(Xb), bits_to_torch(dYb)
+    d = eqat.make_desc(bits, group, out, in_f, tokens)
+    res = []
+    for shift in (0, 16):
+        def place(a):
+            raw = torch.zeros(a.nbytes + 32, dtype=torch.uint8, device="cuda")
+            v = raw[shift:shift + a.nbytes]
+            v.copy_(torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).ravel()))
+            assert v.data_ptr() % 32 == shift
+            return v
+        Pd, z8d, s16d = place(P_o), place(z8_o), place(s16_o)
+        guard = Guarded()
+        Y = guard.empty(tokens, out, dtype=torch.bfloat16)
+        dX = guard.empty(tokens, in_f, dtype=torch.bfloat16)
+        ds = guard.empty(out, ng)
+        eqat.qlinear_packed_fwd(d, Xd, Pd, s16d, z8d, Y)
+        eqat.qlinear_packed_bwd_dx(d, dYd, Pd, s16d, z8d, dX)
+        eqat.qlinear_packed_bwd_ds(d, Xd, dYd, Pd, z8d, s16d, ds)
+        guard.check()
+        res.append((Y.clone(), dX.clone(), ds.clone()))
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
+    q = O.unpack_rows(P_o, bits, in_f)
+    What_o = O.dequantize(q, s16_o.astype(np.float32), z8_o, group)
+    assert rel_err(torch_to_f64(res[1][0]), O.linear_fwd(f32(Xb), What_o)) <= TOL
+
+
+@pytest.mark.parametrize("which,name", [(0, "GEMM kernels"), (1, "streaming kernels")])
+def test_a_bounded_wait_runs_out_cleanly(eqat, which, name):
+    """One warp waits 1 ms for a barrier that nothing signals, through the kernels' own wait routine: the kernel
+    must end normally, the status word must say TIMEOUT with the self-test's site code exactly once, and the
+    library must work afterwards (the context is intact)."""
+    torch.cuda.synchronize()
+    assert eqat.device_status() == (0, 0)
+    eqat.eqat_selftest_wait_expiry(which)
+    torch.cuda.synchronize()                                   # the kernel returned: no hang, no fault
+    assert eqat.device_status() == (eqat.EQAT_ERR_TIMEOUT, 9)
+    assert eqat.device_status() == (0, 0)                      # reading clears it
+    cfg = get_config("c1"); lin = cfg.linears[0]
+    s, z = O.minmax_init(f32(weight_for(cfg, lin)), cfg.bits, cfg.group)
+    check_block_ap(run_block_ap(eqat, cfg, lin, cfg.tokens, s, z), s, z, cfg.bits, cfg.group)

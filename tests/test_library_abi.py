@@ -41,7 +41,10 @@ def test_status_strings(eqat):
 
 def test_workspace_sizes(eqat):
     d = eqat.make_desc(2, 64, 512, 512, 256)
-    assert eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD) == 512 * 512 * 2
+    assert eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD) == 0          # reduced inside the GEMM: no scratch
+    assert eqat.workspace_bytes(eqat.make_desc(2, 256, 512, 512, 256), eqat.EQAT_OP_FAKEQUANT_BWD) == 0
+    dc = eqat.make_desc(2, 512, 512, 512, 256)                               # channel-wise: dW_hat in bf16
+    assert eqat.workspace_bytes(dc, eqat.EQAT_OP_FAKEQUANT_BWD) == 512 * 512 * 2
     assert eqat.workspace_bytes(d, eqat.EQAT_OP_PACKED_BWD_DS) == 0
     with pytest.raises(eqat.EqatError):
         eqat.workspace_bytes(d, 99)
@@ -74,8 +77,10 @@ def test_null_and_misaligned_pointers(eqat):
     assert eqat.lib.qlinear_packed_fwd(ctypes.byref(d0), ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_SHAPE
     d96 = eqat.make_desc(2, 64, 96, 512, 256)
     assert eqat.lib.qlinear_fakequant_fwd(ctypes.byref(d96), ok, ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_SHAPE
-    # workspace: missing, too small, misaligned
+    # workspace of the channel-wise backward: missing, too small, misaligned
+    dc = eqat.make_desc(2, 512, 512, 512, 256)
     args = [ok] * 10
-    assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(d), *args, None, 0, None) == eqat.EQAT_ERR_WORKSPACE
-    assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(d), *args, ok, 16, None) == eqat.EQAT_ERR_WORKSPACE
-    assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(d), *args, ctypes.c_void_p(0x1010), 1 << 20, None) == eqat.EQAT_ERR_WORKSPACE
+    assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(dc), *args, None, 0, None) == eqat.EQAT_ERR_WORKSPACE
+    assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(dc), *args, ok, 16, None) == eqat.EQAT_ERR_WORKSPACE
+    assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(dc), *args, ctypes.c_void_p(0x1010), 1 << 20, None) == eqat.EQAT_ERR_WORKSPACE
+    assert eqat.lib.eqat_selftest_wait_expiry(7, None) == eqat.EQAT_ERR_UNSUPPORTED

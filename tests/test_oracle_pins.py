@@ -308,6 +308,30 @@ def pin_sizes(o):
     assert (o.unpack_rows(P, 2, 128) == q).all() and (z8 == z).all()
 
 
+def pin_handoff_side_outputs(o):
+    """Step sizes as FP16 bit patterns and zero points as N-bit bytes, against hand-derived values."""
+    rows = []
+    with open(os.path.join(GOLDEN, "handoff_side_outputs.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                rows.append([x.strip() for x in line.split("|")])
+    s_rows = [(float(v), int(h, 16)) for k, v, h in rows if k == "s"]
+    assert len(s_rows) == 4
+    for kind, bits in (("z2", 2), ("z4", 4)):
+        z_rows = [(float(v), int(b)) for k, v, b in rows if k == kind]
+        assert len(z_rows) >= 3
+        ng = len(z_rows)
+        s = np.array([[s_rows[i % len(s_rows)][0] for i in range(ng)]], np.float32)
+        z = np.array([[v for v, _ in z_rows]], np.float32)
+        W = np.zeros((1, ng * 8), np.float32)
+        P, z8, s16 = o.quantize_pack(W, s, z, bits, 8)
+        assert z8.dtype == np.uint8 and s16.dtype == np.float16
+        assert z8.tolist() == [[b for _, b in z_rows]]
+        assert s16.view(np.uint16).tolist() == [[s_rows[i % len(s_rows)][1] for i in range(ng)]]
+        # w = 0 quantises to clamp(0 + rint(z), 0, Q): the packed codes repeat the stored zero point
+        assert (o.unpack_rows(P, bits, ng * 8) == np.repeat(z8, 8, axis=1)).all()
+
+
 def pin_shapes_other_models(o):
     assert sum(l.out_features * l.in_features * l.count for l in LINEARS["13b"]) == 317_194_240
     assert sum(l.out_features * l.in_features * l.count for l in LINEARS["70b"]) == 855_638_016
@@ -319,7 +343,8 @@ def pin_shapes_other_models(o):
 
 PINS = [pin_worked_example, pin_rounding_is_half_to_even, pin_inclusive_bounds, pin_quantiser_invariants,
         pin_zero_point_is_rounded_in_forward, pin_ste_against_forward, pin_contractions, pin_e2e_ds,
-        pin_minmax, pin_pack_golden, pin_pack_roundtrip_and_bigint, pin_sizes, pin_shapes_other_models]
+        pin_minmax, pin_pack_golden, pin_pack_roundtrip_and_bigint, pin_sizes, pin_handoff_side_outputs,
+        pin_shapes_other_models]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
@@ -357,6 +382,13 @@ MUTATIONS = {
     "pack_msb_first": [('np.packbits(bitplanes.ravel().astype(np.uint8), bitorder="little")',
                         'np.packbits(bitplanes.ravel().astype(np.uint8), bitorder="big")')],
     "minmax_z_sign": [("z = -np.rint(mn / s)", "z = np.rint(mn / s)")],
+    "handoff_zero_point_clamp_dropped": [("z8 = np.clip(round_zero_point(z), 0, qmax(bits)).astype(np.uint8)",
+                                          "z8 = round_zero_point(z).astype(np.int64).astype(np.uint8)")],
+    "handoff_zero_point_truncated": [("z8 = np.clip(round_zero_point(z), 0, qmax(bits)).astype(np.uint8)",
+                                      "z8 = np.clip(np.trunc(np.asarray(z, np.float64)), 0, qmax(bits)).astype(np.uint8)")],
+    "handoff_step_size_truncated_to_fp16": [("s16 = np.asarray(s, np.float32).astype(np.float16)",
+                                             "s16 = (np.ascontiguousarray(s, np.float32).view(np.uint32) & np.uint32(0xFFFFE000))"
+                                             ".view(np.float32).astype(np.float16)")],
     "group_sum_wrong_axis": [("return A.reshape(out, in_f // group, group).sum(axis=2, dtype=np.float64)",
                               "return A.reshape(out, group, in_f // group).sum(axis=1, dtype=np.float64)")],
 }

@@ -2,9 +2,11 @@
 allocate device memory (their device memory belongs to another framework's pool,
 or they sit where the synchronisation cudaMalloc may imply is unacceptable).
 
-It must give what qlinear_fakequant_bwd gives with a caller-allocated workspace,
-on two calls in a row (the built-in scratch array is shared by all calls and keeps
-the previous call's contents), and must refuse problems larger than the array.
+It must give exactly what qlinear_fakequant_bwd gives with a caller-allocated
+workspace (same kernels, same inputs: bit for bit) and what the oracle gives
+(within the tolerance of the other parity tests), on two calls in a row (the
+built-in scratch array is shared by all calls and keeps the previous call's
+contents), and must refuse problems larger than the array.
 Collected last so that a failure here cannot mask any other test.
 """
 import ctypes
@@ -62,7 +64,11 @@ def test_matches_the_workspace_variant_twice_in_a_row(eqat, channel_wise):
     # two different upstream gradients, so the second call must not see the first call's scratch
     dY1 = bits_to_torch(dYb)
     dY2 = (dY1.float() * -0.5 + 0.003).to(torch.bfloat16)
-    ws = torch.empty(eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD), dtype=torch.uint8, device="cuda")
+    n_ws = eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD)
+    assert (n_ws > 0) == channel_wise
+    ws = torch.empty(n_ws, dtype=torch.uint8, device="cuda") if n_ws else None
+    W32, X32 = f32(Wb), f32(Xb)
+    What_o = O.fake_quant_weight(W32, s, z, bits, g)
     for dY in (dY1, dY2):
         ref = outputs(); got = outputs()
         eqat.qlinear_fakequant_bwd(d, Xd, dY, Wd, sd, zd, What, *ref, ws)
@@ -70,5 +76,10 @@ def test_matches_the_workspace_variant_twice_in_a_row(eqat, channel_wise):
         torch.cuda.synchronize()
         for name, a, b in zip(("dX", "dW", "ds", "dz"), got, ref):
             assert np.linalg.norm(torch_to_f64(b)) > 0, name
-            assert rel_err(torch_to_f64(a), torch_to_f64(b)) <= TOL, name
+            assert torch.equal(a, b), name                       # the same kernels on the same inputs
+        # and against the oracle (Eqs. 3-5 on the fp64 weight gradient)
+        dY64 = torch_to_f64(dY)
+        dW_o, ds_o, dz_o = O.ste_bwd(O.weight_grad(dY64, X32), W32, s, z, bits, g)
+        for name, a, b in zip(("dX", "dW", "ds", "dz"), got, (O.linear_bwd_dx(dY64, What_o), dW_o, ds_o, dz_o)):
+            assert rel_err(torch_to_f64(a), b) <= TOL, name
     assert eqat.device_status() == (0, 0)
