@@ -11,6 +11,11 @@ Prints one JSON line (rank 0).  `value` is the tensor-core throughput of the six
 contractions per linear (2*T*in*out flop each) over the whole step, all kernels
 included in the time; dequantisation, STE and epilogue arithmetic are not counted
 as flops.
+
+On one GPU the same run then times, outside the headline's timed region and reported under their own keys:
+the other workloads (7B w4g128 Block-AP, 13B w3g128 E2E-QP, 70B w2g64 both modes) under "configs", and the five
+streaming kernels cold and back to back over buffer sets several times the L2 under "streaming".
+`--gpus N` started without a launcher spawns the N ranks itself.
 """
 from __future__ import annotations
 
@@ -36,6 +41,18 @@ BITS, GROUP = 2, 64
 T_BLOCK_AP, T_E2E = 4096, 16384
 WORKLOAD = "llama2-7b decoder-block linears, w2g64: Block-AP fwd+bwd @4096 tok, hand-off, E2E-QP fwd/dX/ds @16384 tok"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# Nominal figures of the part, for context beside the measured denominators: dense bf16 tensor throughput and the
+# HBM3e bandwidth the workload description quotes ("~8 TB/s").
+NOMINAL_PEAKS = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
+
+# The other workloads: same path, other bit widths, group sizes and models.  Each is timed after the headline
+# step and reported under "configs" (the headline line itself stays the 7B w2g64 step).
+#   model, bits, group, Block-AP tokens (0 = mode not run), E2E-QP tokens, weight recipe (dist, scale, outlier fraction)
+EXTRA_CONFIGS = {
+    "c2_7b_w4g128_block_ap": dict(model="7b", bits=4, group=128, t_ap=4096, t_e2e=0, w=("student_t4", 0.02, 0.01), steps=10),
+    "c4_13b_w3g128_e2e_qp": dict(model="13b", bits=3, group=128, t_ap=0, t_e2e=8192, w=("student_t4", 0.02, 0.01), steps=10),
+    "c5_70b_w2g64_both": dict(model="70b", bits=2, group=64, t_ap=8192, t_e2e=8192, w=("student_t4", 0.015, 0.0), steps=5),
+}
 
 
 # DRAM bytes (read + write) per launch of the packed-weight GEMMs at 16384 tokens, w2g64, by linear shape: ncu
@@ -85,8 +102,8 @@ def load_peaks():
     return d
 
 
-def step_flops(t_block_ap=T_BLOCK_AP, t_e2e=T_E2E):
-    per_token = sum(2 * l.in_features * l.out_features * l.count for l in LINEARS["7b"])
+def step_flops(t_block_ap=T_BLOCK_AP, t_e2e=T_E2E, model="7b"):
+    per_token = sum(2 * l.in_features * l.out_features * l.count for l in LINEARS[model])
     return 3 * per_token * t_block_ap, 3 * per_token * t_e2e
 
 
@@ -166,37 +183,79 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- the workload on one GPU
-class BlockWorkload:
-    """Device buffers for the seven linears; activations shared per shape, weights per linear."""
+def synth_weight(shape, recipe, gen, device):
+    """Synthetic stand-in for a trained weight, drawn on the device: N(0, scale^2) or scale * Student-t(4)
+    (Z / sqrt(mean of four squared normals)), optionally with a fraction of the input channels scaled by 10."""
+    dist, scale, outlier_frac = recipe
+    w = torch.randn(shape, generator=gen, device=device, dtype=torch.float32)
+    if dist == "student_t4":
+        chi = torch.zeros(shape, device=device, dtype=torch.float32)
+        for _ in range(4):
+            chi += torch.randn(shape, generator=gen, device=device, dtype=torch.float32) ** 2
+        w = w / torch.sqrt(chi / 4)
+    w *= scale
+    if outlier_frac > 0:
+        n = int(np.ceil(outlier_frac * shape[1]))
+        cols = torch.randperm(shape[1], generator=gen, device=device)[:n]
+        w[:, cols] *= 10.0
+    return w.to(torch.bfloat16)
 
-    def __init__(self, eqat, device, seed, t_block_ap=T_BLOCK_AP, t_e2e=T_E2E):
+
+# kernels launched by one call of each class (groups of at most 256 elements)
+KERNELS_PER_CALL = {"minmax_init": 1, "fakequant_fwd": 2, "fakequant_bwd": 2, "quantize_pack": 1, "unpack": 1,
+                    "packed_fwd": 1, "packed_bwd_dx": 1, "packed_bwd_ds": 1}
+# contractions (2*T*in*out flop each) inside one call of each class
+CONTRACTIONS = {"fakequant_fwd": 1, "fakequant_bwd": 2, "packed_fwd": 1, "packed_bwd_dx": 1, "packed_bwd_ds": 1}
+
+
+class BlockWorkload:
+    """Device buffers for the linears of one decoder block; activations shared per shape, weights per linear.
+
+    One step = for every linear: [min/max init,] Block-AP forward + backward at `t_ap` tokens, [quantise + pack,
+    unpack,] E2E-QP forward / dX / ds at `t_e2e` tokens.  A mode with 0 tokens is left out; the bracketed
+    hand-off calls are part of the step only with `handoff` (the headline step), otherwise they run once here."""
+
+    def __init__(self, eqat, device, seed, t_block_ap=T_BLOCK_AP, t_e2e=T_E2E, model="7b", bits=BITS, group=GROUP,
+                 weight=("normal", 0.02, 0.0), handoff=True):
         self.eqat, self.device = eqat, device
-        self.t_ap, self.t_e2e = t_block_ap, t_e2e
+        self.t_ap, self.t_e2e, self.model, self.bits, self.group, self.handoff = t_block_ap, t_e2e, model, bits, group, handoff
         g = torch.Generator(device=device); g.manual_seed(seed)
         bf, dev = torch.bfloat16, device
+        t_max = max(t_block_ap, t_e2e)
         self.shapes, self.layers = {}, []
-        for lin in LINEARS["7b"]:
-            out, in_f, ng = lin.out_features, lin.in_features, lin.in_features // GROUP
+        for lin in LINEARS[model]:
+            out, in_f, ng = lin.out_features, lin.in_features, lin.in_features // group
             sh = dict(lin=lin,
-                      X=torch.randn(t_e2e, in_f, generator=g, device=dev, dtype=torch.float32).to(bf),
-                      dY=(torch.randn(t_e2e, out, generator=g, device=dev, dtype=torch.float32) * 1e-2).to(bf),
-                      Y=torch.empty(t_e2e, out, dtype=bf, device=dev), dX=torch.empty(t_e2e, in_f, dtype=bf, device=dev),
+                      X=torch.randn(t_max, in_f, generator=g, device=dev, dtype=torch.float32).to(bf),
+                      dY=(torch.randn(t_max, out, generator=g, device=dev, dtype=torch.float32) * 1e-2).to(bf),
+                      Y=torch.empty(t_max, out, dtype=bf, device=dev), dX=torch.empty(t_max, in_f, dtype=bf, device=dev),
                       What=torch.empty(out, in_f, dtype=bf, device=dev), dW=torch.empty(out, in_f, dtype=bf, device=dev),
                       ds=torch.empty(out, ng, device=dev), dz=torch.empty(out, ng, device=dev),
                       ds2=torch.empty(out, ng, device=dev),
-                      codes=torch.empty(out, in_f, dtype=torch.uint8, device=dev),
-                      d_ap=eqat.make_desc(BITS, GROUP, out, in_f, t_block_ap), d_e2e=eqat.make_desc(BITS, GROUP, out, in_f, t_e2e))
-            sh["ws"] = torch.empty(eqat.workspace_bytes(sh["d_ap"], eqat.EQAT_OP_FAKEQUANT_BWD), dtype=torch.uint8, device=dev)
+                      codes=torch.empty(out, in_f, dtype=torch.uint8, device=dev) if handoff else None,
+                      d_ap=eqat.make_desc(bits, group, out, in_f, max(t_block_ap, 1)),
+                      d_e2e=eqat.make_desc(bits, group, out, in_f, max(t_e2e, 1)))
+            n_ws = eqat.workspace_bytes(sh["d_ap"], eqat.EQAT_OP_FAKEQUANT_BWD)
+            sh["ws"] = torch.empty(n_ws, dtype=torch.uint8, device=dev) if n_ws else None
             self.shapes[lin.name] = sh
             for i in range(lin.count):
-                W = (torch.randn(out, in_f, generator=g, device=dev, dtype=torch.float32) * 0.02).to(bf)
-                self.layers.append(dict(shape=lin.name, W=W,
-                                        s=torch.empty(out, ng, device=dev), z=torch.empty(out, ng, device=dev),
-                                        P=torch.empty(out, in_f * BITS // 8, dtype=torch.uint8, device=dev),
-                                        z8=torch.empty(out, ng, dtype=torch.uint8, device=dev),
-                                        s16=torch.empty(out, ng, dtype=torch.float16, device=dev)))
-        self.calls_per_step = 8 * len(self.layers)
-        self.kernels_per_step = 10 * len(self.layers)     # fwd = 2 kernels, bwd = 2 (group <= 256), the other six calls 1 each
+                W = synth_weight((out, in_f), weight, g, dev)
+                L = dict(shape=lin.name, W=W,
+                         s=torch.empty(out, ng, device=dev), z=torch.empty(out, ng, device=dev),
+                         P=torch.empty(out, in_f * bits // 8, dtype=torch.uint8, device=dev),
+                         z8=torch.empty(out, ng, dtype=torch.uint8, device=dev),
+                         s16=torch.empty(out, ng, dtype=torch.float16, device=dev))
+                eqat.eqat_minmax_init(sh["d_ap"], W, L["s"], L["z"])
+                eqat.eqat_quantize_pack(sh["d_ap"], W, L["s"], L["z"], L["P"], L["z8"], L["s16"])
+                self.layers.append(L)
+        self.classes = ((["minmax_init"] if handoff else []) + (["fakequant_fwd", "fakequant_bwd"] if t_block_ap else [])
+                        + (["quantize_pack", "unpack"] if handoff else [])
+                        + (["packed_fwd", "packed_bwd_dx", "packed_bwd_ds"] if t_e2e else []))
+        self.calls_per_step = len(self.classes) * len(self.layers)
+        self.kernels_per_step = sum(KERNELS_PER_CALL[c] for c in self.classes) * len(self.layers)
+
+    def flops(self):
+        return step_flops(self.t_ap, self.t_e2e, self.model)
 
     def step(self, timers=None):
         e = self.eqat
@@ -208,17 +267,22 @@ class BlockWorkload:
             timers.setdefault(name, []).append((a, b))
         for L in self.layers:
             S = self.shapes[L["shape"]]
-            Xa, dYa, Ya, dXa = S["X"][: self.t_ap], S["dY"][: self.t_ap], S["Y"][: self.t_ap], S["dX"][: self.t_ap]
             tag = L["shape"]
-            timed("minmax_init/" + tag, lambda: e.eqat_minmax_init(S["d_ap"], L["W"], L["s"], L["z"]))
-            timed("fakequant_fwd/" + tag, lambda: e.qlinear_fakequant_fwd(S["d_ap"], Xa, L["W"], L["s"], L["z"], Ya, S["What"]))
-            timed("fakequant_bwd/" + tag, lambda: e.qlinear_fakequant_bwd(S["d_ap"], Xa, dYa, L["W"], L["s"], L["z"], S["What"],
-                                                                            dXa, S["dW"], S["ds"], S["dz"], S["ws"]))
-            timed("quantize_pack/" + tag, lambda: e.eqat_quantize_pack(S["d_ap"], L["W"], L["s"], L["z"], L["P"], L["z8"], L["s16"]))
-            timed("unpack/" + tag, lambda: e.eqat_unpack(S["d_ap"], L["P"], S["codes"]))
-            timed("packed_fwd/" + tag, lambda: e.qlinear_packed_fwd(S["d_e2e"], S["X"], L["P"], L["s16"], L["z8"], S["Y"]))
-            timed("packed_bwd_dx/" + tag, lambda: e.qlinear_packed_bwd_dx(S["d_e2e"], S["dY"], L["P"], L["s16"], L["z8"], S["dX"]))
-            timed("packed_bwd_ds/" + tag, lambda: e.qlinear_packed_bwd_ds(S["d_e2e"], S["X"], S["dY"], L["P"], L["z8"], L["s16"], S["ds2"]))
+            if self.handoff:
+                timed("minmax_init/" + tag, lambda: e.eqat_minmax_init(S["d_ap"], L["W"], L["s"], L["z"]))
+            if self.t_ap:
+                Xa, dYa, Ya, dXa = S["X"][: self.t_ap], S["dY"][: self.t_ap], S["Y"][: self.t_ap], S["dX"][: self.t_ap]
+                timed("fakequant_fwd/" + tag, lambda: e.qlinear_fakequant_fwd(S["d_ap"], Xa, L["W"], L["s"], L["z"], Ya, S["What"]))
+                timed("fakequant_bwd/" + tag, lambda: e.qlinear_fakequant_bwd(S["d_ap"], Xa, dYa, L["W"], L["s"], L["z"], S["What"],
+                                                                                dXa, S["dW"], S["ds"], S["dz"], S["ws"]))
+            if self.handoff:
+                timed("quantize_pack/" + tag, lambda: e.eqat_quantize_pack(S["d_ap"], L["W"], L["s"], L["z"], L["P"], L["z8"], L["s16"]))
+                timed("unpack/" + tag, lambda: e.eqat_unpack(S["d_ap"], L["P"], S["codes"]))
+            if self.t_e2e:
+                Xe, dYe, Ye, dXe = S["X"][: self.t_e2e], S["dY"][: self.t_e2e], S["Y"][: self.t_e2e], S["dX"][: self.t_e2e]
+                timed("packed_fwd/" + tag, lambda: e.qlinear_packed_fwd(S["d_e2e"], Xe, L["P"], L["s16"], L["z8"], Ye))
+                timed("packed_bwd_dx/" + tag, lambda: e.qlinear_packed_bwd_dx(S["d_e2e"], dYe, L["P"], L["s16"], L["z8"], dXe))
+                timed("packed_bwd_ds/" + tag, lambda: e.qlinear_packed_bwd_ds(S["d_e2e"], Xe, dYe, L["P"], L["z8"], L["s16"], S["ds2"]))
 
 
 class HostStaging:
@@ -301,7 +365,8 @@ class HostStaging:
 def oracle_sample(seed=0):
     """The oracle on a bounded sample of the same workload: the 4096x4096 linear,
     element-wise steps on 512 output rows, contractions on 256 token rows x 512
-    output rows.  Returns (flops counted the same way, seconds, description)."""
+    output rows.  Returns (flops counted the same way, seconds, description, seconds
+    spent inside the five matrix products)."""
     from oracle import eqat_oracle as O
     from workloads import from_bf16_bits, get_config, normal_bf16
     rows, toks, in_f = 512, 256, 4096
@@ -309,20 +374,24 @@ def oracle_sample(seed=0):
     Xb = normal_bf16((toks, in_f), 1.0, "bench_oracle", seed, "X")
     dYb = normal_bf16((toks, rows), 1e-2, "bench_oracle", seed, "dY")
     W, X, dY = from_bf16_bits(Wb), from_bf16_bits(Xb), from_bf16_bits(dYb)
+    mm = [0.0]
+    def product(fn, *a):
+        t = time.perf_counter(); r = fn(*a); mm[0] += time.perf_counter() - t
+        return r
     t0 = time.perf_counter()
     s, z = O.minmax_init(W, BITS, GROUP)
     What = O.fake_quant_weight(W, s, z, BITS, GROUP)
-    Y = O.linear_fwd(X, What); dX = O.linear_bwd_dx(dY, What)
-    G = O.weight_grad(dY, X)
+    Y = product(O.linear_fwd, X, What); dX = product(O.linear_bwd_dx, dY, What)
+    G = product(O.weight_grad, dY, X)
     O.ste_bwd(G, W, s, z, BITS, GROUP)
     P, z8, s16 = O.quantize_pack(W, s, z, BITS, GROUP)
     q = O.unpack_rows(P, BITS, in_f)
     Wq = O.dequantize(q, s16.astype(np.float32), z8, GROUP)
-    O.linear_fwd(X, Wq); O.linear_bwd_dx(dY, Wq)
-    O.e2e_ds(dY, X, q, z8, GROUP)
+    product(O.linear_fwd, X, Wq); product(O.linear_bwd_dx, dY, Wq)
+    O.e2e_ds(dY, X, q, z8, GROUP)            # forms the weight gradient once more (a sixth product), then the group sums
     dt = time.perf_counter() - t0
     flops = 6 * 2 * toks * in_f * rows
-    return flops, dt, f"4096-wide linear, {rows} output rows x {toks} tokens, all steps of the path (w2g64)"
+    return flops, dt, f"4096-wide linear, {rows} output rows x {toks} tokens, all steps of the path (w2g64)", mm[0]
 
 
 def blas_threads():
@@ -331,47 +400,259 @@ def blas_threads():
         n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
         return max(n) if n else 1
     except Exception:
-        return os.cpu_count() or 1
+        return 1
+
+
+def oracle_threads(matmul_share):
+    """What the oracle really ran on: numpy hands its fp64 matrix products to the BLAS thread pool; everything else
+    (Eq. 1-5 element by element, the group sums, the bit packing with its Python loop over rows) is one thread."""
+    n = blas_threads()
+    return {"cores": n,
+            "threads": {"matrix products (BLAS pool)": n, "element-wise steps, group sums, bit packing": 1},
+            "time_share_of_matrix_products": round(matmul_share, 3)}
 
 
 def cpu_baseline(budget_s=15.0):
-    flops, dt, what = oracle_sample(0)
-    reps, total_f, total_t = 1, flops, dt
+    flops, dt, what, mm = oracle_sample(0)
+    reps, total_f, total_t, total_mm = 1, flops, dt, mm
     while total_t < budget_s and reps < 64:
-        f, t, _ = oracle_sample(reps)
-        total_f += f; total_t += t; reps += 1
-    return {"value": total_f / total_t / 1e12, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle",
-            "sample": f"{reps} x ({what}); {total_t:.1f} s of CPU time"}
+        f, t, _, m = oracle_sample(reps)
+        total_f += f; total_t += t; total_mm += m; reps += 1
+    out = {"value": total_f / total_t / 1e12, "unit": "TFLOP/s", "kind": "oracle",
+           "sample": f"{reps} x ({what}); {total_t:.1f} s of CPU time"}
+    out.update(oracle_threads(total_mm / total_t))
+    return out
 
 
 def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    times, flops = [], 0
+    times, flops, mm = [], 0, 0.0
     for i in range(args.warmup + args.steps):
-        f, t, what = oracle_sample(i)
+        f, t, what, m = oracle_sample(i)
         if i >= args.warmup:
-            times.append(t); flops = f
+            times.append(t); flops = f; mm += m
     ms = 1e3 * sum(times) / len(times)
     val = flops / (ms * 1e-3) / 1e12
+    base = {"value": val, "unit": "TFLOP/s", "kind": "oracle", "sample": what}
+    base.update(oracle_threads(mm / sum(times)))
     out = {"impl": "reference", "metric": "QLinear fwd+bwd TFLOP/s", "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
            "config": {"workload": WORKLOAD, "step": "bounded sample: " + what},
-           "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle", "sample": what},
+           "cpu_baseline": base,
            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out), flush=True)
 
 
-# ----------------------------------------------------------------------------- main
+# ----------------------------------------------------------------------------- reporting
 def summarise(timers):
     out = {}
     for name, pairs in timers.items():
         ms = [a.elapsed_time(b) for a, b in pairs]
         out[name] = {"launches": len(ms), "avg_ms": sum(ms) / len(ms), "total_ms": sum(ms)}
     return out
+
+
+def tensor_roofline(achieved_tflops, peaks, region_s, sm_mhz):
+    """A tensor-bound figure against every denominator there is.  `frac` uses the burst peak for a timed region of
+    under two seconds (the GPU has not settled under its power cap yet, like the burst measurement) and the
+    sustained one for a longer region; the other fractions are given beside it."""
+    burst, sust = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+    use_burst = region_s < 2.0
+    peak = burst if use_burst else sust
+    r = {"bound": "tensor", "achieved": achieved_tflops, "peak": peak, "unit": "TFLOP/s", "frac": achieved_tflops / peak,
+         "peak_source": f"{peaks['source']} ({'burst' if use_burst else 'sustained'}; timed region {region_s:.2f} s)",
+         "frac_vs_burst": achieved_tflops / burst, "frac_vs_sustained": achieved_tflops / sust,
+         "frac_vs_nominal": achieved_tflops / NOMINAL_PEAKS["bf16_tflops"],
+         "peaks": {"burst": burst, "sustained": sust, "nominal_dense_bf16": NOMINAL_PEAKS["bf16_tflops"]},
+         "sm_mhz": {"this_run_median": sm_mhz,
+                    "sustained_peak_measured_at": (peaks.get("clocks_under_load") or {}).get("sm_mhz_median")}}
+    return r
+
+
+def hbm_roofline(achieved_gbs, peaks):
+    return {"bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (copy)",
+            "frac_vs_nominal": achieved_gbs / NOMINAL_PEAKS["hbm_gbs"]}
+
+
+def class_report(wl, timers, steps, peaks, region_s, sm_mhz):
+    """Per call class: time per step, share, and the roofline figure of the class (contractions against the
+    tensor peaks; the three one-kernel streaming calls of the hand-off against the copy bandwidth: those are
+    per-call events around 10-50 us kernels inside the step, launch gaps included - the cold, back-to-back
+    figures are in the streaming leg)."""
+    kern = summarise(timers)
+    by_class = {}
+    for name, v in kern.items():
+        c = name.split("/")[0]
+        by_class[c] = by_class.get(c, 0.0) + v["total_ms"]
+    total = sum(by_class.values())
+    lin = LINEARS[wl.model]
+    n_elem = sum(l.in_features * l.out_features * l.count for l in lin)
+    n_grp = n_elem / wl.group
+    hbm_bytes = {"minmax_init": 2 * n_elem + 8 * n_grp,
+                 "quantize_pack": (2 + wl.bits / 8) * n_elem + 11 * n_grp,
+                 "unpack": (1 + wl.bits / 8) * n_elem}
+    classes = {}
+    for c, t in by_class.items():
+        sec = t * 1e-3 / steps
+        classes[c] = {"total_ms_per_step": t / steps, "share": t / total, "kernels_per_call": KERNELS_PER_CALL[c]}
+        if c in CONTRACTIONS:
+            tok = wl.t_ap if c.startswith("fakequant") else wl.t_e2e
+            fl = CONTRACTIONS[c] * 2 * tok * n_elem
+            classes[c]["roofline"] = tensor_roofline(fl / sec / 1e12, peaks, region_s, sm_mhz)
+        elif c in hbm_bytes:
+            classes[c]["roofline"] = hbm_roofline(hbm_bytes[c] / sec / 1e9, peaks)
+    return by_class, classes
+
+
+def mode_figures(wl, by_class, steps, world=1):
+    f_ap, f_e2e = wl.flops()
+    ap_ms = sum(by_class.get(c, 0.0) for c in ("fakequant_fwd", "fakequant_bwd")) / steps
+    qp_ms = sum(by_class.get(c, 0.0) for c in ("packed_fwd", "packed_bwd_dx", "packed_bwd_ds")) / steps
+    tok, tf = {}, {}
+    if wl.t_ap:
+        tok["block_ap"] = world * wl.t_ap / (ap_ms * 1e-3); tf["block_ap"] = f_ap / (ap_ms * 1e-3) / 1e12
+    if wl.t_e2e:
+        tok["e2e_qp"] = world * wl.t_e2e / (qp_ms * 1e-3); tf["e2e_qp"] = f_e2e / (qp_ms * 1e-3) / 1e12
+    return tok, tf
+
+
+def time_steps(wl, steps, warmup):
+    for _ in range(warmup):
+        wl.step()
+    torch.cuda.synchronize()
+    timers = {}
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        wl.step(timers)
+    t1.record()
+    torch.cuda.synchronize()
+    return t0.elapsed_time(t1) / steps, timers
+
+
+def run_extra_config(eqat, device, name, spec, peaks):
+    """One of the other workloads: the same path at its bit width, group size, model shapes and token counts."""
+    wl = BlockWorkload(eqat, device, seed=20240711, t_block_ap=spec["t_ap"], t_e2e=spec["t_e2e"], model=spec["model"],
+                       bits=spec["bits"], group=spec["group"], weight=spec["w"], handoff=False)
+    sampler = ClockSampler(device.index or 0)
+    sampler.start()
+    import datetime
+    t_begin = datetime.datetime.now()
+    ms, timers = time_steps(wl, spec["steps"], 3)
+    clocks = sampler.stop(t_begin, datetime.datetime.now())
+    if eqat.device_status() != (0, 0):
+        raise SystemExit(f"{name}: a kernel abandoned a wait")
+    region_s = ms * spec["steps"] * 1e-3
+    by_class, classes = class_report(wl, timers, spec["steps"], peaks, region_s, clocks["sm_mhz"])
+    tok, tf = mode_figures(wl, by_class, spec["steps"])
+    f_ap, f_e2e = wl.flops()
+    top = max(by_class, key=by_class.get)
+    out = {"workload": f"llama2-{spec['model']} decoder-block linears, w{spec['bits']}g{spec['group']}"
+                       + (f", Block-AP fwd+bwd @{spec['t_ap']} tok" if spec["t_ap"] else "")
+                       + (f", E2E-QP fwd/dX/ds @{spec['t_e2e']} tok" if spec["t_e2e"] else ""),
+           "steps": spec["steps"], "warmup": 3, "ms_per_step": ms, "value": (f_ap + f_e2e) / (ms * 1e-3) / 1e12,
+           "unit": "TFLOP/s", "tflops_by_mode": tf, "block_tokens_per_s": tok,
+           "dominant": dict(kernel_class=top, **classes[top].get("roofline", {})),
+           "kernel_classes": {c: {"ms_per_step": v["total_ms_per_step"], "share": v["share"],
+                                  **({"achieved": v["roofline"]["achieved"], "unit": v["roofline"]["unit"],
+                                      "frac_vs_burst": v["roofline"].get("frac_vs_burst"),
+                                      "frac_vs_sustained": v["roofline"].get("frac_vs_sustained")} if "roofline" in v else {})}
+                              for c, v in classes.items()},
+           "per_shape_ms": {k: v["avg_ms"] for k, v in summarise(timers).items()},
+           "clocks": clocks, "gpu_launches": wl.kernels_per_step * spec["steps"]}
+    del wl
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_streaming_leg(eqat, device, peaks, bits, group, shape=(11008, 4096), min_launches=56, min_bytes=640e6):
+    """The five streaming kernels, each timed cold: `n` distinct sets of inputs and outputs whose combined size is
+    several times the L2 (so no launch finds its operands or leaves its results in cache for the next one), at
+    least `min_launches` launches back to back between one pair of events.  Bytes counted are the algorithmic
+    ones (every input read once, every output written once)."""
+    out_f, in_f = shape
+    n_elem, ng = out_f * in_f, out_f * in_f // group
+    d = eqat.make_desc(bits, group, out_f, in_f)
+    bf = torch.bfloat16
+    g = torch.Generator(device=device); g.manual_seed(7)
+    per = {"fakequant_weight": (4 + 8 / group) * n_elem, "ste_bwd": (6 + 16 / group) * n_elem,
+           "minmax_init": (2 + 8 / group) * n_elem, "quantize_pack": (2 + bits / 8 + 11 / group) * n_elem,
+           "unpack": (1 + bits / 8) * n_elem}
+    res = {}
+    for name, nbytes in per.items():
+        n = max(4, int(np.ceil(min_bytes / nbytes)))
+        sets = []
+        for i in range(n):
+            W = (torch.randn(out_f, in_f, generator=g, device=device, dtype=torch.float32) * 0.02).to(bf)
+            S = dict(W=W, s=torch.empty(out_f, in_f // group, device=device), z=torch.empty(out_f, in_f // group, device=device))
+            eqat.eqat_minmax_init(d, W, S["s"], S["z"])
+            if name == "fakequant_weight":
+                S["What"] = torch.empty_like(W)
+                S["call"] = lambda S=S: eqat.eqat_fakequant_weight(d, S["W"], S["s"], S["z"], S["What"])
+            elif name == "ste_bwd":
+                S["G"] = (torch.randn(out_f, in_f, generator=g, device=device, dtype=torch.float32) * 1e-2).to(bf)
+                S["dW"] = torch.empty_like(W); S["ds"] = torch.empty_like(S["s"]); S["dz"] = torch.empty_like(S["s"])
+                S["call"] = lambda S=S: eqat.eqat_ste_bwd(d, S["G"], S["W"], S["s"], S["z"], S["dW"], S["ds"], S["dz"])
+            elif name == "minmax_init":
+                S["call"] = lambda S=S: eqat.eqat_minmax_init(d, S["W"], S["s"], S["z"])
+            else:
+                S["P"] = torch.empty(out_f, in_f * bits // 8, dtype=torch.uint8, device=device)
+                S["z8"] = torch.empty(out_f, in_f // group, dtype=torch.uint8, device=device)
+                S["s16"] = torch.empty(out_f, in_f // group, dtype=torch.float16, device=device)
+                eqat.eqat_quantize_pack(d, W, S["s"], S["z"], S["P"], S["z8"], S["s16"])
+                if name == "quantize_pack":
+                    S["call"] = lambda S=S: eqat.eqat_quantize_pack(d, S["W"], S["s"], S["z"], S["P"], S["z8"], S["s16"])
+                else:
+                    S["codes"] = torch.empty(out_f, in_f, dtype=torch.uint8, device=device)
+                    S["call"] = lambda S=S: eqat.eqat_unpack(d, S["P"], S["codes"])
+                    del S["W"]
+            sets.append(S)
+        rounds = int(np.ceil(min_launches / n))
+        for S in sets:
+            S["call"]()                                   # warm-up: one pass over every set
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(rounds):
+            for S in sets:
+                S["call"]()
+        e1.record()
+        torch.cuda.synchronize()
+        launches = rounds * n
+        us = e0.elapsed_time(e1) * 1e3 / launches
+        r = hbm_roofline(nbytes / us / 1e3, peaks)
+        r.update({"us_per_launch": us, "launches": launches, "distinct_buffer_sets": n,
+                  "bytes_per_launch": nbytes, "bytes_touched_per_round": n * nbytes})
+        res[name] = r
+        del sets
+        torch.cuda.empty_cache()
+    return {"shape": f"{out_f} x {in_f}", "bits": bits, "group": group,
+            "method": "distinct input/output sets per launch (combined > 4 x L2), all launches between one pair of CUDA events",
+            "kernels": res}
+
+
+# ----------------------------------------------------------------------------- main
+def spawn_ranks(args):
+    """`--gpus N` without a launcher: start N copies of this script, one per GPU, with the environment
+    torch.distributed's launcher would have given them; rank 0's line is the job's line."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(args.gpus):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(args.gpus), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
+    rc = 0
+    for pr in procs:
+        rc = max(rc, abs(pr.wait()))
+    return rc
 
 
 def run_ours(args):
@@ -387,13 +668,14 @@ def run_ours(args):
     build_library()
     from paper_2407_11062_b200 import binding as eqat
     peaks = load_peaks()
+    warmup = max(args.warmup, 3)
 
     import datetime
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
     wl = BlockWorkload(eqat, device, seed=20240711 + rank)     # each rank: its own token batch (weak scaling)
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(warmup):
         wl.step()
     torch.cuda.synchronize()
     timers = {}
@@ -415,7 +697,7 @@ def run_ours(args):
 
     # end-to-end leg: host buffers in, gradients out, copies inside the timed region
     stage = HostStaging(wl)
-    e2e_steps = max(1, min(args.steps, 3))
+    e2e_steps = max(1, args.steps)
     stage.step(); torch.cuda.synchronize(); barrier()
     t0.record()
     for _ in range(e2e_steps):
@@ -423,66 +705,53 @@ def run_ours(args):
     t1.record()
     torch.cuda.synchronize(); barrier()
     e2e_ms = max_over_ranks(t0.elapsed_time(t1) / e2e_steps, device)
+    wl_h2d, wl_d2h = stage.h2d, stage.d2h
+    del stage
 
-    f_ap, f_e2e = step_flops()
+    f_ap, f_e2e = wl.flops()
     flops = (f_ap + f_e2e) * world
     if rank == 0:
-        kern = summarise(timers)
-        by_class = {}
-        for name, v in kern.items():
-            c = name.split("/")[0]
-            by_class.setdefault(c, 0.0)
-            by_class[c] += v["total_ms"]
+        region_s = ms * args.steps * 1e-3
+        by_class, classes = class_report(wl, timers, args.steps, peaks, region_s, clocks["sm_mhz"])
         top_class = max(by_class, key=by_class.get)
-        # roofline of the dominant kernel (each packed_* call is exactly one kernel launch)
-        t_tok = {"packed_fwd": T_E2E, "packed_bwd_dx": T_E2E, "packed_bwd_ds": T_E2E}
         roof = None
-        if top_class in t_tok:
-            tot_f = sum(2 * T_E2E * l.in_features * l.out_features * l.count for l in LINEARS["7b"]) * args.steps
-            tot_ms = by_class[top_class]
-            ach = tot_f / (tot_ms * 1e-3) / 1e12
-            peak = peaks["bf16_tflops_sustained"]
-            roof = {"kernel": "gemm_kernel (" + top_class + ")", "bound": "tensor", "achieved": ach, "peak": peak,
-                    "unit": "TFLOP/s", "frac": ach / peak, "peak_source": peaks["source"] + " (sustained)", "traffic": traffic_per_launch(top_class),
-                    "traffic_unit": "DRAM bytes per launch (ncu, launch-weighted mean over the class)",
-                    "algorithmic_bytes": sum((T_E2E * (l.in_features + l.out_features) * 2
-                                              + l.in_features * l.out_features * BITS // 8) * l.count
-                                             for l in LINEARS["7b"]) / sum(l.count for l in LINEARS["7b"])}
-        classes = {c: {"total_ms_per_step": t / args.steps, "share": t / sum(by_class.values())} for c, t in by_class.items()}
-        # every class that is exactly one kernel launch per call also gets its own roofline figure:
-        # the contractions against the sustained bf16 peak, the streaming kernels against the copy bandwidth
-        n_elem = sum(l.in_features * l.out_features * l.count for l in LINEARS["7b"])
-        n_grp = n_elem / GROUP
-        hbm_bytes = {"minmax_init": 2 * n_elem + 8 * n_grp,
-                     "quantize_pack": (2 + BITS / 8) * n_elem + 11 * n_grp,
-                     "unpack": (1 + BITS / 8) * n_elem}
-        e2e_flops = sum(2 * T_E2E * l.in_features * l.out_features * l.count for l in LINEARS["7b"])
-        for c, t in by_class.items():
-            sec = t * 1e-3 / args.steps
-            if c in hbm_bytes:
-                ach = hbm_bytes[c] / sec / 1e9
-                classes[c]["roofline"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                          "frac": ach / peaks["hbm_gbs"]}
-            elif c in t_tok:
-                ach = e2e_flops / sec / 1e12
-                classes[c]["roofline"] = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
-                                          "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
-                                          "traffic": traffic_per_launch(c)}
-        out = {"metric": "QLinear fwd+bwd TFLOP/s", "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": world,
-               "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        if top_class in CONTRACTIONS:
+            roof = dict(kernel="gemm_kernel (" + top_class + ")", **classes[top_class]["roofline"])
+            roof["traffic"] = traffic_per_launch(top_class)
+            roof["traffic_unit"] = "DRAM bytes per launch (ncu, launch-weighted mean over the class)"
+            lin = LINEARS["7b"]
+            roof["algorithmic_bytes"] = sum((T_E2E * (l.in_features + l.out_features) * 2
+                                             + l.in_features * l.out_features * BITS // 8) * l.count for l in lin) / sum(l.count for l in lin)
+        for c in ("packed_fwd", "packed_bwd_dx", "packed_bwd_ds"):
+            if c in classes:
+                classes[c]["roofline"]["traffic"] = traffic_per_launch(c)
+        tok, tf = mode_figures(wl, by_class, args.steps, world)
+        value = flops / (ms * 1e-3) / 1e12
+        out = {"metric": "QLinear fwd+bwd TFLOP/s", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+               "steps": args.steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                "config": {"workload": WORKLOAD, "bits": BITS, "group": GROUP, "tokens_block_ap": T_BLOCK_AP, "tokens_e2e_qp": T_E2E,
                           "l2": "inputs larger than L2 (working set > 2 GB per shape, weights per linear)"},
-               "pct_of_bf16_peak": 100.0 * flops / world / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
-               "block_tokens_per_s": {"block_ap": None, "e2e_qp": None},
+               "pct_of_bf16_peak": {"vs_burst": 100.0 * value / world / peaks["bf16_tflops"],
+                                    "vs_sustained": 100.0 * value / world / peaks["bf16_tflops_sustained"],
+                                    "vs_nominal_dense": 100.0 * value / world / NOMINAL_PEAKS["bf16_tflops"]},
+               "block_tokens_per_s": tok, "tflops_by_mode": tf,
                "roofline": roof, "kernel_classes": classes, "clocks": clocks,
-               "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
-                       "h2d_bytes_per_step": stage.h2d, "d2h_bytes_per_step": stage.d2h},
+               "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms, "steps": e2e_steps,
+                       "h2d_bytes_per_step": wl_h2d, "d2h_bytes_per_step": wl_d2h},
                "gpu_launches": wl.kernels_per_step * args.steps}
-        ap_ms = sum(by_class.get(c, 0.0) for c in ("fakequant_fwd", "fakequant_bwd")) / args.steps
-        qp_ms = sum(by_class.get(c, 0.0) for c in ("packed_fwd", "packed_bwd_dx", "packed_bwd_ds")) / args.steps
-        out["block_tokens_per_s"] = {"block_ap": world * T_BLOCK_AP / (ap_ms * 1e-3), "e2e_qp": world * T_E2E / (qp_ms * 1e-3)}
-        out["tflops_by_mode"] = {"block_ap": f_ap / (ap_ms * 1e-3) / 1e12, "e2e_qp": f_e2e / (qp_ms * 1e-3) / 1e12}
+    del wl
+    torch.cuda.empty_cache()
+    if rank == 0:
+        if world == 1 and not args.headline_only:
+            # the other workloads and the cold streaming figures (one GPU is enough for them: the path is replicated)
+            out["configs"] = {name: run_extra_config(eqat, device, name, spec, peaks) for name, spec in EXTRA_CONFIGS.items()}
+            out["streaming"] = {"w2g64": run_streaming_leg(eqat, device, peaks, 2, 64),
+                                "w4g128": run_streaming_leg(eqat, device, peaks, 4, 128)}
+            alias = {"fakequant_weight": "fakequant_weight", "ste_bwd": "ste_bwd", "minmax_init": "minmax_init_cold",
+                     "quantize_pack": "quantize_pack_cold", "unpack": "unpack_cold"}
+            for k, v in out["streaming"]["w2g64"]["kernels"].items():
+                out["kernel_classes"][alias[k]] = {"roofline": v, "timed": "streaming leg (cold, back to back), not part of the step"}
         if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline()
         print(json.dumps(out), flush=True)
@@ -492,15 +761,19 @@ def run_ours(args):
 
 
 def run_kernel_case(args):
-    """One call class on one linear shape, a few launches: the small case used for ncu captures."""
+    """One linear shape of one workload, a few steps: the small case used for ncu captures."""
     torch.cuda.set_device(0)
     from paper_2407_11062_b200.build import build_library
     build_library()
     from paper_2407_11062_b200 import binding as eqat
-    wl = BlockWorkload(eqat, torch.device("cuda", 0), seed=1, t_block_ap=args.case_tokens, t_e2e=args.case_tokens)
+    mode = args.case_mode
+    wl = BlockWorkload(eqat, torch.device("cuda", 0), seed=1, model=args.case_model, bits=args.case_bits, group=args.case_group,
+                       t_block_ap=args.case_tokens if mode in ("both", "block_ap") else 0,
+                       t_e2e=args.case_tokens if mode in ("both", "e2e_qp") else 0, handoff=(mode == "both"))
     wl.layers = [L for L in wl.layers if L["shape"] == args.case_shape][:1]
+    assert wl.layers, f"no linear named {args.case_shape} in model {args.case_model}"
     for _ in range(2):
-        wl.step()                       # fills s, z, packed codes
+        wl.step()
     torch.cuda.synchronize()
     timers = {}
     for _ in range(args.case_iters):
@@ -508,6 +781,19 @@ def run_kernel_case(args):
     torch.cuda.synchronize()
     assert eqat.device_status() == (0, 0)
     print(json.dumps({k: v for k, v in summarise(timers).items()}), flush=True)
+
+
+def run_streaming_case(args):
+    """The cold streaming leg alone (for profiler captures and kernel work)."""
+    torch.cuda.set_device(0)
+    from paper_2407_11062_b200.build import build_library
+    build_library()
+    from paper_2407_11062_b200 import binding as eqat
+    lin = next(l for l in LINEARS[args.case_model] if l.name == args.case_shape)
+    r = run_streaming_leg(eqat, torch.device("cuda", 0), load_peaks(), args.case_bits, args.case_group,
+                          (lin.out_features, lin.in_features), min_launches=args.case_iters * 4, min_bytes=640e6)
+    assert eqat.device_status() == (0, 0)
+    print(json.dumps(r), flush=True)
 
 
 def run_decode_case(args):
@@ -564,19 +850,29 @@ def main():
     ap.add_argument("--kernel-case", action="store_true", help="run one linear shape a few times (for profilers)")
     ap.add_argument("--decode-case", action="store_true",
                     help="time the few-token packed forward on the block's linear shapes (uses --case-iters)")
-    ap.add_argument("--case-shape", default="qkvo", choices=[l.name for l in LINEARS["7b"]])
+    ap.add_argument("--streaming-case", action="store_true", help="the cold streaming-kernel leg alone")
+    ap.add_argument("--case-model", default="7b", choices=sorted(LINEARS))
+    ap.add_argument("--case-shape", default="qkvo")
     ap.add_argument("--case-tokens", type=int, default=16384)
+    ap.add_argument("--case-bits", type=int, default=BITS)
+    ap.add_argument("--case-group", type=int, default=GROUP)
+    ap.add_argument("--case-mode", default="both", choices=["both", "block_ap", "e2e_qp"])
     ap.add_argument("--case-iters", type=int, default=2)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true", help="skip the other workloads and the streaming leg")
     args = ap.parse_args()
     if args.kernel_case:
         run_kernel_case(args)
     elif args.decode_case:
         run_decode_case(args)
+    elif args.streaming_case:
+        run_streaming_case(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -78,8 +78,47 @@ def test_reference_arm_line_and_idle_ranks():
     assert line["impl"] == "reference" and line["unit"] == "TFLOP/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["config"]["workload"] == bench.WORKLOAD
+    assert line["cpu_baseline"]["cores"] >= 1 and line["cpu_baseline"]["threads"]["element-wise steps, group sums, bit packing"] == 1
+    assert 0.0 < line["cpu_baseline"]["time_share_of_matrix_products"] < 1.0
     # under torchrun only rank 0 works; the others exit 0 silently
     env1 = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
     out1 = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
                            "--warmup", "0", "--gpus", "2"], capture_output=True, text=True, env=env1, timeout=600)
     assert out1.returncode == 0 and out1.stdout.strip() == ""
+
+
+def test_gpus_flag_spawns_the_ranks_itself():
+    """`bench.py --gpus 2` with no launcher around it starts two ranks (here on the CPU, through the reference arm):
+    exactly one line comes back, rank 0's, and it says n_gpus 2."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                          "--warmup", "0", "--gpus", "2"], capture_output=True, text=True, env=env, timeout=600)
+    assert out.returncode == 0, out.stderr
+    lines = [l for l in out.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
+
+
+def test_rooflines_carry_every_denominator():
+    peaks = bench.load_peaks()
+    r = bench.tensor_roofline(1000.0, peaks, 0.4, 1500.0)
+    assert r["peak"] == peaks["bf16_tflops"] and "burst" in r["peak_source"]            # a short timed region
+    assert r["frac_vs_burst"] == pytest.approx(1000.0 / peaks["bf16_tflops"])
+    assert r["frac_vs_sustained"] == pytest.approx(1000.0 / peaks["bf16_tflops_sustained"])
+    assert r["frac_vs_nominal"] == pytest.approx(1000.0 / 2250.0)
+    assert bench.tensor_roofline(1000.0, peaks, 5.0, 1400.0)["peak"] == peaks["bf16_tflops_sustained"]
+    h = bench.hbm_roofline(4000.0, peaks)
+    assert h["frac"] == pytest.approx(4000.0 / peaks["hbm_gbs"]) and h["frac_vs_nominal"] == pytest.approx(0.5)
+
+
+def test_extra_configs_match_the_workload_table():
+    from workloads import CONFIGS
+    by_name = {c.name: c for c in CONFIGS}
+    for name, spec in bench.EXTRA_CONFIGS.items():
+        c = by_name[name]
+        assert (spec["bits"], spec["group"]) == (c.bits, c.group)
+        assert c.linears == bench.LINEARS[spec["model"]]
+        assert {spec["t_ap"], spec["t_e2e"]} - {0} == {c.tokens}
+        assert (spec["t_ap"] > 0) == ("block_ap" in c.modes) and (spec["t_e2e"] > 0) == ("e2e_qp" in c.modes)
+        assert spec["w"] == (c.weight_dist, c.weight_scale, c.outlier_frac)

@@ -6,7 +6,9 @@ compared on a seeded sample it can compute directly:
   * Y on 192 token rows x 256 output rows, dX on 192 token rows x 4 column groups,
   * dW / ds / dz (and the packed ds) on 96 output rows x all columns,
   * codes, packed bytes, zero points and step sizes bit-exactly on those rows,
-and whole-tensor identities that hold at any size tie the rest together:
+each sampled block by its norm and element by element (helpers.contraction_bound); a second, dense block
+always covers the last row-tile and the last column-tile of Y and dX (last 256 tokens x last 256 outputs /
+inputs), where a ragged edge would show; and whole-tensor identities that hold at any size tie the rest together:
   <dY, Y> = <dX, X>  (adjoint),  sum s*ds = <dY, Y>  (Y is linear in s).
 The E2E-QP cases also push the first one and four tokens through the forward alone (decoding).
 """
@@ -14,7 +16,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import TOL, bits_to_torch, f32, rel_err, torch_to_f64
+from helpers import TOL, assert_elementwise, bits_to_torch, contraction_bound, f32, rel_err, torch_to_f64
 from oracle import eqat_oracle as O
 from workloads import CONFIGS, activations_for, get_config, tensor_seed, weight_for
 
@@ -59,6 +61,17 @@ def inner_product_tol(dY, Y, dX, X) -> float:
     def scale(u, v):
         return np.sqrt(dot64(u, u) * dot64(v, v) / u.numel())
     return TOL * (scale(dY, Y) + scale(dX, X))
+
+
+def check_block(got, A, B_rows, what):
+    """got ~ A @ B_rows.T for the oracle's operands (fp64): norm criterion and element-wise bound."""
+    ref = O.linear_fwd(A, B_rows)
+    assert rel_err(torch_to_f64(got), ref) <= TOL, what
+    bound = contraction_bound(ref, O.linear_fwd(np.abs(A), np.abs(B_rows)), O.linear_fwd(A ** 2, B_rows ** 2))
+    assert_elementwise(torch_to_f64(got), ref, bound, what)
+
+
+CORNER = 256
 
 
 CASES = [(c.name, l.name, mode) for c in CONFIGS[1:] for l in c.linears for mode in c.modes]
@@ -107,12 +120,21 @@ def test_full_size(eqat, cfg_name, lin_name, mode):
         torch.cuda.synchronize()
         What_rows = O.fake_quant_weight(W_rows, s_rows, z_rows, bits, g)
         assert rel_err(torch_to_f64(What[rows_all]), What_rows) <= TOL
-        assert rel_err(torch_to_f64(Y[tok][:, rows_y]), O.linear_fwd(X_tok, What_rows[iy])) <= TOL
+        check_block(Y[tok][:, rows_y], X_tok, What_rows[iy], "Y sample")
         What_cols = O.fake_quant_weight(f32(Wb[:, cols]), s_cols, z_cols, bits, g)
-        assert rel_err(torch_to_f64(dX[tok][:, cols]), O.linear_bwd_dx(dY_tok, What_cols)) <= TOL
+        check_block(dX[tok][:, cols], dY_tok, What_cols.T, "dX sample")
+        # the last row-tile and column-tile of both outputs, densely
+        s_last, z_last = O.minmax_init(f32(Wb[-CORNER:]), bits, g)
+        check_block(Y[-CORNER:, -CORNER:], f32(Xb[-CORNER:]), O.fake_quant_weight(f32(Wb[-CORNER:]), s_last, z_last, bits, g),
+                    "Y corner")
+        s_lc, z_lc = O.minmax_init(f32(Wb[:, -CORNER:]), bits, g)
+        check_block(dX[-CORNER:, -CORNER:], f32(dYb[-CORNER:]), O.fake_quant_weight(f32(Wb[:, -CORNER:]), s_lc, z_lc, bits, g).T,
+                    "dX corner")
         G = O.weight_grad(f32(dYb[:, rows_g]), f32(Xb))
         dW_o, ds_o, dz_o = O.ste_bwd(G, W_rows[ig], s_rows[ig], z_rows[ig], bits, g)
         assert rel_err(torch_to_f64(dW[rows_g]), dW_o) <= TOL
+        absG = O.weight_grad(np.abs(f32(dYb[:, rows_g])), np.abs(f32(Xb)))
+        assert_elementwise(torch_to_f64(dW[rows_g]), dW_o, contraction_bound(dW_o, absG, 0.0, 0), "dW sample")
         assert rel_err(torch_to_f64(ds[rows_g]), ds_o) <= TOL
         if np.linalg.norm(dz_o) > 0:
             assert rel_err(torch_to_f64(dz[rows_g]), dz_o) <= TOL
@@ -139,10 +161,18 @@ def test_full_size(eqat, cfg_name, lin_name, mode):
         eqat.qlinear_packed_bwd_ds(d, Xd, dYd, P, z8, s16, ds, dz)
         torch.cuda.synchronize()
         What_rows = O.dequantize(q_rows, s16_rows.astype(np.float32), z8_rows, g)
-        assert rel_err(torch_to_f64(Y[tok][:, rows_y]), O.linear_fwd(X_tok, What_rows[iy])) <= TOL
+        check_block(Y[tok][:, rows_y], X_tok, What_rows[iy], "Y sample")
         q_cols, _, _ = O.quantize_codes(f32(Wb[:, cols]), s_cols, z_cols, bits, g)
         What_cols = O.dequantize(q_cols, s_cols.astype(np.float16).astype(np.float32), z_cols, g)
-        assert rel_err(torch_to_f64(dX[tok][:, cols]), O.linear_bwd_dx(dY_tok, What_cols)) <= TOL
+        check_block(dX[tok][:, cols], dY_tok, What_cols.T, "dX sample")
+        # the last row-tile and column-tile of both outputs, densely (codes, fp16 step sizes and zero points of
+        # those rows / columns from the oracle's own hand-off)
+        def handoff(Wpart):
+            s_p, z_p = O.minmax_init(Wpart, bits, g)
+            P_p, z8_p, s16_p = O.quantize_pack(Wpart, s_p, z_p, bits, g)
+            return O.dequantize(O.unpack_rows(P_p, bits, Wpart.shape[1]), s16_p.astype(np.float32), z8_p, g)
+        check_block(Y[-CORNER:, -CORNER:], f32(Xb[-CORNER:]), handoff(f32(Wb[-CORNER:])), "Y corner")
+        check_block(dX[-CORNER:, -CORNER:], f32(dYb[-CORNER:]), handoff(f32(Wb[:, -CORNER:])).T, "dX corner")
         dYg, Xf = f32(dYb[:, rows_g]), f32(Xb)
         assert rel_err(torch_to_f64(ds[rows_g]), O.e2e_ds(dYg, Xf, q_rows[ig], z8_rows[ig], g)) <= TOL
         assert rel_err(torch_to_f64(dz[rows_g]), O.e2e_dz(dYg, Xf, s16_rows[ig].astype(np.float32), g)) <= TOL
