@@ -38,8 +38,8 @@
  * multiple of 32 dividing in_features (e.g. group == in_features, one group
  * per row) for the element-wise and codec entry points; in_features a
  * multiple of 128.  The GEMM entry points also need out_features a multiple
- * of 64; tokens may be any positive number.  The packed-weight GEMMs need
- * group in {64,128,256}.
+ * of 64; tokens may be any positive number.  The packed-weight GEMMs take
+ * group in {32,64,128,256} or group == in_features (channel-wise).
  */
 #ifndef EQAT_H_
 #define EQAT_H_
@@ -75,8 +75,17 @@ typedef struct {
   int32_t dz_mode;            /* clamped-branch value of d w_hat / d z:
                                  0 = -s (derivative of Eq. 2 at a saturated code),
                                  1 = -1 (Eq. 4 as printed)                            */
-  int32_t reserved;           /* must be 0                                            */
+  int32_t zero_point_format;  /* how the packed-weight (E2E-QP) entry points read their
+                                 zero points: EQAT_ZP_U8 or EQAT_ZP_FP16; must be
+                                 EQAT_ZP_U8 (0) for every other entry point           */
 } eqat_desc;
+
+/* Zero points of the packed-weight entry points.  EQAT_ZP_U8: one byte per group,
+ * the frozen N-bit integers of the hand-off.  EQAT_ZP_FP16: one fp16 value per
+ * group, used as it is (not rounded): the variant of Sec. 3.3 that also trains z
+ * and therefore keeps it in FP16 (2 + 32/64 = 2.50 bits per weight at w2g64 in
+ * the paper's table of E2E-QP variants). */
+enum { EQAT_ZP_U8 = 0, EQAT_ZP_FP16 = 1 };
 
 /* Operations that need caller-provided scratch memory (eqat_workspace_bytes). */
 enum { EQAT_OP_FAKEQUANT_BWD = 1, EQAT_OP_PACKED_BWD_DS = 2 };
@@ -203,18 +212,21 @@ int eqat_unpack_zeros(const eqat_desc* desc, const uint8_t* z_packed, uint8_t* z
 
 /* ------------------------------------------------------------------ E2E-QP */
 
+/* In the three calls below `z` is [out,in/g] uint8, or [out,in/g] fp16 when
+ * desc->zero_point_format is EQAT_ZP_FP16. */
+
 /* Y = X * ((W_int - z) * s)^T, the packed codes expanded tile by tile in
  * shared memory inside the GEMM (Eq. 2; Sec. 3.3).  With one to four tokens
- * (decoding) a matrix-vector kernel streams the packed weight instead and
- * keeps (W_int - z) * s in fp32.
- *   X [T,in] bf16, Wq_packed, s16, z8 (in)   Y [T,out] bf16 (out) */
+ * (decoding) and groups of at least 64 a matrix-vector kernel streams the
+ * packed weight instead and keeps (W_int - z) * s in fp32.
+ *   X [T,in] bf16, Wq_packed, s16, z (in)   Y [T,out] bf16 (out) */
 int qlinear_packed_fwd(const eqat_desc* desc, const eqat_bf16* X, const uint8_t* Wq_packed,
-                       const eqat_fp16* s16, const uint8_t* z8, eqat_bf16* Y, void* stream);
+                       const eqat_fp16* s16, const void* z, eqat_bf16* Y, void* stream);
 
 /* dX = dY * ((W_int - z) * s).
- *   dY [T,out] bf16, Wq_packed, s16, z8 (in)   dX [T,in] bf16 (out) */
+ *   dY [T,out] bf16, Wq_packed, s16, z (in)   dX [T,in] bf16 (out) */
 int qlinear_packed_bwd_dx(const eqat_desc* desc, const eqat_bf16* dY, const uint8_t* Wq_packed,
-                          const eqat_fp16* s16, const uint8_t* z8, eqat_bf16* dX, void* stream);
+                          const eqat_fp16* s16, const void* z, eqat_bf16* dX, void* stream);
 
 /* Step-size gradient (Sec. 3.3, d w_hat/d s = w_q - z):
  *   ds[o,g] = sum_{j in g} (sum_t dY[t,o] X[t,j]) * (W_int[o,j] - z[o,g]),
@@ -223,10 +235,12 @@ int qlinear_packed_bwd_dx(const eqat_desc* desc, const eqat_bf16* dY, const uint
  * zero-point gradient of the same layer (the Sec. 3.3 variant that trains z),
  * dz[o,g] = -s[o,g] * sum_{j in g} G[o,j]; s16 is then required, else it may be
  * NULL.  Needs eqat_workspace_bytes(desc, EQAT_OP_PACKED_BWD_DS) bytes of
- * scratch (0 for every supported shape: workspace may then be NULL).
- *   X [T,in], dY [T,out] bf16, Wq_packed, z8 (in)   ds [out,in/g] fp32 (out) */
+ * scratch: 0 for groups of up to 256 elements (workspace may then be NULL);
+ * with one group per row the sums of the 256-column tiles of a row pass through
+ * it and are added up in a fixed order.
+ *   X [T,in], dY [T,out] bf16, Wq_packed, z (in)   ds [out,in/g] fp32 (out) */
 int qlinear_packed_bwd_ds(const eqat_desc* desc, const eqat_bf16* X, const eqat_bf16* dY,
-                          const uint8_t* Wq_packed, const uint8_t* z8, const eqat_fp16* s16,
+                          const uint8_t* Wq_packed, const void* z, const eqat_fp16* s16,
                           float* ds, float* dz, void* workspace, size_t workspace_bytes, void* stream);
 
 #ifdef __cplusplus

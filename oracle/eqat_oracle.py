@@ -85,11 +85,19 @@ def quantize_codes(W, s, z, bits: int, group: int):
     return q, r, p
 
 
-def dequantize(q, s, z, group: int) -> np.ndarray:
+def _zero_point(z, real_zero_point: bool) -> np.ndarray:
+    """The zero point Eq. 2 subtracts.  In Block-AP and in E2E-QP with frozen zero points it is the integer that is
+    stored in N bits (``round_zero_point``).  The E2E-QP variants that train z (Sec. 3.3 and the table of E2E-QP
+    trainable parameters, where z is promoted to FP16: 2.50 average bits at w2g64) run no quantiser, only Eq. 2, so
+    their z enters as the real number it is: ``real_zero_point=True`` takes it unrounded."""
+    return np.asarray(z, np.float64) if real_zero_point else round_zero_point(z)
+
+
+def dequantize(q, s, z, group: int, real_zero_point: bool = False) -> np.ndarray:
     """Eq. 2:  W_hat = (W_int - z) * s, in float64."""
     q64 = np.asarray(q, np.float64)
     s64 = _per_element(np.asarray(s, np.float64), group)
-    z64 = _per_element(round_zero_point(z), group)
+    z64 = _per_element(_zero_point(z, real_zero_point), group)
     return (q64 - z64) * s64
 
 
@@ -156,12 +164,12 @@ def ste_bwd(G, W, s, z, bits: int, group: int, dz_mode: int = 0):
     return G64 * dw_dw, _group_sum(G64 * dw_ds, group), _group_sum(G64 * dw_dz, group)
 
 
-def e2e_ds(dY, X, q, z, group: int) -> np.ndarray:
+def e2e_ds(dY, X, q, z, group: int, real_zero_point: bool = False) -> np.ndarray:
     """E2E-QP step-size gradient (Sec. 3.3: d w_hat / d s = w_q - z):
     ds[o,g] = sum_{j in g} (sum_t dY[t,o] X[t,j]) * (q[o,j] - z[o,g]).
     The full weight gradient is materialised first, then multiplied and summed."""
     G = weight_grad(dY, X)
-    z64 = _per_element(round_zero_point(z), group)
+    z64 = _per_element(_zero_point(z, real_zero_point), group)
     return _group_sum(G * (np.asarray(q, np.float64) - z64), group)
 
 

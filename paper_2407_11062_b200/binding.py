@@ -20,6 +20,7 @@ EQAT_OK = 0
 EQAT_ERR_NULL, EQAT_ERR_SHAPE, EQAT_ERR_ALIGN, EQAT_ERR_UNSUPPORTED = -1, -2, -3, -4
 EQAT_ERR_WORKSPACE, EQAT_ERR_CUDA, EQAT_ERR_TIMEOUT = -5, -6, -7
 EQAT_OP_FAKEQUANT_BWD, EQAT_OP_PACKED_BWD_DS = 1, 2
+EQAT_ZP_U8, EQAT_ZP_FP16 = 0, 1
 
 
 class EqatError(RuntimeError):
@@ -30,7 +31,7 @@ class EqatError(RuntimeError):
 
 class eqat_desc(Structure):
     _fields_ = [("bits", c_int32), ("group", c_int32), ("out_features", c_int32), ("in_features", c_int32),
-                ("tokens", c_int64), ("dz_mode", c_int32), ("reserved", c_int32)]
+                ("tokens", c_int64), ("dz_mode", c_int32), ("zero_point_format", c_int32)]
 
 
 def _load():
@@ -74,8 +75,9 @@ def status_string(status: int) -> str:
     return lib.eqat_status_string(int(status)).decode()
 
 
-def make_desc(bits, group, out_features, in_features, tokens=0, dz_mode=0) -> eqat_desc:
-    return eqat_desc(int(bits), int(group), int(out_features), int(in_features), int(tokens), int(dz_mode), 0)
+def make_desc(bits, group, out_features, in_features, tokens=0, dz_mode=0, zero_point_format=EQAT_ZP_U8) -> eqat_desc:
+    return eqat_desc(int(bits), int(group), int(out_features), int(in_features), int(tokens), int(dz_mode),
+                     int(zero_point_format))
 
 
 def _ptr(t):

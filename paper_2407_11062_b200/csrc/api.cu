@@ -18,7 +18,7 @@ inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 // Geometry every entry point shares.
 int check_weight_desc(const eqat_desc* d) {
   if (d == nullptr) return EQAT_ERR_NULL;
-  if (d->reserved != 0) return EQAT_ERR_UNSUPPORTED;
+  if (d->zero_point_format != EQAT_ZP_U8 && d->zero_point_format != EQAT_ZP_FP16) return EQAT_ERR_UNSUPPORTED;
   if (d->bits < 2 || d->bits > 4) return EQAT_ERR_UNSUPPORTED;
   if (d->dz_mode != 0 && d->dz_mode != 1) return EQAT_ERR_UNSUPPORTED;
   if (d->out_features <= 0 || d->in_features <= 0 || d->group <= 0) return EQAT_ERR_SHAPE;
@@ -30,12 +30,20 @@ int check_weight_desc(const eqat_desc* d) {
   return EQAT_OK;
 }
 
-int check_gemm_desc(const eqat_desc* d, bool packed) {
+// Entry points that read no packed zero points take the default format only.
+int check_plain_desc(const eqat_desc* d) {
   const int rc = check_weight_desc(d);
+  if (rc != EQAT_OK) return rc;
+  return d->zero_point_format == EQAT_ZP_U8 ? EQAT_OK : EQAT_ERR_UNSUPPORTED;
+}
+
+int check_gemm_desc(const eqat_desc* d, bool packed) {
+  const int rc = packed ? check_weight_desc(d) : check_plain_desc(d);
   if (rc != EQAT_OK) return rc;
   if (d->tokens <= 0 || d->tokens > (int64_t)1 << 30) return EQAT_ERR_SHAPE;
   if (d->out_features % 64 != 0) return EQAT_ERR_SHAPE;
-  if (packed && !(d->group == 64 || d->group == 128 || d->group == 256)) return EQAT_ERR_UNSUPPORTED;
+  // packed kernels: a group is a power of two up to 256, or the whole row
+  if (packed && d->group > 256 && d->group != d->in_features) return EQAT_ERR_UNSUPPORTED;
   return EQAT_OK;
 }
 
@@ -86,7 +94,7 @@ size_t eqat_workspace_bytes(const eqat_desc* d, int op) {
   }
   if (op == EQAT_OP_PACKED_BWD_DS) {
     if (check_gemm_desc(d, true) != EQAT_OK) return (size_t)-1;
-    return 0;
+    return packed_ds_workspace_bytes(*d);
   }
   return (size_t)-1;
 }
@@ -109,14 +117,14 @@ int eqat_selftest_wait_expiry(int which, void* stream) {
 }
 
 int eqat_minmax_init(const eqat_desc* d, const eqat_bf16* W, float* s, float* z, void* stream) {
-  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_plain_desc(d));
   EQAT_TRY(check_ptrs(W, s, z));
   return launch_minmax(*d, W, s, z, as_stream(stream));
 }
 
 int eqat_fakequant_weight(const eqat_desc* d, const eqat_bf16* W, const float* s, const float* z, eqat_bf16* W_hat,
                           void* stream) {
-  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_plain_desc(d));
   EQAT_TRY(check_ptrs(W, s, z, W_hat));
   return launch_fakequant(*d, W, s, z, W_hat, as_stream(stream));
 }
@@ -131,7 +139,7 @@ int qlinear_fakequant_fwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf1
 
 int eqat_ste_bwd(const eqat_desc* d, const eqat_bf16* dW_hat, const eqat_bf16* W, const float* s, const float* z,
                  eqat_bf16* dW, float* ds, float* dz, void* stream) {
-  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_plain_desc(d));
   EQAT_TRY(check_ptrs(dW_hat, W, s, z, dW, ds));
   if (dz != nullptr && !aligned16(dz)) return EQAT_ERR_ALIGN;
   return launch_ste_bwd(*d, dW_hat, W, s, z, dW, ds, dz, as_stream(stream));
@@ -162,62 +170,63 @@ int qlinear_fakequant_bwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf1
 
 int eqat_quantize_pack(const eqat_desc* d, const eqat_bf16* W, const float* s, const float* z, uint8_t* Wq_packed,
                        uint8_t* z8, eqat_fp16* s16, void* stream) {
-  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_plain_desc(d));
   EQAT_TRY(check_ptrs(W, s, z, Wq_packed, z8, s16));
   return launch_quantize_pack(*d, W, s, z, Wq_packed, z8, s16, as_stream(stream));
 }
 
 int eqat_pack(const eqat_desc* d, const uint8_t* codes, uint8_t* Wq_packed, void* stream) {
-  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_plain_desc(d));
   EQAT_TRY(check_ptrs(codes, Wq_packed));
   return launch_pack(*d, codes, Wq_packed, as_stream(stream));
 }
 
 int eqat_unpack(const eqat_desc* d, const uint8_t* Wq_packed, uint8_t* codes, void* stream) {
-  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_plain_desc(d));
   EQAT_TRY(check_ptrs(Wq_packed, codes));
   return launch_unpack(*d, Wq_packed, codes, as_stream(stream));
 }
 
 int eqat_pack_zeros(const eqat_desc* d, const uint8_t* z8, uint8_t* z_packed, void* stream) {
-  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_plain_desc(d));
   EQAT_TRY(check_ptrs(z8, z_packed));
   if (((int64_t)d->out_features * d->in_features / d->group) % 8 != 0) return EQAT_ERR_SHAPE;
   return launch_pack_zeros(*d, z8, z_packed, as_stream(stream));
 }
 
 int eqat_unpack_zeros(const eqat_desc* d, const uint8_t* z_packed, uint8_t* z8, void* stream) {
-  EQAT_TRY(check_weight_desc(d));
+  EQAT_TRY(check_plain_desc(d));
   EQAT_TRY(check_ptrs(z_packed, z8));
   if (((int64_t)d->out_features * d->in_features / d->group) % 8 != 0) return EQAT_ERR_SHAPE;
   return launch_unpack_zeros(*d, z_packed, z8, as_stream(stream));
 }
 
 int qlinear_packed_fwd(const eqat_desc* d, const eqat_bf16* X, const uint8_t* Wq_packed, const eqat_fp16* s16,
-                       const uint8_t* z8, eqat_bf16* Y, void* stream) {
+                       const void* z, eqat_bf16* Y, void* stream) {
   EQAT_TRY(check_gemm_desc(d, true));
-  EQAT_TRY(check_ptrs(X, Wq_packed, s16, z8, Y));
+  EQAT_TRY(check_ptrs(X, Wq_packed, s16, z, Y));
   // a handful of tokens (decoding): one pass over the packed weight instead of near-empty tensor-core tiles
-  if (packed_gemv_applies(*d)) return launch_packed_gemv(*d, X, Wq_packed, s16, z8, Y, as_stream(stream));
-  return launch_packed_fwd(*d, X, Wq_packed, s16, z8, Y, as_stream(stream));
+  if (packed_gemv_applies(*d)) return launch_packed_gemv(*d, X, Wq_packed, s16, z, Y, as_stream(stream));
+  return launch_packed_fwd(*d, X, Wq_packed, s16, z, Y, as_stream(stream));
 }
 
 int qlinear_packed_bwd_dx(const eqat_desc* d, const eqat_bf16* dY, const uint8_t* Wq_packed, const eqat_fp16* s16,
-                          const uint8_t* z8, eqat_bf16* dX, void* stream) {
+                          const void* z, eqat_bf16* dX, void* stream) {
   EQAT_TRY(check_gemm_desc(d, true));
-  EQAT_TRY(check_ptrs(dY, Wq_packed, s16, z8, dX));
-  return launch_packed_dx(*d, dY, Wq_packed, s16, z8, dX, as_stream(stream));
+  EQAT_TRY(check_ptrs(dY, Wq_packed, s16, z, dX));
+  return launch_packed_dx(*d, dY, Wq_packed, s16, z, dX, as_stream(stream));
 }
 
 int qlinear_packed_bwd_ds(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* dY, const uint8_t* Wq_packed,
-                          const uint8_t* z8, const eqat_fp16* s16, float* ds, float* dz, void* workspace,
+                          const void* z, const eqat_fp16* s16, float* ds, float* dz, void* workspace,
                           size_t workspace_bytes, void* stream) {
-  (void)workspace;
-  (void)workspace_bytes;
   EQAT_TRY(check_gemm_desc(d, true));
-  EQAT_TRY(check_ptrs(X, dY, Wq_packed, z8, ds));
+  EQAT_TRY(check_ptrs(X, dY, Wq_packed, z, ds));
   if (dz != nullptr) EQAT_TRY(check_ptrs(dz, s16));
-  return launch_packed_ds(*d, X, dY, Wq_packed, z8, s16, ds, dz, as_stream(stream));
+  const size_t need = packed_ds_workspace_bytes(*d);
+  if (need != 0 && (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0))
+    return EQAT_ERR_WORKSPACE;
+  return launch_packed_ds(*d, X, dY, Wq_packed, z, s16, ds, dz, workspace, as_stream(stream));
 }
 
 }  // extern "C"

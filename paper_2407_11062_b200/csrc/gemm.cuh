@@ -15,14 +15,17 @@ int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X,
 // the gradient of W_hat is never stored.
 int launch_dense_dw_ste(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X, const eqat_bf16* W, const float* s,
                         const float* z, eqat_bf16* dW, float* ds, float* dz, cudaStream_t st);
-// Y = X * dequant(Wq)^T and dX = dY * dequant(Wq), codes expanded in shared memory
+// Y = X * dequant(Wq)^T and dX = dY * dequant(Wq), codes expanded in shared memory.  zq: zero points as uint8 or,
+// with desc.zero_point_format == EQAT_ZP_FP16, as fp16 values.
 int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
-                      const uint8_t* z8, eqat_bf16* Y, cudaStream_t st);
+                      const void* zq, eqat_bf16* Y, cudaStream_t st);
 int launch_packed_dx(const eqat_desc& d, const eqat_bf16* dY, const uint8_t* Wq, const eqat_fp16* s16,
-                     const uint8_t* z8, eqat_bf16* dX, cudaStream_t st);
-// ds (and optionally dz) reduced in the epilogue of dY^T * X
+                     const void* zq, eqat_bf16* dX, cudaStream_t st);
+// ds (and optionally dz) reduced in the epilogue of dY^T * X.  One group per row needs
+// packed_ds_workspace_bytes(d) bytes of scratch for the per-tile partial sums (0 otherwise).
+size_t packed_ds_workspace_bytes(const eqat_desc& d);
 int launch_packed_ds(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* dY, const uint8_t* Wq,
-                     const uint8_t* z8, const eqat_fp16* s16, float* ds, float* dz, cudaStream_t st);
+                     const void* zq, const eqat_fp16* s16, float* ds, float* dz, void* workspace, cudaStream_t st);
 
 // Self-test of the bounded wait: one warp waits 1 ms for a barrier that is never signalled, records
 // EQAT_ERR_TIMEOUT / WAIT_SELFTEST in the status word and returns.

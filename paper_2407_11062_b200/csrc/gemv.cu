@@ -69,8 +69,8 @@ __device__ __forceinline__ void load_unit(const uint8_t* p, uint32_t (&w)[2 * BI
 template <int BITS, int T>
 __global__ void __launch_bounds__(kThreads)
 packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ Wq, const eqat_fp16* __restrict__ s16,
-                   const uint8_t* __restrict__ z8, eqat_bf16* __restrict__ Y, int out_features, int in_features,
-                   int group_shift, int sectors) {
+                   const void* __restrict__ zq, eqat_bf16* __restrict__ Y, int out_features, int in_features,
+                   int group_shift, int groups_per_row, int sectors, int z_fp16) {
   extern __shared__ __align__(16) float smem_f[];
   const int units = in_features >> 6;
   float* xs = smem_f;                                   // [T][in]
@@ -80,10 +80,12 @@ packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ 
 
   const int row = blockIdx.x * kRows + lane;
   const bool live = row < out_features;
-  const int groups_per_row = in_features >> group_shift;
   const uint8_t* wrow = Wq + (size_t)(live ? row : 0) * ((size_t)in_features * BITS / 8);
   const eqat_fp16* srow = s16 + (size_t)(live ? row : 0) * groups_per_row;
-  const uint8_t* zrow = z8 + (size_t)(live ? row : 0) * groups_per_row;
+  // zero points: one byte each, or (z_fp16) one fp16 value each; kept as 16 raw bits next to the step size
+  const size_t zrow = (size_t)(live ? row : 0) * groups_per_row;
+  const uint8_t* z8 = static_cast<const uint8_t*>(zq);
+  const eqat_fp16* z16 = static_cast<const eqat_fp16*>(zq);
   // whole pairs of units per warp (in_features is a multiple of 128): a pair is 32-byte aligned for 2- and
   // 4-bit codes, and lies in one group or in two consecutive ones
   const int pairs = units >> 1;
@@ -126,11 +128,18 @@ packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ 
         const int g = ((u0 + k) << 6) >> group_shift;
         if (group_shift == 6) {
           const uint32_t s2 = __ldg(reinterpret_cast<const uint32_t*>(srow + g));
-          const uint32_t z2 = __ldg(reinterpret_cast<const unsigned short*>(zrow + g));
-          sz_nxt[k] = (s2 & 0xFFFFu) | ((z2 & 0xFFu) << 16);
-          sz_nxt[k + 1] = (s2 >> 16) | ((z2 >> 8) << 16);
+          if (z_fp16) {
+            const uint32_t z2 = __ldg(reinterpret_cast<const uint32_t*>(z16 + zrow + g));
+            sz_nxt[k] = (s2 & 0xFFFFu) | (z2 << 16);
+            sz_nxt[k + 1] = (s2 >> 16) | (z2 & 0xFFFF0000u);
+          } else {
+            const uint32_t z2 = __ldg(reinterpret_cast<const unsigned short*>(z8 + zrow + g));
+            sz_nxt[k] = (s2 & 0xFFFFu) | ((z2 & 0xFFu) << 16);
+            sz_nxt[k + 1] = (s2 >> 16) | ((z2 >> 8) << 16);
+          }
         } else {
-          sz_nxt[k] = sz_nxt[k + 1] = (uint32_t)__ldg(srow + g) | ((uint32_t)__ldg(zrow + g) << 16);
+          const uint32_t zraw = z_fp16 ? (uint32_t)__ldg(z16 + zrow + g) : (uint32_t)__ldg(z8 + zrow + g);
+          sz_nxt[k] = sz_nxt[k + 1] = (uint32_t)__ldg(srow + g) | (zraw << 16);
         }
       }
   };
@@ -179,7 +188,7 @@ packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ 
       const int u = u0 + k;
       if (u < u_end) {
         const float s = __half2float(__ushort_as_half((unsigned short)(sz[k] & 0xFFFFu)));
-        const float z = (float)(sz[k] >> 16);
+        const float z = z_fp16 ? __half2float(__ushort_as_half((unsigned short)(sz[k] >> 16))) : (float)(sz[k] >> 16);
         // four independent partial sums per token and kAhead activation loads in flight: the loop is otherwise a
         // single chain of dependent multiply-adds behind one shared-memory load
         constexpr int kAhead = T == 1 ? 4 : (T == 2 ? 2 : 1);
@@ -231,7 +240,7 @@ packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ 
 }
 
 template <int BITS, int T>
-int launch_one(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const uint8_t* z8,
+int launch_one(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
                eqat_bf16* Y, int group_shift, cudaStream_t st) {
   auto kern = packed_gemv_kernel<BITS, T>;
   const size_t smem = smem_floats(T, d.in_features) * sizeof(float);
@@ -241,36 +250,41 @@ int launch_one(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const 
   }
   const int grid = (d.out_features + kRows - 1) / kRows;
   const int sectors = (reinterpret_cast<uintptr_t>(Wq) & 31u) == 0 ? 1 : 0;
-  kern<<<grid, kThreads, smem, st>>>(X, Wq, s16, z8, Y, d.out_features, d.in_features, group_shift, sectors);
+  kern<<<grid, kThreads, smem, st>>>(X, Wq, s16, zq, Y, d.out_features, d.in_features, group_shift,
+                                     d.in_features / d.group, sectors, d.zero_point_format == EQAT_ZP_FP16 ? 1 : 0);
   return launch_status();
 }
 
 template <int BITS>
-int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const uint8_t* z8,
+int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
                 eqat_bf16* Y, int group_shift, cudaStream_t st) {
   switch ((int)d.tokens) {
-    case 1: return launch_one<BITS, 1>(d, X, Wq, s16, z8, Y, group_shift, st);
-    case 2: return launch_one<BITS, 2>(d, X, Wq, s16, z8, Y, group_shift, st);
-    case 3: return launch_one<BITS, 3>(d, X, Wq, s16, z8, Y, group_shift, st);
-    default: return launch_one<BITS, 4>(d, X, Wq, s16, z8, Y, group_shift, st);
+    case 1: return launch_one<BITS, 1>(d, X, Wq, s16, zq, Y, group_shift, st);
+    case 2: return launch_one<BITS, 2>(d, X, Wq, s16, zq, Y, group_shift, st);
+    case 3: return launch_one<BITS, 3>(d, X, Wq, s16, zq, Y, group_shift, st);
+    default: return launch_one<BITS, 4>(d, X, Wq, s16, zq, Y, group_shift, st);
   }
 }
 
 }  // namespace
 
 bool packed_gemv_applies(const eqat_desc& d) {
-  return d.tokens >= 1 && d.tokens <= kGemvMaxTokens &&
+  // a 64-code unit must lie inside one group: groups of 32 go through the tiled kernel
+  return d.tokens >= 1 && d.tokens <= kGemvMaxTokens && d.group >= 64 &&
          smem_floats((int)d.tokens, d.in_features) * sizeof(float) <= kMaxSmem;
 }
 
 int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
-                       const uint8_t* z8, eqat_bf16* Y, cudaStream_t st) {
-  int group_shift = 0;
-  while ((1 << group_shift) < d.group) ++group_shift;
+                       const void* zq, eqat_bf16* Y, cudaStream_t st) {
+  int group_shift = 31;                                  // one group per row: every group index shifts to 0
+  if (d.group <= 256) {
+    group_shift = 0;
+    while ((1 << group_shift) < d.group) ++group_shift;
+  }
   switch (d.bits) {
-    case 2: return launch_bits<2>(d, X, Wq, s16, z8, Y, group_shift, st);
-    case 3: return launch_bits<3>(d, X, Wq, s16, z8, Y, group_shift, st);
-    default: return launch_bits<4>(d, X, Wq, s16, z8, Y, group_shift, st);
+    case 2: return launch_bits<2>(d, X, Wq, s16, zq, Y, group_shift, st);
+    case 3: return launch_bits<3>(d, X, Wq, s16, zq, Y, group_shift, st);
+    default: return launch_bits<4>(d, X, Wq, s16, zq, Y, group_shift, st);
   }
 }
 

@@ -377,8 +377,9 @@ def test_block_ap_is_deterministic(eqat):
 
 
 # --------------------------------------------------------------------------- E2E-QP layer
-def run_e2e(eqat, cfg, lin, tokens, with_dz=True, fp16_steps=False):
-    """Hand-off (quantise + pack on the oracle's side) then the three packed-weight calls."""
+def run_e2e(eqat, cfg, lin, tokens, with_dz=True, fp16_steps=False, real_z=False):
+    """Hand-off (quantise + pack on the oracle's side) then the three packed-weight calls.  `real_z`: the zero
+    points are handed over as fp16 values moved off the integers (the variant that trains z), codes unchanged."""
     Wb = weight_for(cfg, lin); W32 = f32(Wb)
     Xb, dYb = activations_for(cfg, lin, tokens)
     out, in_f, ng = lin.out_features, lin.in_features, lin.in_features // cfg.group
@@ -386,8 +387,16 @@ def run_e2e(eqat, cfg, lin, tokens, with_dz=True, fp16_steps=False):
     if fp16_steps:
         s = s.astype(np.float16).astype(np.float32)
     P_o, z8_o, s16_o = O.quantize_pack(W32, s, z, cfg.bits, cfg.group)
-    d = eqat.make_desc(cfg.bits, cfg.group, out, in_f, tokens)
-    Pd, z8d = dev(P_o), dev(z8_o)
+    zfmt = eqat.EQAT_ZP_FP16 if real_z else eqat.EQAT_ZP_U8
+    d = eqat.make_desc(cfg.bits, cfg.group, out, in_f, tokens, 0, zfmt)
+    if real_z:
+        drift = np.random.default_rng(ng + out).uniform(-0.45, 0.45, z8_o.shape)
+        z_o = (z8_o + drift).astype(np.float16)                          # what a few optimiser steps leave behind
+        zd = torch.from_numpy(z_o.view(np.int16)).view(torch.float16).cuda()
+        z_o = z_o.astype(np.float32)
+    else:
+        z_o, zd = z8_o, dev(z8_o)
+    Pd = dev(P_o)
     s16d = torch.from_numpy(s16_o.view(np.int16)).view(torch.float16).cuda()
     Xd, dYd = bits_to_torch(Xb), bits_to_torch(dYb)
     guard = Guarded()
@@ -395,28 +404,37 @@ def run_e2e(eqat, cfg, lin, tokens, with_dz=True, fp16_steps=False):
     dX = guard.empty(tokens, in_f, dtype=torch.bfloat16)
     ds = guard.empty(out, ng)
     dz = guard.empty(out, ng) if with_dz else None
-    eqat.qlinear_packed_fwd(d, Xd, Pd, s16d, z8d, Y)
-    eqat.qlinear_packed_bwd_dx(d, dYd, Pd, s16d, z8d, dX)
-    eqat.qlinear_packed_bwd_ds(d, Xd, dYd, Pd, z8d, s16d, ds, dz)
+    n_ws = eqat.workspace_bytes(d, eqat.EQAT_OP_PACKED_BWD_DS)
+    assert (n_ws > 0) == (cfg.group > 256)                               # only one group per row needs scratch
+    ws = guard.empty(n_ws, dtype=torch.uint8) if n_ws else None
+    eqat.qlinear_packed_fwd(d, Xd, Pd, s16d, zd, Y)
+    eqat.qlinear_packed_bwd_dx(d, dYd, Pd, s16d, zd, dX)
+    eqat.qlinear_packed_bwd_ds(d, Xd, dYd, Pd, zd, s16d, ds, dz, ws)
     guard.check()
     q = O.unpack_rows(P_o, cfg.bits, in_f)
-    return dict(X=f32(Xb), dY=f32(dYb), q=q, z8=z8_o, s16=s16_o.astype(np.float32), Y=Y, dX=dX, ds=ds, dz=dz,
-                W=W32, s=s, z=z)
+    return dict(X=f32(Xb), dY=f32(dYb), q=q, z8=z_o, s16=s16_o.astype(np.float32), Y=Y, dX=dX, ds=ds, dz=dz,
+                W=W32, s=s, z=z, real_z=real_z)
 
 
 def check_e2e(r, group):
-    What_o = O.dequantize(r["q"], r["s16"], r["z8"], group)
+    rz = r["real_z"]
+    What_o = O.dequantize(r["q"], r["s16"], r["z8"], group, real_zero_point=rz)
     check_contractions(r, What_o)
-    assert rel_err(torch_to_f64(r["ds"]), O.e2e_ds(r["dY"], r["X"], r["q"], r["z8"], group)) <= TOL
+    assert rel_err(torch_to_f64(r["ds"]), O.e2e_ds(r["dY"], r["X"], r["q"], r["z8"], group, real_zero_point=rz)) <= TOL
     if r["dz"] is not None:
         assert rel_err(torch_to_f64(r["dz"]), O.e2e_dz(r["dY"], r["X"], r["s16"], group)) <= TOL
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
-@pytest.mark.parametrize("group", [64, 128, 256])
-def test_e2e_small(eqat, bits, group):
-    cfg = small_cfg(f"e2e_{bits}_{group}", 512, 512, bits, group, 256, "student_t4", 0.02, 0.01)
-    check_e2e(run_e2e(eqat, cfg, cfg.linears[0], 256), group)
+@pytest.mark.parametrize("group", [32, 64, 128, 256, 512])
+@pytest.mark.parametrize("real_z", [False, True], ids=["z_u8", "z_fp16"])
+def test_e2e_small(eqat, bits, group, real_z):
+    """Every group size of the paper's ablation (32 .. 256) and one group per row (512 = in_features, the
+    channel-wise setting of its Q-PEFT comparison), with frozen integer zero points and with trained fp16 ones.
+    600 tokens: a pair of CTAs per tile with a ragged last row-tile; 256: single CTAs."""
+    for tokens in (600, 256):
+        cfg = small_cfg(f"e2e_{bits}_{group}", 512, 512, bits, group, tokens, "student_t4", 0.02, 0.01)
+        check_e2e(run_e2e(eqat, cfg, cfg.linears[0], tokens, real_z=real_z), group)
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
@@ -453,10 +471,14 @@ def test_few_token_forward_agrees_with_tiled_forward(eqat):
     (1024, 256, 520, 2, 64),
     (64, 11008, 4, 2, 64),          # few-token kernel with more than 48 KB of staged activations
     (64, 28672, 2, 4, 128),         # activations too large to stage: two tokens through the tiled kernel
+    (448, 1408, 700, 3, 32),        # groups of 32, nothing a multiple of a tile
+    (320, 1408, 1100, 2, 1408),     # one group per row with in_features not a power of two: 5.5 column tiles
+    (192, 640, 3, 4, 640),          # one group per row through the few-token kernel
+    (192, 640, 3, 2, 32),           # groups of 32 with few tokens: the tiled kernel
 ])
 def test_e2e_ragged(eqat, out, in_f, tokens, bits, group):
     cfg = small_cfg(f"e2er_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens)
-    check_e2e(run_e2e(eqat, cfg, cfg.linears[0], tokens, with_dz=(bits != 4)), group)
+    check_e2e(run_e2e(eqat, cfg, cfg.linears[0], tokens, with_dz=(bits != 4), real_z=(group in (32, 640))), group)
 
 
 def test_e2e_is_deterministic_and_matches_block_ap_forward(eqat):

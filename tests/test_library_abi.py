@@ -70,9 +70,20 @@ def test_null_and_misaligned_pointers(eqat):
     assert eqat.lib.eqat_fakequant_weight(ctypes.byref(d), ok, odd, ok, ok, None) == eqat.EQAT_ERR_ALIGN
     assert eqat.lib.eqat_fakequant_weight(None, ok, ok, ok, ok, None) == eqat.EQAT_ERR_NULL
     assert eqat.lib.qlinear_packed_fwd(ctypes.byref(d), ok, ok, ok, ok, None, None) == eqat.EQAT_ERR_NULL
-    # packed GEMMs accept group 64/128/256 only; GEMMs need tokens > 0 and out % 64 == 0
-    d32 = eqat.make_desc(2, 32, 512, 512, 256)
-    assert eqat.lib.qlinear_packed_fwd(ctypes.byref(d32), ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_UNSUPPORTED
+    # packed GEMMs: a group longer than 256 must be the whole row; GEMMs need tokens > 0 and out % 64 == 0
+    d512 = eqat.make_desc(2, 512, 512, 1024, 256)
+    assert eqat.lib.qlinear_packed_fwd(ctypes.byref(d512), ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_UNSUPPORTED
+    # zero-point formats: fp16 zero points exist for the packed entry points only; unknown formats nowhere
+    dz16 = eqat.make_desc(2, 64, 512, 512, 256, 0, eqat.EQAT_ZP_FP16)
+    assert eqat.lib.eqat_fakequant_weight(ctypes.byref(dz16), ok, ok, ok, ok, None) == eqat.EQAT_ERR_UNSUPPORTED
+    assert eqat.lib.qlinear_fakequant_fwd(ctypes.byref(dz16), ok, ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_UNSUPPORTED
+    assert eqat.lib.qlinear_packed_fwd(ctypes.byref(dz16), ok, ok, ok, None, ok, None) == eqat.EQAT_ERR_NULL
+    dz9 = eqat.make_desc(2, 64, 512, 512, 256, 0, 9)
+    assert eqat.lib.qlinear_packed_fwd(ctypes.byref(dz9), ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_UNSUPPORTED
+    # one group per row: the step-size gradient needs scratch for the per-tile sums
+    dcw = eqat.make_desc(2, 1024, 512, 1024, 256)
+    assert eqat.workspace_bytes(dcw, eqat.EQAT_OP_PACKED_BWD_DS) == 2 * 4 * 512 * 4
+    assert eqat.lib.qlinear_packed_bwd_ds(ctypes.byref(dcw), ok, ok, ok, ok, ok, ok, None, None, 0, None) == eqat.EQAT_ERR_WORKSPACE
     d0 = eqat.make_desc(2, 64, 512, 512, 0)
     assert eqat.lib.qlinear_packed_fwd(ctypes.byref(d0), ok, ok, ok, ok, ok, None) == eqat.EQAT_ERR_SHAPE
     d96 = eqat.make_desc(2, 64, 96, 512, 256)

@@ -214,6 +214,37 @@ def pin_e2e_ds(o):
 
 
 # --------------------------------------------------------------------------- min/max initialisation
+def pin_real_zero_point(o):
+    """E2E-QP with a trained, real-valued zero point: Eq. 2 uses it unrounded.  Eq. 2 is linear in z, so
+    W_hat(z) = W_hat(0) - z s exactly (up to the product's rounding), finite differences in z are exact for any
+    step, and an integer-valued z gives the frozen-zero-point result bit for bit."""
+    g = np.random.default_rng(21)
+    q = g.integers(0, 4, (5, 24))
+    s = (np.abs(g.standard_normal((5, 3))) * 0.01 + 0.002).astype(np.float32)
+    z = (g.random((5, 3)) * 3).astype(np.float32)                   # fractional
+    s_el, z_el = np.repeat(s.astype(np.float64), 8, 1), np.repeat(z.astype(np.float64), 8, 1)
+    Wr = o.dequantize(q, s, z, 8, real_zero_point=True)
+    np.testing.assert_allclose(Wr, o.dequantize(q, s, np.zeros_like(z), 8) - z_el * s_el, rtol=0, atol=1e-15)
+    assert np.abs(Wr - o.dequantize(q, s, z, 8)).max() > 1e-4         # rounding z would be a different layer
+    # hand value: q = 3, z = 1.25, s = 0.5  ->  (3 - 1.25) * 0.5 = 0.875
+    assert o.dequantize(np.array([[3]]), np.array([[0.5]], np.float32), np.array([[1.25]], np.float32), 1,
+                        real_zero_point=True)[0, 0] == 0.875
+    zi = np.rint(z)
+    np.testing.assert_array_equal(o.dequantize(q, s, zi, 8, real_zero_point=True), o.dequantize(q, s, zi, 8))
+    # the gradients: ds is linear in z as well, dz = -s * sum G is the exact derivative of the loss <dY, Y> in z
+    X = g.standard_normal((7, 24)); dY = g.standard_normal((7, 5))
+    G = o.weight_grad(dY, X)
+    ds = o.e2e_ds(dY, X, q, z, 8, real_zero_point=True)
+    brute = np.array([[sum(G[r, 8 * k + j] * (q[r, 8 * k + j] - float(z[r, k])) for j in range(8)) for k in range(3)]
+                      for r in range(5)])
+    np.testing.assert_allclose(ds, brute, rtol=1e-12, atol=1e-12)
+    loss = lambda zz: float((dY * o.linear_fwd(X, o.dequantize(q, s, zz, 8, real_zero_point=True))).sum())
+    dz = o.e2e_dz(dY, X, s, 8)
+    for r, k, h in ((0, 0, 0.37), (4, 2, -1.6)):
+        z2 = z.astype(np.float64).copy(); z2[r, k] += h
+        assert abs((loss(z2) - loss(z.astype(np.float64))) / h - dz[r, k]) <= 1e-9 * (1 + abs(dz[r, k]))
+
+
 def pin_minmax(o):
     W = np.array([[-0.3, 0.1, 0.6, 0.0, 1.0, 1.0, 1.0, 1.0]], np.float32)
     s, z = o.minmax_init(W, 2, 4)
@@ -343,7 +374,7 @@ def pin_shapes_other_models(o):
 
 PINS = [pin_worked_example, pin_rounding_is_half_to_even, pin_inclusive_bounds, pin_quantiser_invariants,
         pin_zero_point_is_rounded_in_forward, pin_ste_against_forward, pin_contractions, pin_e2e_ds,
-        pin_minmax, pin_pack_golden, pin_pack_roundtrip_and_bigint, pin_sizes, pin_handoff_side_outputs,
+        pin_real_zero_point, pin_minmax, pin_pack_golden, pin_pack_roundtrip_and_bigint, pin_sizes, pin_handoff_side_outputs,
         pin_shapes_other_models]
 
 
@@ -381,6 +412,8 @@ MUTATIONS = {
                                "return _group_sum(G * (np.asarray(q, np.float64)), group)")],
     "pack_msb_first": [('np.packbits(bitplanes.ravel().astype(np.uint8), bitorder="little")',
                         'np.packbits(bitplanes.ravel().astype(np.uint8), bitorder="big")')],
+    "real_zero_point_rounded_anyway": [("return np.asarray(z, np.float64) if real_zero_point else round_zero_point(z)",
+                                        "return round_zero_point(z)")],
     "minmax_z_sign": [("z = -np.rint(mn / s)", "z = np.rint(mn / s)")],
     "handoff_zero_point_clamp_dropped": [("z8 = np.clip(round_zero_point(z), 0, qmax(bits)).astype(np.uint8)",
                                           "z8 = round_zero_point(z).astype(np.int64).astype(np.uint8)")],
