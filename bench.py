@@ -216,8 +216,9 @@ class BlockWorkload:
     hand-off calls are part of the step only with `handoff` (the headline step), otherwise they run once here."""
 
     def __init__(self, eqat, device, seed, t_block_ap=T_BLOCK_AP, t_e2e=T_E2E, model="7b", bits=BITS, group=GROUP,
-                 weight=("normal", 0.02, 0.0), handoff=True):
+                 weight=("normal", 0.02, 0.0), handoff=True, store_w_hat=True):
         self.eqat, self.device = eqat, device
+        self.store_w_hat = store_w_hat                     # False: W_hat is not kept, the GEMMs fake-quantise W themselves
         self.t_ap, self.t_e2e, self.model, self.bits, self.group, self.handoff = t_block_ap, t_e2e, model, bits, group, handoff
         g = torch.Generator(device=device); g.manual_seed(seed)
         bf, dev = torch.bfloat16, device
@@ -272,8 +273,9 @@ class BlockWorkload:
                 timed("minmax_init/" + tag, lambda: e.eqat_minmax_init(S["d_ap"], L["W"], L["s"], L["z"]))
             if self.t_ap:
                 Xa, dYa, Ya, dXa = S["X"][: self.t_ap], S["dY"][: self.t_ap], S["Y"][: self.t_ap], S["dX"][: self.t_ap]
-                timed("fakequant_fwd/" + tag, lambda: e.qlinear_fakequant_fwd(S["d_ap"], Xa, L["W"], L["s"], L["z"], Ya, S["What"]))
-                timed("fakequant_bwd/" + tag, lambda: e.qlinear_fakequant_bwd(S["d_ap"], Xa, dYa, L["W"], L["s"], L["z"], S["What"],
+                What = S["What"] if self.store_w_hat else None
+                timed("fakequant_fwd/" + tag, lambda: e.qlinear_fakequant_fwd(S["d_ap"], Xa, L["W"], L["s"], L["z"], Ya, What))
+                timed("fakequant_bwd/" + tag, lambda: e.qlinear_fakequant_bwd(S["d_ap"], Xa, dYa, L["W"], L["s"], L["z"], What,
                                                                                 dXa, S["dW"], S["ds"], S["dz"], S["ws"]))
             if self.handoff:
                 timed("quantize_pack/" + tag, lambda: e.eqat_quantize_pack(S["d_ap"], L["W"], L["s"], L["z"], L["P"], L["z8"], L["s16"]))
@@ -570,6 +572,26 @@ def run_extra_config(eqat, device, name, spec, peaks):
     return out
 
 
+def run_block_ap_forms(eqat, device, steps=10):
+    """Block-AP forward + backward of the headline workload in its two forms, timed in the same process: W_hat
+    written once by the streaming fake quantiser and read by the GEMMs (what the headline step uses), against
+    W_hat never stored, each tile of W fake-quantised inside the forward and the dX GEMM."""
+    out = {}
+    f_ap = step_flops(T_BLOCK_AP, 0)[0]
+    for name, stored in (("stored_w_hat", True), ("fake_quantised_in_the_gemm", False), ("stored_w_hat_again", True)):
+        wl = BlockWorkload(eqat, device, seed=3, t_block_ap=T_BLOCK_AP, t_e2e=0, handoff=False, store_w_hat=stored)
+        ms, timers = time_steps(wl, steps, 3)
+        by = {}
+        for k, v in summarise(timers).items():
+            by[k.split("/")[0]] = by.get(k.split("/")[0], 0.0) + v["total_ms"] / steps
+        out[name] = {"ms_per_step": ms, "tflops": f_ap / (ms * 1e-3) / 1e12, "fwd_ms": by["fakequant_fwd"], "bwd_ms": by["fakequant_bwd"]}
+        del wl
+        torch.cuda.empty_cache()
+    out["tokens"] = T_BLOCK_AP
+    out["used_by_the_headline_step"] = "stored_w_hat"
+    return out
+
+
 def run_streaming_leg(eqat, device, peaks, bits, group, shape=(11008, 4096), min_launches=56, min_bytes=640e6):
     """The five streaming kernels, each timed cold: `n` distinct sets of inputs and outputs whose combined size is
     several times the L2 (so no launch finds its operands or leaves its results in cache for the next one), at
@@ -746,6 +768,7 @@ def run_ours(args):
         if world == 1 and not args.headline_only:
             # the other workloads and the cold streaming figures (one GPU is enough for them: the path is replicated)
             out["configs"] = {name: run_extra_config(eqat, device, name, spec, peaks) for name, spec in EXTRA_CONFIGS.items()}
+            out["block_ap_forms"] = run_block_ap_forms(eqat, device)
             out["streaming"] = {"w2g64": run_streaming_leg(eqat, device, peaks, 2, 64),
                                 "w4g128": run_streaming_leg(eqat, device, peaks, 4, 128)}
             alias = {"fakequant_weight": "fakequant_weight", "ste_bwd": "ste_bwd", "minmax_init": "minmax_init_cold",

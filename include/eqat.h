@@ -130,8 +130,15 @@ int eqat_fakequant_weight(const eqat_desc* desc, const eqat_bf16* W, const float
                           eqat_bf16* W_hat, void* stream);
 
 /* Block-AP forward (Sec. 3.2): W_hat as above, then Y = X * W_hat^T with fp32
- * accumulation.  W_hat is written out because the backward pass reads it.
- *   X [T,in] bf16, W, s, z (in)   Y [T,out] bf16, W_hat [out,in] bf16 (out) */
+ * accumulation.  Two forms, same Y bit for bit:
+ *   - W_hat != NULL: W_hat is computed once by a streaming kernel and written out
+ *     (the backward pass can then read it); the faster form.
+ *   - W_hat == NULL: nothing is stored; every tile of W is fake-quantised inside
+ *     the GEMM after it has been copied to shared memory (Eq. 1-2 "integrated
+ *     within the computation graph" taken literally).  It saves out*in*2 bytes of
+ *     memory and costs more time, because each tile of W is quantised once per
+ *     512 tokens instead of once.  Needs group <= 256 or group == in_features.
+ *   X [T,in] bf16, W, s, z (in)   Y [T,out] bf16, W_hat [out,in] bf16 (out, optional) */
 int qlinear_fakequant_fwd(const eqat_desc* desc, const eqat_bf16* X, const eqat_bf16* W, const float* s,
                           const float* z, eqat_bf16* Y, eqat_bf16* W_hat, void* stream);
 
@@ -146,7 +153,9 @@ int eqat_ste_bwd(const eqat_desc* desc, const eqat_bf16* dW_hat, const eqat_bf16
                  const float* z, eqat_bf16* dW, float* ds, float* dz, void* stream);
 
 /* Block-AP backward: dX = dY * W_hat, dW_hat = dY^T * X, then Eqs. 3-5 as in
- * eqat_ste_bwd.  With groups of up to 256 elements Eqs. 3-5 are applied to the
+ * eqat_ste_bwd.  W_hat is the array qlinear_fakequant_fwd stored, or NULL, in
+ * which case the dX GEMM fake-quantises W tile by tile itself (same dX; same
+ * restriction on the group as in the forward).  With groups of up to 256 elements Eqs. 3-5 are applied to the
  * fp32 accumulators of dW_hat inside the same kernel and dW_hat is never
  * stored; longer groups (channel-wise) keep dW_hat in bf16 in the workspace and
  * run eqat_ste_bwd on it.  Needs eqat_workspace_bytes(desc,

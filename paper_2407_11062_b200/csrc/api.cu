@@ -47,6 +47,9 @@ int check_gemm_desc(const eqat_desc* d, bool packed) {
   return EQAT_OK;
 }
 
+// The kernels that fake-quantise the latent weight tile by tile index groups with a shift, or not at all.
+inline bool latent_group_ok(const eqat_desc* d) { return d->group <= 256 || d->group == d->in_features; }
+
 template <typename... P>
 int check_ptrs(P... ptrs) {
   const void* v[] = {static_cast<const void*>(ptrs)...};
@@ -132,7 +135,13 @@ int eqat_fakequant_weight(const eqat_desc* d, const eqat_bf16* W, const float* s
 int qlinear_fakequant_fwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* W, const float* s, const float* z,
                           eqat_bf16* Y, eqat_bf16* W_hat, void* stream) {
   EQAT_TRY(check_gemm_desc(d, false));
-  EQAT_TRY(check_ptrs(X, W, s, z, Y, W_hat));
+  EQAT_TRY(check_ptrs(X, W, s, z, Y));
+  if (W_hat == nullptr) {
+    // W_hat is not wanted: fake-quantise each tile of W inside the GEMM, after it has reached shared memory
+    if (!latent_group_ok(d)) return EQAT_ERR_UNSUPPORTED;
+    return launch_latent_fwd(*d, X, W, s, z, Y, as_stream(stream));
+  }
+  if (!aligned16(W_hat)) return EQAT_ERR_ALIGN;
   EQAT_TRY(launch_fakequant(*d, W, s, z, W_hat, as_stream(stream)));
   return launch_dense_fwd(*d, X, W_hat, Y, as_stream(stream));
 }
@@ -149,8 +158,10 @@ int qlinear_fakequant_bwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf1
                           const float* s, const float* z, const eqat_bf16* W_hat, eqat_bf16* dX, eqat_bf16* dW,
                           float* ds, float* dz, void* workspace, size_t workspace_bytes, void* stream) {
   EQAT_TRY(check_gemm_desc(d, false));
-  EQAT_TRY(check_ptrs(X, dY, W, s, z, W_hat, dX, dW, ds));
+  EQAT_TRY(check_ptrs(X, dY, W, s, z, dX, dW, ds));
   if (dz != nullptr && !aligned16(dz)) return EQAT_ERR_ALIGN;
+  if (W_hat != nullptr && !aligned16(W_hat)) return EQAT_ERR_ALIGN;
+  if (W_hat == nullptr && !latent_group_ok(d)) return EQAT_ERR_UNSUPPORTED;
   // A group that fits inside one output tile is reduced in the weight-gradient GEMM's epilogue and needs no
   // scratch; a longer one (channel-wise quantisation) spans tiles, so its gradient goes through the workspace
   // and a second kernel.
@@ -162,7 +173,8 @@ int qlinear_fakequant_bwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf1
   }
   eqat_bf16* dW_hat = static_cast<eqat_bf16*>(workspace);
   cudaStream_t st = as_stream(stream);
-  EQAT_TRY(launch_dense_dx(*d, dY, W_hat, dX, st));
+  if (W_hat != nullptr) EQAT_TRY(launch_dense_dx(*d, dY, W_hat, dX, st));
+  else EQAT_TRY(launch_latent_dx(*d, dY, W, s, z, dX, st));      // no stored W_hat: Eq. 1-2 inside the dX GEMM
   if (fused) return launch_dense_dw_ste(*d, dY, X, W, s, z, dW, ds, dz, st);
   EQAT_TRY(launch_dense_dw(*d, dY, X, dW_hat, st));
   return launch_ste_bwd(*d, dW_hat, W, s, z, dW, ds, dz, st);

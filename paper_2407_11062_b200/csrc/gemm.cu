@@ -128,6 +128,7 @@ struct Control {
   uint64_t empty[8];         //                                                         (each CTA its own)
   uint64_t full_b[8];        // packed kernels: B stage expanded                        (pair: first CTA's)
   uint64_t empty_b[8];
+  uint64_t raw_b[8];         // latent-weight kernels: B stage filled by TMA, not yet fake-quantised (each CTA its own)
   uint64_t acc_full[2];      //                                                         (each CTA its own)
   uint64_t acc_empty[2];     //                                                         (pair: first CTA's)
   uint64_t drain;
@@ -371,13 +372,16 @@ __device__ __forceinline__ void quad_transpose(uint32_t (&o)[16], int lane) {
   }
 }
 
-// A_MN / B_MN: operand is MN-major.  PACKED: B is expanded from N-bit codes.  PAIR: the tile is computed by two
-// CTAs sharing one MMA.  BITS is used by PACKED and by EPI_DS.
+// A_MN / B_MN: operand is MN-major.  PACKED: the B operand is produced by the CTA's warps: expanded from N-bit
+// codes (BITS = 2, 3, 4), or (BITS = 16, Block-AP) fetched by TMA as the latent bf16 weight and fake-quantised in
+// place, Eq. 1 then Eq. 2, before the tensor core reads it.  PAIR: the tile is computed by two CTAs sharing one
+// MMA.  BITS is used by PACKED and by EPI_DS.
 template <int MT, bool A_MN, bool B_MN, bool PACKED, int EPI, int BITS, bool PAIR>
 __global__ void __launch_bounds__(Cfg<MT, PACKED, PAIR>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const GemmParams p) {
   using C = Cfg<MT, PACKED, PAIR>;
+  constexpr bool LATENT = PACKED && BITS == 16;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_addr(smem_raw);
   const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
@@ -409,6 +413,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       for (int s = 0; s < C::kStagesB; ++s) {
         ptx::mbar_init(ptx::smem_addr(&ctl->full_b[s]), C::kCtas * (C::kBRows / 32));
         ptx::mbar_init(ptx::smem_addr(&ctl->empty_b[s]), 1);
+        ptx::mbar_init(ptx::smem_addr(&ctl->raw_b[s]), 1);
       }
     }
     for (int a = 0; a < C::kAccSets; ++a) {
@@ -419,7 +424,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     ctl->abort = 0;
     ptx::fence_mbar_init();
     ptx::tma_prefetch_desc(&tmap_a);
-    if (!PACKED) ptx::tma_prefetch_desc(&tmap_b);
+    if (!PACKED || LATENT) ptx::tma_prefetch_desc(&tmap_b);
   }
   if (warp == 1) {
     if (PAIR) {
@@ -592,7 +597,92 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (lane == 0 && LATENT) {
+      // Two rings, one thread: the A operand goes to the first CTA's tensor core as it lands, the latent weight
+      // goes to this CTA's own warps first (raw_b), which fake-quantise it in place.  The rings have different
+      // depths and drain at different times, so the thread polls both and serves whichever has a free stage.
+      struct Cursor {
+        int tile, kb, m_blk, n_blk;
+        long n;
+      };
+      auto start = [&](Cursor& c) {
+        c.tile = cluster_id; c.kb = 0; c.n = 0;
+        if (c.tile < num_tiles) tile_coords<PACKED, kBand>(c.tile, num_m, num_n, c.m_blk, c.n_blk);
+      };
+      auto advance = [&](Cursor& c) {
+        ++c.n;
+        if (++c.kb == num_kb) {
+          c.kb = 0;
+          c.tile += num_clusters;
+          if (c.tile < num_tiles) tile_coords<PACKED, kBand>(c.tile, num_m, num_n, c.m_blk, c.n_blk);
+        }
+      };
+      Cursor ca, cb;
+      start(ca); start(cb);
+      uint64_t t_last = ptx::globaltimer_ns();
+      uint32_t idle = 0;
+      while (ca.tile < num_tiles || cb.tile < num_tiles) {
+        bool progress = false;
+        if (ca.tile < num_tiles) {
+          const int st_a = (int)(ca.n % C::kStages);
+          const uint32_t par = (uint32_t)((ca.n / C::kStages) & 1) ^ 1u;
+          const uint32_t bar = ptx::smem_addr(&ctl->empty[st_a]);
+          if (PAIR ? ptx::mbar_try_wait_cluster(bar, par) : ptx::mbar_try_wait(bar, par)) {
+            const uint32_t full = lead(ptx::smem_addr(&ctl->full[st_a]));
+            const uint32_t a_dst = smem_base + C::a_offset(st_a);
+            const int m0 = ca.m_blk * C::kClusterM + rank * C::kTileM;
+            if (PAIR) {
+              ptx::mbar_expect_tx_cluster(full, C::kABytes);
+              ptx::tma_load_2d_pair(a_dst, &tmap_a, ca.kb * BK, m0, full);
+            } else {
+              ptx::mbar_expect_tx(full, C::kABytes);
+              ptx::tma_load_2d(a_dst, &tmap_a, ca.kb * BK, m0, full);
+            }
+            advance(ca);
+            progress = true;
+          }
+        }
+        if (cb.tile < num_tiles) {
+          const int st_b = (int)(cb.n % C::kStagesB);
+          const uint32_t par = (uint32_t)((cb.n / C::kStagesB) & 1) ^ 1u;
+          const uint32_t bar = ptx::smem_addr(&ctl->empty_b[st_b]);
+          if (PAIR ? ptx::mbar_try_wait_cluster(bar, par) : ptx::mbar_try_wait(bar, par)) {
+            const uint32_t raw = ptx::smem_addr(&ctl->raw_b[st_b]);
+            const uint32_t b_dst = smem_base + C::b_offset(st_b);
+            const int n0 = cb.n_blk * BN + rank * C::kBRows;
+            ptx::mbar_expect_tx(raw, C::kBBytes);
+            if (B_MN) {
+#pragma unroll
+              for (int b = 0; b < C::kBRows / 64; ++b)
+                ptx::tma_load_2d(b_dst + b * (BK * 128), &tmap_b, n0 + b * 64, cb.kb * BK, raw);
+            } else {
+              ptx::tma_load_2d(b_dst, &tmap_b, cb.kb * BK, n0, raw);
+            }
+            advance(cb);
+            progress = true;
+          }
+        }
+        if (progress) {
+          idle = 0;
+          t_last = ptx::globaltimer_ns();
+        } else {
+          __nanosleep(64);
+          if ((++idle & 31u) == 0u) {
+            if (*abort_flag) break;
+            if (ptx::globaltimer_ns() - t_last > kWaitLimitNs) {
+              *abort_flag = 1;
+              atomicExch(&g_device_status[1], (int)WAIT_PRODUCER_EMPTY);
+              atomicExch(&g_device_status[0], (int)EQAT_ERR_TIMEOUT);
+              break;
+            }
+          }
+        }
+      }
+      if (*abort_flag) {                                           // outwait the copies in flight (microseconds)
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    } else if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       long issued = 0;
@@ -744,7 +834,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       const int tid = (int)threadIdx.x - 64;
       const int t = tid & (U - 1);                                 // unit within the stage
       const int grp = tid / U;
-      const size_t pitch = (size_t)p.in_features * BITS / 8;      // bytes per packed row
+      const size_t pitch = LATENT ? 0 : (size_t)p.in_features * BITS / 8;      // bytes per packed row
       const int chunks_in = p.in_features >> 6;                   // 64-code units per row
       bool ok = true;
       const int kr = (t & 7) | ((t / (8 * kBoxes)) << 3);         // MN-major: k-row 0..63
@@ -757,11 +847,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       // Register ring of two runs: the loads for the thread's next-but-one run (2*NG*R K blocks ahead) are
       // issued as soon as the current run has been expanded.  A run's step sizes and zero points (one to four
       // consecutive groups of the row) travel with its codes.
+      // Latent weights (BITS = 16): the unit's 128 bytes are already in the stage (TMA); only the group's
+      // fp32 step size and zero point travel through the ring.
       constexpr int R = (!B_MN && BITS == 2) ? 2 : 1;
       constexpr int kStep = NG * R;                                // K blocks between a group's runs
       static_assert(C::kStagesB == 2 * NG && (C::kStagesB & (C::kStagesB - 1)) == 0, "stage = K block index mod 2*NG");
-      uint32_t ring_w[2][R][2 * BITS];
+      constexpr int kCodeWords = LATENT ? 1 : 2 * BITS;
+      uint32_t ring_w[2][R][kCodeWords];
       GroupParamsRaw ring_g[2];
+      float ring_ls[2][2], ring_lz[2][2];                          // latent weights: s, z of the unit's one or two groups
       // groups per run / per unit, and where a 32-code half finds its group among those fetched
       const int span = B_MN ? 64 : 64 * R;                        // codes of one row a fetch covers
       const int g_count = max(1, span >> p.group_shift);          // 1, 2 or 4
@@ -779,12 +873,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         const int wrow0 = B_MN ? kb_first * BK + kr : n_blk * BN + rank * U + t;
         const int unit0 = B_MN ? n_blk * (BN / 64) + rank * kBoxes + box : kb_first;
         const bool valid = B_MN ? (unit0 < chunks_in) : (wrow0 < p.out_features);
-        const uint8_t* code_ptr = p.Wq + (valid ? (size_t)wrow0 * pitch + (size_t)unit0 * (8 * BITS) : 0);
+        const uint8_t* code_ptr = LATENT ? nullptr : p.Wq + (valid ? (size_t)wrow0 * pitch + (size_t)unit0 * (8 * BITS) : 0);
         // first group of the row that a run starting at K block kb needs
         const size_t g_row0 = B_MN ? (size_t)kr * p.groups_per_row + (size_t)((unit0 << 6) >> p.group_shift)
                                    : (size_t)(valid ? wrow0 : 0) * p.groups_per_row;
         auto fetch = [&](int j, int kb) {                         // the run starting at K block kb, into ring slot j
-          if (valid) {
+          if constexpr (LATENT) {
+            if (valid) {
+              const size_t gi = B_MN ? g_row0 + (size_t)kb * BK * p.groups_per_row : g_row0 + (size_t)((kb << 6) >> p.group_shift);
+              ring_ls[j][0] = __ldg(p.s32 + gi);
+              ring_lz[j][0] = __ldg(p.z32 + gi);
+              if (split_units) {
+                ring_ls[j][1] = __ldg(p.s32 + gi + 1);
+                ring_lz[j][1] = __ldg(p.z32 + gi + 1);
+              }
+            }
+          } else if (valid) {
             if constexpr (R == 2) {
               // the run's 32 bytes are one sector of the packed row when the matrix itself starts on a 32-byte
               // boundary (row pitch and unit offsets are multiples of 32); otherwise two 16-byte loads
@@ -812,8 +916,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             if (ok && kb < num_kb) {
               const int stage = (int)((gk + kb) & (C::kStagesB - 1));   // R = 2: even; the run's second block is stage + 1
               const uint32_t phase = (uint32_t)(((gk + kb) / C::kStagesB) & 1);
-              bool free_stage = wait_bounded<PAIR>(ptx::smem_addr(&ctl->empty_b[stage]), phase ^ 1u, abort_flag,
-                                                   WAIT_DEQ_OPERAND_EMPTY);
+              // packed codes: the stage must have been released by the tensor core; latent weights: the raw tile
+              // must have landed in it
+              bool free_stage = LATENT ? wait_bounded(ptx::smem_addr(&ctl->raw_b[stage]), phase, abort_flag, WAIT_DEQ_OPERAND_EMPTY)
+                                       : wait_bounded<PAIR>(ptx::smem_addr(&ctl->empty_b[stage]), phase ^ 1u, abort_flag,
+                                                            WAIT_DEQ_OPERAND_EMPTY);
               if (R == 2 && free_stage)
                 free_stage = wait_bounded<PAIR>(ptx::smem_addr(&ctl->empty_b[stage + 1]), phase ^ 1u, abort_flag,
                                                 WAIT_DEQ_OPERAND_EMPTY);
@@ -824,7 +931,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 // and share a phase): twice the independent work for the scheduler to interleave, one fence and one
                 // warp synchronisation for the two stages.
                 const uint32_t row_sx = smem_base + C::b_offset(stage) + smem_row_sx;
-                if (valid) {
+                if constexpr (LATENT) {
+                  // Eq. 1 then Eq. 2 on the unit's 64 latent weights, in place: the same arithmetic, shortcut and
+                  // fallback as the stand-alone fake quantiser, so the operand is bit for bit the W_hat it would store.
+                  // (Rows or columns past the matrix were zero-filled by the copy and stay zero.)
+                  if (valid) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                      const int gsel = split_units ? h : 0;
+                      const float sv = ring_ls[j][gsel];
+                      const float zr = rintf(ring_lz[j][gsel]);
+                      const float rs = group_rcp(sv, zr);
+                      const float lo = -zr, hi = p.Q - zr;
+#pragma unroll
+                      for (int c = 4 * h; c < 4 * h + 4; ++c) {
+                        const uint32_t addr = row_sx ^ ((uint32_t)c << 4);
+                        float w[8], r[8], rt[8];
+                        unpack8(ptx::lds_128(addr), w);
+                        quotient_round8(w, sv, rs, r, rt);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) w[i] = fminf(fmaxf(r[i], lo), hi) * sv;
+                        const uint4 o = pack8(w);
+                        ptx::sts_128(addr, o.x, o.y, o.z, o.w);
+                      }
+                    }
+                  }
+                } else if (valid) {
                   GroupValues<BITS> gv[R][2];
 #pragma unroll
                   for (int u = 0; u < R; ++u) {
@@ -972,7 +1104,7 @@ int launch(const Operand& a, const Operand& b, const GemmParams& p, cudaStream_t
   if (!opt_in.ensure(kern, C::kSmemBytes)) return EQAT_ERR_CUDA;
   CUtensorMap ta, tb;
   if (!operand_tmap(&ta, a, C::kTileM)) return EQAT_ERR_CUDA;
-  if (PACKED) tb = ta;
+  if (PACKED && BITS != 16) tb = ta;                            // packed codes are fetched with ordinary loads
   else if (!operand_tmap(&tb, b, C::kBRows)) return EQAT_ERR_CUDA;
   const int sms = sm_count();
   if (sms < C::kCtas) return EQAT_ERR_CUDA;
@@ -1039,6 +1171,17 @@ void set_weight(GemmParams& p, const eqat_desc& d, const uint8_t* Wq, const eqat
   p.wq_sectors = (reinterpret_cast<uintptr_t>(Wq) & 31u) == 0 ? 1 : 0;
 }
 
+// Block-AP quantiser parameters for the kernels that fake-quantise the latent weight themselves.
+void set_latent(GemmParams& p, const eqat_desc& d, const eqat_bf16* W, const float* s, const float* z) {
+  p.W = W; p.s32 = s; p.z32 = z;
+  p.Q = (float)((1 << d.bits) - 1);
+  p.out_features = d.out_features;
+  p.in_features = d.in_features;
+  const bool whole_row = d.group == d.in_features && d.group > 256;
+  p.group_shift = whole_row ? 31 : log2_exact(d.group);
+  p.groups_per_row = d.in_features / d.group;
+}
+
 // Dense contraction with the plain store epilogue, over the three operand layouts.
 template <bool A_MN, bool B_MN>
 int launch_dense(const Operand& a, const Operand& b, GemmParams& p, cudaStream_t st) {
@@ -1099,6 +1242,26 @@ int launch_dense_dw_ste(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16
   // 128 rows per CTA: with two accumulator sets this epilogue, the longest of the three, runs under the next tile
   return p.M > 128 ? launch<1, true, true, false, EPI_STE, 2, true>(a, b, p, st)
                    : launch<1, true, true, false, EPI_STE, 2, false>(a, b, p, st);
+}
+
+int launch_latent_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* W, const float* s, const float* z,
+                      eqat_bf16* Y, cudaStream_t st) {
+  GemmParams p = base_params((int)d.tokens, d.out_features, d.in_features);
+  p.D = Y;
+  set_latent(p, d, W, s, z);
+  const Operand a{X, (uint64_t)d.tokens, (uint64_t)d.in_features, false}, b{W, (uint64_t)d.out_features, (uint64_t)d.in_features, false};
+  return p.M > 256 ? launch<2, false, false, true, EPI_STORE, 16, true>(a, b, p, st)
+                   : launch<2, false, false, true, EPI_STORE, 16, false>(a, b, p, st);
+}
+
+int launch_latent_dx(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* W, const float* s, const float* z,
+                     eqat_bf16* dX, cudaStream_t st) {
+  GemmParams p = base_params((int)d.tokens, d.in_features, d.out_features);
+  p.D = dX;
+  set_latent(p, d, W, s, z);
+  const Operand a{dY, (uint64_t)d.tokens, (uint64_t)d.out_features, false}, b{W, (uint64_t)d.in_features, (uint64_t)d.out_features, true};
+  return p.M > 256 ? launch<2, false, true, true, EPI_STORE, 16, true>(a, b, p, st)
+                   : launch<2, false, true, true, EPI_STORE, 16, false>(a, b, p, st);
 }
 
 int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,

@@ -15,6 +15,13 @@ int launch_dense_dw(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X,
 // the gradient of W_hat is never stored.
 int launch_dense_dw_ste(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* X, const eqat_bf16* W, const float* s,
                         const float* z, eqat_bf16* dW, float* ds, float* dz, cudaStream_t st);
+// Y = X * W_hat^T and dX = dY * W_hat with W_hat = Eq. 2 of Eq. 1 of the latent weight, computed inside the
+// kernel on each tile of W after it has been copied to shared memory; W_hat is not stored.  The group must be a
+// power of two up to 256 or the whole row.
+int launch_latent_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* W, const float* s, const float* z,
+                      eqat_bf16* Y, cudaStream_t st);
+int launch_latent_dx(const eqat_desc& d, const eqat_bf16* dY, const eqat_bf16* W, const float* s, const float* z,
+                     eqat_bf16* dX, cudaStream_t st);
 // Y = X * dequant(Wq)^T and dX = dY * dequant(Wq), codes expanded in shared memory.  zq: zero points as uint8 or,
 // with desc.zero_point_format == EQAT_ZP_FP16, as fp16 values.
 int launch_packed_fwd(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,

@@ -59,12 +59,16 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
-// Arrivals on a barrier given by its shared::cluster address (own CTA or the peer).
+// Arrivals on a barrier given by its shared::cluster address (own CTA or the peer).  They carry the default
+// (CTA-scope) release: what these barriers order is work of the asynchronous units, made visible by its own
+// fences (fence.proxy.async after shared-memory stores, tcgen05.fence after tensor-memory loads, byte counts of
+// bulk copies); a cluster-scope release here would also wait for the thread's outstanding global stores, which
+// measured a quarter slower on every kernel.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;"
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;"
                ::"r"(cluster_bar), "r"(bytes) : "memory");
 }
 
@@ -182,6 +186,13 @@ __device__ __forceinline__ void ldg_256(const void* p, uint32_t (&r)[8]) {
   asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                : "l"(p));
+}
+
+// 16-byte load from a 32-bit shared-memory address.
+__device__ __forceinline__ uint4 lds_128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
 }
 
 // 16-byte store to a 32-bit shared-memory address.
