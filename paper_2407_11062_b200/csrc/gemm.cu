@@ -1063,8 +1063,10 @@ EncodeFn encode_fn() {
   return fn;
 }
 
+}  // namespace
+
 // bf16 matrix [outer, inner] row-major; box = 64 elements (128 bytes) x box_outer rows, 128-byte swizzle.
-bool make_tmap(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer, uint32_t box_outer) {
+bool make_tmap_bf16(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer, uint32_t box_outer) {
   EncodeFn enc = encode_fn();
   if (enc == nullptr) return false;
   const cuuint64_t dims[2] = {inner, outer};
@@ -1074,6 +1076,12 @@ bool make_tmap(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer
   return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+
+bool make_tmap(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer, uint32_t box_outer) {
+  return make_tmap_bf16(tm, base, inner, outer, box_outer);
 }
 
 // How a contraction's tiles are shaped: rows per CTA (128 * mt) and whether pairs of CTAs share a tile.

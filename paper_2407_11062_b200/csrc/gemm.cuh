@@ -1,9 +1,14 @@
 // Host launchers of the tcgen05 GEMM kernels (arguments already validated).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include "eqat.h"
 
 namespace eqat {
+
+// Tensor map of a bf16 matrix [outer, inner] row-major for copies of 64 elements (128 bytes) x box_outer rows
+// with the 128-byte swizzle (the driver's encoder is looked up once; false if it is missing or refuses).
+bool make_tmap_bf16(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer, uint32_t box_outer);
 
 // Y[T,out] = X[T,in] * What[out,in]^T
 int launch_dense_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* What, eqat_bf16* Y, cudaStream_t st);

@@ -2,23 +2,33 @@
 // straight-through backward (Eqs. 3-5), min/max initialisation and quantise +
 // pack, for groups of at most 256 elements.
 //
-// These kernels are bound by HBM bandwidth, and what decides how close they
-// get to it is the number of bytes in flight per SM.  A plain "load, compute,
-// store" thread keeps its loads in flight only until its arithmetic starts,
-// and the arithmetic here is long (a division-free but exact quantiser per
-// element).  So the loads are taken out of the compute threads: each persistent
-// CTA has one producer thread that streams 8-16 KB chunks of the input(s) into
-// a four-stage shared-memory ring with bulk asynchronous copies (cp.async.bulk,
-// completion on an mbarrier), several chunks ahead, while 8 consumer warps pull
-// 16-byte vectors from the ring, compute, and write results to global memory
-// with coalesced 16-byte stores.  Three CTAs fit on an SM, so 150-190 KB of
-// reads are in flight per SM whatever the consumers are doing.
+// These kernels move 2-6 bytes per element and would be bound by HBM bandwidth
+// if the instruction stream per element were short enough; at 10-25 executed
+// instructions per element it is the issue rate of the SM that decides, so the
+// layout is chosen to keep everything that is per group or per access out of
+// the per-element count:
+//   * the loads are taken out of the compute threads altogether.  Each
+//     persistent CTA has one producer thread that streams 16 KB tiles of the
+//     input(s) into a shared-memory ring with tensor copies
+//     (cp.async.bulk.tensor, completion on an mbarrier) while 8 consumer warps
+//     compute; the flattened weight is described to the copy engine as a matrix
+//     of 128-byte rows with the 128-byte swizzle;
+//   * a consumer lane owns 32 CONSECUTIVE elements (half a row of the tile, four
+//     16-byte vectors, always inside one quantisation group), so the group's
+//     step size, zero point, reciprocal and clamp bounds are set up once per 32
+//     elements, the group sums need one shuffle per doubling of the group
+//     beyond 32, and the lane writes 64 contiguous bytes.  The swizzle makes
+//     the lanes' 16-byte shared-memory reads conflict-free although they are 64
+//     bytes apart.
+// Three CTAs fit on an SM (24 consumer warps, up to 190 KB of reads in flight).
 //
-// A quantisation group is contiguous in the flattened weight and owned by
-// group/8 adjacent lanes of one warp; group sums are fixed-order shuffles, so
+// Group sums are fixed-order (serial inside a lane, then a shuffle tree), so
 // results are run-to-run identical.
+#include <cuda.h>
+
 #include "common.cuh"
 #include "elementwise.cuh"
+#include "gemm.cuh"
 #include "ptx.cuh"
 #include "quant_math.cuh"
 
@@ -30,18 +40,19 @@ namespace {
 
 constexpr int kConsumers = 256;
 constexpr int kThreadsS = kConsumers + 32;           // + one producer warp
-// VPT = 16-byte vectors per consumer thread and chunk (a chunk is VPT * 4 KB per
-// input stream): 4 for the one-input fake quantiser, 2 for the two-input STE
-// backward, whose consumers need twice the registers per vector.
+constexpr int kLaneElems = 32;                       // consecutive elements per consumer lane and tile
+constexpr int kTileRows = kConsumers / 2;            // 128-byte rows per tile (two lanes per row)
+constexpr int kTileElems = kConsumers * kLaneElems;  // 8192
+constexpr int kTileBytes = kTileElems * 2;           // 16 KB per input stream
 constexpr uint64_t kStreamWaitLimitNs = 2000000000ull;
 
-template <int NIN, int VPT>
+template <int NIN>
 struct Ring {
-  static constexpr int kChunkVec = VPT * kConsumers;          // vectors per chunk and stream
-  static constexpr int kChunkBytes = kChunkVec * 16;
-  static constexpr int kStages = 4;
-  static constexpr int kStageBytes = NIN * kChunkBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 256;
+  // two-input kernels hold their inputs in registers while they compute, so two stages of 32 KB keep as many
+  // bytes in flight as four stages of 16 KB and leave room for three CTAs per SM
+  static constexpr int kStages = NIN == 1 ? 4 : 2;
+  static constexpr int kStageBytes = NIN * kTileBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*control block*/;
 };
 
 struct RingCtl {
@@ -71,29 +82,25 @@ __device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity, volatil
   return true;
 }
 
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-// Runs `body(v, raw, params)` on every consumer thread for every chunk this CTA
-// owns: v is the index of the thread's first vector, raw[i][u] the thread's
-// vector u (v + u * 256) of input stream i, and params what `fetch(v)` returned
-// for this chunk.  fetch is called one chunk ahead, so the small per-group loads
-// it makes (step size, zero point) are in flight while the previous chunk is
-// being computed instead of stalling this one.  Vectors at or beyond n_vec hold
-// stale shared memory and must be ignored by the body.
-template <int NIN, int VPT, typename Params, typename Fetch, typename Body>
-__device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], size_t n_vec, Fetch&& fetch,
-                                              Body&& body) {
-  using R = Ring<NIN, VPT>;
-  constexpr int kChunkVec = R::kChunkVec, kChunkBytes = R::kChunkBytes;
-  extern __shared__ __align__(128) uint8_t smem[];
-  RingCtl* ctl = reinterpret_cast<RingCtl*>(smem + R::kStages * R::kStageBytes);
+// Runs `body(e0, raw, params)` on every consumer lane for every tile this CTA
+// owns: e0 is the index of the lane's first element, raw[i][u] the lane's
+// vector u (elements e0 + 8u .. e0 + 8u + 7) of input stream i, and params what
+// `fetch(e0)` returned for this tile.  fetch is called one tile ahead, so the
+// small per-group loads it makes (step size, zero point) are in flight while
+// the previous tile is being computed.  The maps describe each input as
+// [n_elem / 64, 64] bf16; rows beyond the end read as zeros, and a lane whose
+// e0 is at or beyond n_elem must ignore its vectors.
+template <int NIN, typename Params, typename Fetch, typename Body>
+__device__ __forceinline__ void stream_tiles(const CUtensorMap* const (&maps)[NIN], size_t n_elem, Fetch&& fetch,
+                                             Body&& body) {
+  using R = Ring<NIN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+  const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;            // stages are 1024-byte aligned (swizzle period)
+  RingCtl* ctl = reinterpret_cast<RingCtl*>(smem_raw + (smem_base - raw_addr) + R::kStages * R::kStageBytes);
   volatile int* abort_flag = &ctl->abort;
-  const uint32_t smem_base = ptx::smem_addr(smem);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const size_t n_chunks = (n_vec + kChunkVec - 1) / kChunkVec;
+  const size_t n_tiles = (n_elem + kTileElems - 1) / kTileElems;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < R::kStages; ++s) {
@@ -108,22 +115,22 @@ __device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], 
   if (warp == kConsumers / 32) {
     // ---------------------------------------------------------------- producer
     if (lane == 0) {
+#pragma unroll
+      for (int i = 0; i < NIN; ++i) ptx::tma_prefetch_desc(maps[i]);
       int stage = 0;
       uint32_t phase = 0;
       size_t issued = 0;
       bool ok = true;
-      for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+      for (size_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         if (!ring_wait(ptx::smem_addr(&ctl->empty[stage]), phase ^ 1u, abort_flag, WAIT_STREAM_EMPTY, 32)) {
           ok = false;
           break;
         }
-        const size_t v0 = chunk * kChunkVec;
-        const uint32_t bytes = (uint32_t)((n_vec - v0 < (size_t)kChunkVec ? n_vec - v0 : (size_t)kChunkVec) * 16);
         const uint32_t full = ptx::smem_addr(&ctl->full[stage]);
-        ptx::mbar_expect_tx(full, NIN * bytes);
+        ptx::mbar_expect_tx(full, NIN * kTileBytes);               // rows past the end are zero-filled and counted
 #pragma unroll
         for (int i = 0; i < NIN; ++i)
-          bulk_load(smem_base + stage * R::kStageBytes + i * kChunkBytes, src[i] + v0 * 16, bytes, full);
+          ptx::tma_load_2d(smem_base + stage * R::kStageBytes + i * kTileBytes, maps[i], 0, (int)(tile * kTileRows), full);
         ++issued;
         if (++stage == R::kStages) { stage = 0; phase ^= 1u; }
       }
@@ -145,81 +152,87 @@ __device__ __forceinline__ void stream_chunks(const uint8_t* const (&src)[NIN], 
     }
   } else {
     // ---------------------------------------------------------------- consumers
+    // lane t owns half (t & 1) of row (t >> 1): 16-byte chunk c of a row sits at chunk (c ^ (row & 7))
+    const uint32_t row = threadIdx.x >> 1;
+    const uint32_t row_off = row * 128u, sx = row & 7u, c0 = (threadIdx.x & 1u) * 4u;
     int stage = 0;
     uint32_t phase = 0;
-    Params next = fetch((size_t)blockIdx.x * kChunkVec + threadIdx.x);
-    for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+    Params next = fetch((size_t)blockIdx.x * kTileElems + (size_t)threadIdx.x * kLaneElems);
+    for (size_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
       const Params cur = next;
-      if (chunk + gridDim.x < n_chunks) next = fetch((chunk + gridDim.x) * kChunkVec + threadIdx.x);
+      if (tile + gridDim.x < n_tiles) next = fetch((tile + gridDim.x) * kTileElems + (size_t)threadIdx.x * kLaneElems);
       // the lanes of a warp leave together: the bodies shuffle across the whole warp
       const bool got = ring_wait(ptx::smem_addr(&ctl->full[stage]), phase, abort_flag, WAIT_STREAM_FULL, 0);
       if (!__all_sync(0xFFFFFFFFu, got)) break;
-      uint4 raw[NIN][VPT];
-      const uint8_t* st = smem + stage * R::kStageBytes;
+      uint4 raw[NIN][4];
+      const uint32_t st = smem_base + stage * R::kStageBytes + row_off;
 #pragma unroll
       for (int i = 0; i < NIN; ++i)
 #pragma unroll
-        for (int u = 0; u < VPT; ++u)
-          raw[i][u] = *reinterpret_cast<const uint4*>(st + i * kChunkBytes + (u * kConsumers + threadIdx.x) * 16);
+        for (int u = 0; u < 4; ++u) raw[i][u] = ptx::lds_128(st + i * kTileBytes + (((c0 + u) ^ sx) << 4));
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->empty[stage]));   // the stage can be refilled now
       if (++stage == R::kStages) { stage = 0; phase ^= 1u; }
-      body(chunk * kChunkVec + threadIdx.x, raw, cur);
+      body(tile * kTileElems + (size_t)threadIdx.x * kLaneElems, raw, cur);
     }
   }
 }
 
-constexpr int kFakequantVpt = 4, kSteVpt = 2, kMinmaxVpt = 4, kPackVpt = 4;
-
-// Step size and zero point of the groups of a thread's vectors.
-template <int VPT>
+// Step size and (already rounded) zero point of the group a lane's elements belong to.
 struct GroupParams {
-  float s[VPT], z[VPT];
+  float s, z;
 };
 
-template <int VPT>
-__device__ __forceinline__ GroupParams<VPT> fetch_groups(const float* __restrict__ s, const float* __restrict__ z,
-                                                    size_t v0, size_t n_vec, int vec_shift) {
-  GroupParams<VPT> p;
-#pragma unroll
-  for (int u = 0; u < VPT; ++u) {
-    const size_t v = v0 + (size_t)u * kConsumers;
-    p.s[u] = 1.0f;
-    p.z[u] = 0.0f;
-    if (v < n_vec) {
-      p.s[u] = __ldg(s + (v >> vec_shift));
-      p.z[u] = __ldg(z + (v >> vec_shift));
-    }
+__device__ __forceinline__ GroupParams fetch_group(const float* __restrict__ s, const float* __restrict__ z, size_t e0,
+                                                   size_t n_elem, int group_shift) {
+  GroupParams p{1.0f, 0.0f};
+  if (e0 < n_elem) {
+    p.s = __ldg(s + (e0 >> group_shift));
+    p.z = __ldg(z + (e0 >> group_shift));
   }
   return p;
 }
 
+// A lane's 64 output bytes: two 32-byte stores where the tensor allows it, four 16-byte stores otherwise.
+__device__ __forceinline__ void store_lane(eqat_bf16* dst, const uint4 (&o)[4], bool wide) {
+  if (wide) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 16 * h), "r"(o[2 * h].x),
+                   "r"(o[2 * h].y), "r"(o[2 * h].z), "r"(o[2 * h].w), "r"(o[2 * h + 1].x), "r"(o[2 * h + 1].y),
+                   "r"(o[2 * h + 1].z), "r"(o[2 * h + 1].w) : "memory");
+  } else {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) reinterpret_cast<uint4*>(dst)[u] = o[u];
+  }
+}
+
 // ------------------------------------------------------------------ Eq. 1 + Eq. 2
 // (clamp(r + z, 0, Q) - z) * s == clamp(r, -z, Q - z) * s for integer r and z.
-__global__ void __launch_bounds__(kThreadsS)
-fakequant_stream_kernel(const eqat_bf16* __restrict__ W, const float* __restrict__ s, const float* __restrict__ z,
-                        eqat_bf16* __restrict__ What, size_t n_vec, int vec_shift, float Q) {
-  const uint8_t* const src[1] = {reinterpret_cast<const uint8_t*>(W)};
-  constexpr int VPT = kFakequantVpt;
-  stream_chunks<1, VPT, GroupParams<VPT>>(src, n_vec,
-      [&](size_t v0) { return fetch_groups<VPT>(s, z, v0, n_vec, vec_shift); },
-      [&](size_t v0, const uint4 (&raw)[1][VPT], const GroupParams<VPT>& gp) {
+__global__ void __launch_bounds__(kThreadsS, 3)
+fakequant_stream_kernel(const __grid_constant__ CUtensorMap map_w, const float* __restrict__ s,
+                        const float* __restrict__ z, eqat_bf16* __restrict__ What, size_t n_elem, int group_shift,
+                        float Q, int wide) {
+  const CUtensorMap* const maps[1] = {&map_w};
+  stream_tiles<1, GroupParams>(maps, n_elem,
+      [&](size_t e0) { return fetch_group(s, z, e0, n_elem, group_shift); },
+      [&](size_t e0, const uint4 (&raw)[1][4], const GroupParams& gp) {
+    if (e0 >= n_elem) return;
+    const float sv = gp.s;
+    const float zr = rintf(gp.z);
+    const float rs = group_rcp(sv, zr);
+    const float lo = -zr, hi = Q - zr;
+    uint4 o[4];
 #pragma unroll
-    for (int u = 0; u < VPT; ++u) {
-      const size_t v = v0 + (size_t)u * kConsumers;
-      if (v < n_vec) {
-        const float sv = gp.s[u];
-        const float zr = rintf(gp.z[u]);
-        const float rs = group_rcp(sv, zr);
-        const float lo = -zr, hi = Q - zr;
-        float w[8], r[8], rt[8];
-        unpack8(raw[0][u], w);
-        quotient_round8(w, sv, rs, r, rt);
+    for (int u = 0; u < 4; ++u) {
+      float w[8], r[8], rt[8];
+      unpack8(raw[0][u], w);
+      quotient_round8(w, sv, rs, r, rt);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) w[i] = fminf(fmaxf(r[i], lo), hi) * sv;
-        reinterpret_cast<uint4*>(What)[v] = pack8(w);
-      }
+      for (int i = 0; i < 8; ++i) w[i] = fminf(fmaxf(r[i], lo), hi) * sv;
+      o[u] = pack8(w);
     }
+    store_lane(What + e0, o, wide != 0);
   });
 }
 
@@ -227,29 +240,27 @@ fakequant_stream_kernel(const eqat_bf16* __restrict__ W, const float* __restrict
 // With lo = -z, hi = Q - z and c = clamp(r, lo, hi): the element is in range iff
 // c == r, and on the clamped branches Eq. 3's value (-z or Q - z) is c itself.
 // Eq. 4 is a constant per group times the sum of the gradient over the clamped
-// elements.  LPG = lanes per group (group / 8).
+// elements.  LPG = lanes per group (group / 32).
 template <int LPG>
-__global__ void __launch_bounds__(kThreadsS)
-ste_bwd_stream_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __restrict__ W,
+__global__ void __launch_bounds__(kThreadsS, 3)
+ste_bwd_stream_kernel(const __grid_constant__ CUtensorMap map_g, const __grid_constant__ CUtensorMap map_w,
                       const float* __restrict__ s, const float* __restrict__ z, eqat_bf16* __restrict__ dW,
-                      float* __restrict__ ds, float* __restrict__ dz, size_t n_vec, float Q, int dz_literal) {
-  const uint8_t* const src[2] = {reinterpret_cast<const uint8_t*>(dWhat), reinterpret_cast<const uint8_t*>(W)};
-  constexpr int vec_shift = LPG == 4 ? 2 : LPG == 8 ? 3 : LPG == 16 ? 4 : 5;
-  constexpr int VPT = kSteVpt;
-  stream_chunks<2, VPT, GroupParams<VPT>>(src, n_vec,
-      [&](size_t v0) { return fetch_groups<VPT>(s, z, v0, n_vec, vec_shift); },
-      [&](size_t v0, const uint4 (&raw)[2][VPT], const GroupParams<VPT>& gp) {
+                      float* __restrict__ ds, float* __restrict__ dz, size_t n_elem, float Q, int dz_literal, int wide) {
+  const CUtensorMap* const maps[2] = {&map_g, &map_w};
+  constexpr int group_shift = LPG == 1 ? 5 : LPG == 2 ? 6 : LPG == 4 ? 7 : 8;
+  stream_tiles<2, GroupParams>(maps, n_elem,
+      [&](size_t e0) { return fetch_group(s, z, e0, n_elem, group_shift); },
+      [&](size_t e0, const uint4 (&raw)[2][4], const GroupParams& gp) {
+    const bool live = e0 < n_elem;                      // uniform over the lanes of a group
+    float acc_s = 0.0f, acc_g = 0.0f;
+    const float sv = gp.s;
+    if (live) {
+      const float zr = rintf(gp.z);
+      const float rs = group_rcp(sv, zr);
+      const float lo = -zr, hi = Q - zr;
+      uint4 o[4];
 #pragma unroll
-    for (int u = 0; u < VPT; ++u) {
-      const size_t v = v0 + (size_t)u * kConsumers;
-      const bool live = v < n_vec;                      // uniform over the lanes of a group
-      const size_t g = v / LPG;
-      float acc_s = 0.0f, acc_g = 0.0f;
-      const float sv = gp.s[u];
-      if (live) {
-        const float zr = rintf(gp.z[u]);
-        const float rs = group_rcp(sv, zr);
-        const float lo = -zr, hi = Q - zr;
+      for (int u = 0; u < 4; ++u) {
         float gr[8], w[8], r[8], rt[8];
         unpack8(raw[0][u], gr);
         unpack8(raw[1][u], w);
@@ -262,17 +273,19 @@ ste_bwd_stream_kernel(const eqat_bf16* __restrict__ dWhat, const eqat_bf16* __re
           acc_g += inside ? 0.0f : gr[i];                      // Eq. 4
           w[i] = inside ? gr[i] : 0.0f;                        // Eq. 5
         }
-        reinterpret_cast<uint4*>(dW)[v] = pack8(w);
+        o[u] = pack8(w);
       }
+      store_lane(dW + e0, o, wide != 0);
+    }
 #pragma unroll
-      for (int d = LPG / 2; d >= 1; d >>= 1) {
-        acc_s += __shfl_xor_sync(0xFFFFFFFFu, acc_s, d);
-        acc_g += __shfl_xor_sync(0xFFFFFFFFu, acc_g, d);
-      }
-      if (live && (v % LPG) == 0) {
-        ds[g] = acc_s;
-        if (dz != nullptr) dz[g] = (dz_literal ? -1.0f : -sv) * acc_g;
-      }
+    for (int d = LPG / 2; d >= 1; d >>= 1) {
+      acc_s += __shfl_xor_sync(0xFFFFFFFFu, acc_s, d);
+      acc_g += __shfl_xor_sync(0xFFFFFFFFu, acc_g, d);
+    }
+    if (live && (threadIdx.x % LPG) == 0) {
+      const size_t g = e0 >> group_shift;
+      ds[g] = acc_s;
+      if (dz != nullptr) dz[g] = (dz_literal ? -1.0f : -sv) * acc_g;
     }
   });
 }
@@ -290,114 +303,94 @@ __device__ __forceinline__ uint32_t bf162_min(uint32_t a, uint32_t b) {
 }
 
 template <int LPG>
-__global__ void __launch_bounds__(kThreadsS)
-minmax_stream_kernel(const eqat_bf16* __restrict__ W, float* __restrict__ s, float* __restrict__ z, size_t n_vec,
-                     float Q) {
-  const uint8_t* const src[1] = {reinterpret_cast<const uint8_t*>(W)};
-  constexpr int VPT = kMinmaxVpt;
-  static_assert(kMinmaxVpt <= 4 && LPG >= 4, "one lane of a group finishes one of the thread's vectors");
-  stream_chunks<1, VPT, NoParams>(src, n_vec, [](size_t) { return NoParams{}; },
-      [&](size_t v0, const uint4 (&raw)[1][VPT], const NoParams&) {
-    // Reduce each of the thread's VPT vectors over the lanes of its group (every lane ends up with the
-    // group's extrema), then let lane u of the group finish vector u: one pass of the division code for
-    // all VPT groups instead of VPT passes with one active lane per group.
-    float mx_sel = 0.0f, mn_sel = 0.0f;
-    const int sub = threadIdx.x % LPG;
+__global__ void __launch_bounds__(kThreadsS, 3)
+minmax_stream_kernel(const __grid_constant__ CUtensorMap map_w, float* __restrict__ s, float* __restrict__ z,
+                     size_t n_elem, float Q) {
+  const CUtensorMap* const maps[1] = {&map_w};
+  constexpr int group_shift = LPG == 1 ? 5 : LPG == 2 ? 6 : LPG == 4 ? 7 : 8;
+  stream_tiles<1, NoParams>(maps, n_elem, [](size_t) { return NoParams{}; },
+      [&](size_t e0, const uint4 (&raw)[1][4], const NoParams&) {
+    // extrema on packed bf16 pairs (exact: comparisons only), widened to fp32 at the end
+    uint32_t mx2 = 0xFF80FF80u, mn2 = 0x7F807F80u;      // (-inf, -inf) and (+inf, +inf) as bf16 pairs
+    const bool live = e0 < n_elem;                      // uniform over the lanes of a group
+    if (live) {
 #pragma unroll
-    for (int u = 0; u < VPT; ++u) {
-      const size_t v = v0 + (size_t)u * kConsumers;
-      // extrema on packed bf16 pairs (exact: comparisons only), widened to fp32 at the end
-      uint32_t mx2 = 0xFF80FF80u, mn2 = 0x7F807F80u;    // (-inf, -inf) and (+inf, +inf) as bf16 pairs
-      if (v < n_vec) {                                  // uniform over the lanes of a group
+      for (int u = 0; u < 4; ++u) {
         const uint4 r4 = raw[0][u];
-        mx2 = bf162_max(bf162_max(r4.x, r4.y), bf162_max(r4.z, r4.w));
-        mn2 = bf162_min(bf162_min(r4.x, r4.y), bf162_min(r4.z, r4.w));
-      }
-#pragma unroll
-      for (int d = LPG / 2; d >= 1; d >>= 1) {
-        mx2 = bf162_max(mx2, __shfl_xor_sync(0xFFFFFFFFu, mx2, d));
-        mn2 = bf162_min(mn2, __shfl_xor_sync(0xFFFFFFFFu, mn2, d));
-      }
-      if (sub == u) {
-        mx_sel = fmaxf(__uint_as_float(mx2 << 16), __uint_as_float(mx2 & 0xFFFF0000u));
-        mn_sel = fminf(__uint_as_float(mn2 << 16), __uint_as_float(mn2 & 0xFFFF0000u));
+        mx2 = bf162_max(mx2, bf162_max(bf162_max(r4.x, r4.y), bf162_max(r4.z, r4.w)));
+        mn2 = bf162_min(mn2, bf162_min(bf162_min(r4.x, r4.y), bf162_min(r4.z, r4.w)));
       }
     }
-    const size_t v = v0 - sub + (size_t)sub * kConsumers;          // first vector of the group this lane finishes
-    if (sub < VPT && v < n_vec) {
+#pragma unroll
+    for (int d = LPG / 2; d >= 1; d >>= 1) {
+      mx2 = bf162_max(mx2, __shfl_xor_sync(0xFFFFFFFFu, mx2, d));
+      mn2 = bf162_min(mn2, __shfl_xor_sync(0xFFFFFFFFu, mn2, d));
+    }
+    if (live && (threadIdx.x % LPG) == 0) {
+      const float mx = fmaxf(__uint_as_float(mx2 << 16), __uint_as_float(mx2 & 0xFFFF0000u));
+      const float mn = fminf(__uint_as_float(mn2 << 16), __uint_as_float(mn2 & 0xFFFF0000u));
       // s = max((max - min) / Q, 2^-14), z = clamp(-round(min / s), 0, Q), all in binary32
-      float sv = __fdiv_rn(mx_sel - mn_sel, Q);
+      float sv = __fdiv_rn(mx - mn, Q);
       sv = fmaxf(sv, 6.103515625e-05f);
-      float zv = -rintf(__fdiv_rn(mn_sel, sv));
+      float zv = -rintf(__fdiv_rn(mn, sv));
       zv = fminf(fmaxf(zv, 0.0f), Q) + 0.0f;
-      s[v / LPG] = sv;
-      z[v / LPG] = zv;
+      s[e0 >> group_shift] = sv;
+      z[e0 >> group_shift] = zv;
     }
   });
 }
 
 // ------------------------------------------------------------------ quantise + pack (hand-off)
-// A thread turns one vector (8 weights) into 8*BITS bits; four adjacent lanes
-// hold 32 consecutive codes, which lane 0 of the four assembles into BITS
-// 32-bit words of the little-endian stream and stores.
+// A lane turns its 32 weights into 32 codes = BITS consecutive 32-bit words of the
+// little-endian stream (code j of the lane at bits [BITS*j, BITS*j + BITS)).
 template <int BITS>
-__global__ void __launch_bounds__(kThreadsS)
-quantize_pack_stream_kernel(const eqat_bf16* __restrict__ W, const float* __restrict__ s, const float* __restrict__ z,
-                            uint8_t* __restrict__ packed, uint8_t* __restrict__ z8, eqat_fp16* __restrict__ s16,
-                            size_t n_vec, int vec_shift) {
-  const uint8_t* const src[1] = {reinterpret_cast<const uint8_t*>(W)};
-  constexpr int VPT = kPackVpt;
+__global__ void __launch_bounds__(kThreadsS, 3)
+quantize_pack_stream_kernel(const __grid_constant__ CUtensorMap map_w, const float* __restrict__ s,
+                            const float* __restrict__ z, uint8_t* __restrict__ packed, uint8_t* __restrict__ z8,
+                            eqat_fp16* __restrict__ s16, size_t n_elem, int group_shift) {
+  const CUtensorMap* const maps[1] = {&map_w};
   constexpr float Q = (float)((1 << BITS) - 1);
-  stream_chunks<1, VPT, GroupParams<VPT>>(src, n_vec,
-      [&](size_t v0) { return fetch_groups<VPT>(s, z, v0, n_vec, vec_shift); },
-      [&](size_t v0, const uint4 (&raw)[1][VPT], const GroupParams<VPT>& gp) {
+  stream_tiles<1, GroupParams>(maps, n_elem,
+      [&](size_t e0) { return fetch_group(s, z, e0, n_elem, group_shift); },
+      [&](size_t e0, const uint4 (&raw)[1][4], const GroupParams& gp) {
+    if (e0 >= n_elem) return;
+    const float sv = gp.s;
+    const float zr = rintf(gp.z);
+    const float rs = group_rcp(sv, zr);
+    uint32_t piece[4];                                  // vector u's 8 codes, code i at bits [BITS*i, BITS*i + BITS)
 #pragma unroll
-    for (int u = 0; u < VPT; ++u) {
-      const size_t v = v0 + (size_t)u * kConsumers;
-      const bool live = v < n_vec;                      // uniform over each 4 adjacent lanes (n_vec % 4 == 0)
-      uint32_t piece = 0u;                              // this vector's 8 codes, code i at bits [BITS*i, BITS*i+BITS)
-      if (live) {
-        const float sv = gp.s[u];
-        const float zr = rintf(gp.z[u]);
-        const float rs = group_rcp(sv, zr);
-        float w[8], r[8], rt[8];
-        unpack8(raw[0][u], w);
-        quotient_round8(w, sv, rs, r, rt);
-        // The piece is sum_i code_i * 2^(BITS*i) with code_i = clamp(r_i + zr, 0, Q): evaluated by Horner's rule on the
-        // integer-valued floats (exact: below 2^24), with one conversion per 16 or 24 bits instead of an add, a mask,
-        // a shift and an or per code.
-        constexpr float kRadix = (float)(1 << BITS);
-        constexpr int kHalf = BITS == 4 ? 4 : 8;                                 // codes per conversion
+    for (int u = 0; u < 4; ++u) {
+      float w[8], r[8], rt[8];
+      unpack8(raw[0][u], w);
+      quotient_round8(w, sv, rs, r, rt);
+      // The piece is sum_i code_i * 2^(BITS*i) with code_i = clamp(r_i + zr, 0, Q): evaluated by Horner's rule on the
+      // integer-valued floats (exact: below 2^24), with one conversion per 16 or 24 bits instead of an add, a mask,
+      // a shift and an or per code.
+      constexpr float kRadix = (float)(1 << BITS);
+      constexpr int kHalf = BITS == 4 ? 4 : 8;                                 // codes per conversion
+      piece[u] = 0u;
 #pragma unroll
-        for (int h = 0; h < 8 / kHalf; ++h) {
-          float acc = fminf(fmaxf(r[h * kHalf + kHalf - 1] + zr, 0.0f), Q);
+      for (int h = 0; h < 8 / kHalf; ++h) {
+        float acc = fminf(fmaxf(r[h * kHalf + kHalf - 1] + zr, 0.0f), Q);
 #pragma unroll
-          for (int i = kHalf - 2; i >= 0; --i) acc = fmaf(acc, kRadix, fminf(fmaxf(r[h * kHalf + i] + zr, 0.0f), Q));
-          piece |= __float2uint_rn(acc) << (h * BITS * kHalf);
-        }
-        if ((v & (((size_t)1 << vec_shift) - 1)) == 0) {
-          const size_t g = v >> vec_shift;
-          z8[g] = (uint8_t)(__float_as_uint(fminf(fmaxf(zr, 0.0f), Q) + 8388608.0f) & 0xFFu);
-          s16[g] = __half_as_ushort(__float2half_rn(sv));
-        }
+        for (int i = kHalf - 2; i >= 0; --i) acc = fmaf(acc, kRadix, fminf(fmaxf(r[h * kHalf + i] + zr, 0.0f), Q));
+        piece[u] |= __float2uint_rn(acc) << (h * BITS * kHalf);
       }
-      if constexpr (BITS == 4) {
-        if (live) reinterpret_cast<uint32_t*>(packed)[v] = piece;                // 32 bits per vector: store directly
-      } else {
-        const uint32_t p1 = __shfl_down_sync(0xFFFFFFFFu, piece, 1);
-        const uint32_t p2 = __shfl_down_sync(0xFFFFFFFFu, piece, 2);
-        const uint32_t p3 = __shfl_down_sync(0xFFFFFFFFu, piece, 3);
-        if (live && (threadIdx.x & 3) == 0) {
-          if constexpr (BITS == 2) {
-            reinterpret_cast<uint2*>(packed)[v >> 2] = make_uint2(piece | (p1 << 16), p2 | (p3 << 16));
-          } else {
-            uint32_t* dst = reinterpret_cast<uint32_t*>(packed) + (v >> 2) * 3;
-            dst[0] = piece | (p1 << 24);
-            dst[1] = (p1 >> 8) | (p2 << 16);
-            dst[2] = (p2 >> 16) | (p3 << 8);
-          }
-        }
-      }
+    }
+    if ((e0 & (((size_t)1 << group_shift) - 1)) == 0) {
+      const size_t g = e0 >> group_shift;
+      z8[g] = (uint8_t)(__float_as_uint(fminf(fmaxf(zr, 0.0f), Q) + 8388608.0f) & 0xFFu);
+      s16[g] = __half_as_ushort(__float2half_rn(sv));
+    }
+    uint32_t* dst = reinterpret_cast<uint32_t*>(packed) + (e0 >> 5) * BITS;
+    if constexpr (BITS == 2) {
+      *reinterpret_cast<uint2*>(dst) = make_uint2(piece[0] | (piece[1] << 16), piece[2] | (piece[3] << 16));
+    } else if constexpr (BITS == 3) {
+      dst[0] = piece[0] | (piece[1] << 24);
+      dst[1] = (piece[1] >> 8) | (piece[2] << 16);
+      dst[2] = (piece[2] >> 16) | (piece[3] << 8);
+    } else {
+      *reinterpret_cast<uint4*>(dst) = make_uint4(piece[0], piece[1], piece[2], piece[3]);
     }
   });
 }
@@ -415,11 +408,18 @@ __global__ void ring_wait_expiry_kernel(uint64_t limit_ns) {
   (void)ring_wait(ptx::smem_addr(&bar), 0u, &abort_word, WAIT_SELFTEST, 0, limit_ns);
 }
 
-// Persistent grid: every CTA resident at once, never more CTAs than chunks.  The kernel is a template
+// The flattened [out, in] weight as rows of 64 elements, one tile of kTileRows rows per copy.
+inline bool weight_map(CUtensorMap* tm, const eqat_bf16* p, size_t n_elem) {
+  return make_tmap_bf16(tm, p, 64, n_elem / 64, kTileRows);
+}
+
+inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
+
+// Persistent grid: every CTA resident at once, never more CTAs than tiles.  The kernel is a template
 // argument so that each kernel has its own per-device state: the shared-memory opt-in and the number of
 // CTAs that fit on an SM (both asked of the runtime once per device).
 template <auto kernel, typename... Args>
-int launch_stream(int smem_bytes, int chunk_vec, size_t n_vec, cudaStream_t st, Args... args) {
+int launch_stream(int smem_bytes, size_t n_elem, cudaStream_t st, Args... args) {
   static SmemOptIn opt_in;
   static std::atomic<int> ctas_per_sm[kMaxCachedDevices];
   if (!opt_in.ensure(kernel, smem_bytes)) return EQAT_ERR_CUDA;
@@ -434,64 +434,72 @@ int launch_stream(int smem_bytes, int chunk_vec, size_t n_vec, cudaStream_t st, 
     }
     if (dev < kMaxCachedDevices) ctas_per_sm[dev].store(per_sm, std::memory_order_relaxed);
   }
-  const size_t chunks = (n_vec + chunk_vec - 1) / chunk_vec;
+  const size_t tiles = (n_elem + kTileElems - 1) / kTileElems;
   const size_t resident = (size_t)sms * per_sm;
-  const unsigned grid = (unsigned)(chunks < resident ? chunks : resident);
+  const unsigned grid = (unsigned)(tiles < resident ? tiles : resident);
   kernel<<<grid, kThreadsS, smem_bytes, st>>>(args...);
   return launch_status();
+}
+
+inline int group_shift_of(int group) {
+  int sh = 5;
+  while ((1 << sh) < group) ++sh;
+  return sh;
 }
 
 }  // namespace
 
 int launch_fakequant_stream(const eqat_desc& d, const eqat_bf16* W, const float* s, const float* z, eqat_bf16* What,
                             cudaStream_t st) {
-  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
+  const size_t n_elem = (size_t)d.out_features * d.in_features;
   const float Q = (float)((1 << d.bits) - 1);
-  int vec_shift = 0;
-  while ((8 << vec_shift) < d.group) ++vec_shift;
-  using R = Ring<1, kFakequantVpt>;
-  return launch_stream<fakequant_stream_kernel>(R::kSmemBytes, R::kChunkVec, n_vec, st, W, s, z, What, n_vec, vec_shift, Q);
+  CUtensorMap mw;
+  if (!weight_map(&mw, W, n_elem)) return EQAT_ERR_CUDA;
+  return launch_stream<fakequant_stream_kernel>(Ring<1>::kSmemBytes, n_elem, st, mw, s, z, What, n_elem,
+                                                group_shift_of(d.group), Q, (int)aligned32(What));
 }
 
 int launch_ste_bwd_stream(const eqat_desc& d, const eqat_bf16* dWhat, const eqat_bf16* W, const float* s,
                           const float* z, eqat_bf16* dW, float* ds, float* dz, cudaStream_t st) {
-  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
+  const size_t n_elem = (size_t)d.out_features * d.in_features;
   const float Q = (float)((1 << d.bits) - 1);
-  const int lit = d.dz_mode == 1;
-  using R = Ring<2, kSteVpt>;
-  constexpr int smem = R::kSmemBytes, cv = R::kChunkVec;
+  const int lit = d.dz_mode == 1, wide = (int)aligned32(dW);
+  CUtensorMap mg, mw;
+  if (!weight_map(&mg, dWhat, n_elem) || !weight_map(&mw, W, n_elem)) return EQAT_ERR_CUDA;
+  constexpr int smem = Ring<2>::kSmemBytes;
   switch (d.group) {
-    case 32:  return launch_stream<ste_bwd_stream_kernel<4>>(smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
-    case 64:  return launch_stream<ste_bwd_stream_kernel<8>>(smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
-    case 128: return launch_stream<ste_bwd_stream_kernel<16>>(smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
-    default:  return launch_stream<ste_bwd_stream_kernel<32>>(smem, cv, n_vec, st, dWhat, W, s, z, dW, ds, dz, n_vec, Q, lit);
+    case 32:  return launch_stream<ste_bwd_stream_kernel<1>>(smem, n_elem, st, mg, mw, s, z, dW, ds, dz, n_elem, Q, lit, wide);
+    case 64:  return launch_stream<ste_bwd_stream_kernel<2>>(smem, n_elem, st, mg, mw, s, z, dW, ds, dz, n_elem, Q, lit, wide);
+    case 128: return launch_stream<ste_bwd_stream_kernel<4>>(smem, n_elem, st, mg, mw, s, z, dW, ds, dz, n_elem, Q, lit, wide);
+    default:  return launch_stream<ste_bwd_stream_kernel<8>>(smem, n_elem, st, mg, mw, s, z, dW, ds, dz, n_elem, Q, lit, wide);
   }
 }
 
 int launch_minmax_stream(const eqat_desc& d, const eqat_bf16* W, float* s, float* z, cudaStream_t st) {
-  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
+  const size_t n_elem = (size_t)d.out_features * d.in_features;
   const float Q = (float)((1 << d.bits) - 1);
-  using R = Ring<1, kMinmaxVpt>;
-  constexpr int smem = R::kSmemBytes, cv = R::kChunkVec;
+  CUtensorMap mw;
+  if (!weight_map(&mw, W, n_elem)) return EQAT_ERR_CUDA;
+  constexpr int smem = Ring<1>::kSmemBytes;
   switch (d.group) {
-    case 32:  return launch_stream<minmax_stream_kernel<4>>(smem, cv, n_vec, st, W, s, z, n_vec, Q);
-    case 64:  return launch_stream<minmax_stream_kernel<8>>(smem, cv, n_vec, st, W, s, z, n_vec, Q);
-    case 128: return launch_stream<minmax_stream_kernel<16>>(smem, cv, n_vec, st, W, s, z, n_vec, Q);
-    default:  return launch_stream<minmax_stream_kernel<32>>(smem, cv, n_vec, st, W, s, z, n_vec, Q);
+    case 32:  return launch_stream<minmax_stream_kernel<1>>(smem, n_elem, st, mw, s, z, n_elem, Q);
+    case 64:  return launch_stream<minmax_stream_kernel<2>>(smem, n_elem, st, mw, s, z, n_elem, Q);
+    case 128: return launch_stream<minmax_stream_kernel<4>>(smem, n_elem, st, mw, s, z, n_elem, Q);
+    default:  return launch_stream<minmax_stream_kernel<8>>(smem, n_elem, st, mw, s, z, n_elem, Q);
   }
 }
 
 int launch_quantize_pack_stream(const eqat_desc& d, const eqat_bf16* W, const float* s, const float* z,
                                 uint8_t* packed, uint8_t* z8, eqat_fp16* s16, cudaStream_t st) {
-  const size_t n_vec = (size_t)d.out_features * d.in_features / 8;
-  int vec_shift = 0;
-  while ((8 << vec_shift) < d.group) ++vec_shift;
-  using R = Ring<1, kPackVpt>;
-  constexpr int smem = R::kSmemBytes, cv = R::kChunkVec;
+  const size_t n_elem = (size_t)d.out_features * d.in_features;
+  const int gs = group_shift_of(d.group);
+  CUtensorMap mw;
+  if (!weight_map(&mw, W, n_elem)) return EQAT_ERR_CUDA;
+  constexpr int smem = Ring<1>::kSmemBytes;
   switch (d.bits) {
-    case 2:  return launch_stream<quantize_pack_stream_kernel<2>>(smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
-    case 3:  return launch_stream<quantize_pack_stream_kernel<3>>(smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
-    default: return launch_stream<quantize_pack_stream_kernel<4>>(smem, cv, n_vec, st, W, s, z, packed, z8, s16, n_vec, vec_shift);
+    case 2:  return launch_stream<quantize_pack_stream_kernel<2>>(smem, n_elem, st, mw, s, z, packed, z8, s16, n_elem, gs);
+    case 3:  return launch_stream<quantize_pack_stream_kernel<3>>(smem, n_elem, st, mw, s, z, packed, z8, s16, n_elem, gs);
+    default: return launch_stream<quantize_pack_stream_kernel<4>>(smem, n_elem, st, mw, s, z, packed, z8, s16, n_elem, gs);
   }
 }
 
