@@ -592,6 +592,31 @@ def run_block_ap_forms(eqat, device, steps=10):
     return out
 
 
+def time_rotation(calls, rounds):
+    """Device time per launch (us) of `calls` issued in order, `rounds` times over: one pass is captured in a CUDA
+    graph (so the host's launch cost is not in the figure) and replayed between a pair of events on its stream."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for c in calls:
+            c()                                           # warm-up: one pass over every set, outside the capture
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for c in calls:
+                c()
+        graph.replay()
+        side.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        for _ in range(rounds):
+            graph.replay()
+        e1.record(side)
+        side.synchronize()
+    torch.cuda.current_stream().wait_stream(side)
+    return e0.elapsed_time(e1) * 1e3 / (rounds * len(calls))
+
+
 def run_streaming_leg(eqat, device, peaks, bits, group, shape=(11008, 4096), min_launches=56, min_bytes=640e6):
     """The five streaming kernels, each timed cold: `n` distinct sets of inputs and outputs whose combined size is
     several times the L2 (so no launch finds its operands or leaves its results in cache for the next one), at
@@ -635,27 +660,32 @@ def run_streaming_leg(eqat, device, peaks, bits, group, shape=(11008, 4096), min
                     del S["W"]
             sets.append(S)
         rounds = int(np.ceil(min_launches / n))
-        for S in sets:
-            S["call"]()                                   # warm-up: one pass over every set
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(rounds):
-            for S in sets:
-                S["call"]()
-        e1.record()
-        torch.cuda.synchronize()
+        us = time_rotation([S["call"] for S in sets], rounds)
         launches = rounds * n
-        us = e0.elapsed_time(e1) * 1e3 / launches
         r = hbm_roofline(nbytes / us / 1e3, peaks)
         r.update({"us_per_launch": us, "launches": launches, "distinct_buffer_sets": n,
                   "bytes_per_launch": nbytes, "bytes_touched_per_round": n * nbytes})
         res[name] = r
         del sets
         torch.cuda.empty_cache()
+    # yardstick: a device-to-device copy of the same weight (read 2 bytes, write 2 bytes per element), timed the same
+    # way on the same GPU in the same state; what a kernel with no arithmetic at all reaches at this size
+    n = max(4, int(np.ceil(min_bytes / (4 * n_elem))))
+    src = [torch.empty(out_f, in_f, dtype=bf, device=device).normal_(generator=g) for _ in range(n)]
+    dst = [torch.empty_like(t) for t in src]
+    rounds = int(np.ceil(min_launches / n))
+    us = time_rotation([lambda a=a, b=b: b.copy_(a) for a, b in zip(src, dst)], rounds)
+    yard = hbm_roofline(4 * n_elem / us / 1e3, peaks)
+    yard.update({"us_per_launch": us, "launches": rounds * n, "distinct_buffer_sets": n, "bytes_per_launch": 4.0 * n_elem,
+                 "what": "torch copy_ of one weight-sized bf16 tensor (not a kernel of this library)"})
+    for r in res.values():
+        r["frac_of_same_size_copy"] = r["achieved"] / yard["achieved"]
+    del src, dst
+    torch.cuda.empty_cache()
     return {"shape": f"{out_f} x {in_f}", "bits": bits, "group": group,
-            "method": "distinct input/output sets per launch (combined > 4 x L2), all launches between one pair of CUDA events",
-            "kernels": res}
+            "method": "distinct input/output sets per launch (combined > 4 x L2); the launches of one pass over the sets are "
+                      "captured in a CUDA graph and the graph is replayed back to back between one pair of CUDA events",
+            "kernels": res, "copy_yardstick": yard}
 
 
 # ----------------------------------------------------------------------------- main

@@ -45,12 +45,18 @@ constexpr int kTileRows = kConsumers / 2;            // 128-byte rows per tile (
 constexpr int kTileElems = kConsumers * kLaneElems;  // 8192
 constexpr int kTileBytes = kTileElems * 2;           // 16 KB per input stream
 constexpr uint64_t kStreamWaitLimitNs = 2000000000ull;
+// Ring depth and CTAs per SM.  The stage a consumer works on is released as soon as its vectors are in
+// registers, so a few stages are enough to keep the copy engine busy.
+#ifndef EQAT_STREAM_CTAS1
+#define EQAT_STREAM_CTAS1 3
+#define EQAT_STREAM_STAGES1 4
+#endif
+constexpr int kStages1 = EQAT_STREAM_STAGES1, kCtas1 = EQAT_STREAM_CTAS1;   // kernels with one input stream
+constexpr int kStages2 = 2, kCtas2 = 3;                                    // two input streams (32 KB per stage)
 
-template <int NIN>
+template <int NIN, int STAGES>
 struct Ring {
-  // two-input kernels hold their inputs in registers while they compute, so two stages of 32 KB keep as many
-  // bytes in flight as four stages of 16 KB and leave room for three CTAs per SM
-  static constexpr int kStages = NIN == 1 ? 4 : 2;
+  static constexpr int kStages = STAGES;
   static constexpr int kStageBytes = NIN * kTileBytes;
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*control block*/;
 };
@@ -90,10 +96,10 @@ __device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity, volatil
 // the previous tile is being computed.  The maps describe each input as
 // [n_elem / 64, 64] bf16; rows beyond the end read as zeros, and a lane whose
 // e0 is at or beyond n_elem must ignore its vectors.
-template <int NIN, typename Params, typename Fetch, typename Body>
+template <int NIN, int STAGES, typename Params, typename Fetch, typename Body>
 __device__ __forceinline__ void stream_tiles(const CUtensorMap* const (&maps)[NIN], size_t n_elem, Fetch&& fetch,
                                              Body&& body) {
-  using R = Ring<NIN>;
+  using R = Ring<NIN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_addr(smem_raw);
   const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;            // stages are 1024-byte aligned (swizzle period)
@@ -209,12 +215,12 @@ __device__ __forceinline__ void store_lane(eqat_bf16* dst, const uint4 (&o)[4], 
 
 // ------------------------------------------------------------------ Eq. 1 + Eq. 2
 // (clamp(r + z, 0, Q) - z) * s == clamp(r, -z, Q - z) * s for integer r and z.
-__global__ void __launch_bounds__(kThreadsS, 3)
+__global__ void __launch_bounds__(kThreadsS, kCtas1)
 fakequant_stream_kernel(const __grid_constant__ CUtensorMap map_w, const float* __restrict__ s,
                         const float* __restrict__ z, eqat_bf16* __restrict__ What, size_t n_elem, int group_shift,
                         float Q, int wide) {
   const CUtensorMap* const maps[1] = {&map_w};
-  stream_tiles<1, GroupParams>(maps, n_elem,
+  stream_tiles<1, kStages1, GroupParams>(maps, n_elem,
       [&](size_t e0) { return fetch_group(s, z, e0, n_elem, group_shift); },
       [&](size_t e0, const uint4 (&raw)[1][4], const GroupParams& gp) {
     if (e0 >= n_elem) return;
@@ -242,13 +248,13 @@ fakequant_stream_kernel(const __grid_constant__ CUtensorMap map_w, const float* 
 // Eq. 4 is a constant per group times the sum of the gradient over the clamped
 // elements.  LPG = lanes per group (group / 32).
 template <int LPG>
-__global__ void __launch_bounds__(kThreadsS, 3)
+__global__ void __launch_bounds__(kThreadsS, kCtas2)
 ste_bwd_stream_kernel(const __grid_constant__ CUtensorMap map_g, const __grid_constant__ CUtensorMap map_w,
                       const float* __restrict__ s, const float* __restrict__ z, eqat_bf16* __restrict__ dW,
                       float* __restrict__ ds, float* __restrict__ dz, size_t n_elem, float Q, int dz_literal, int wide) {
   const CUtensorMap* const maps[2] = {&map_g, &map_w};
   constexpr int group_shift = LPG == 1 ? 5 : LPG == 2 ? 6 : LPG == 4 ? 7 : 8;
-  stream_tiles<2, GroupParams>(maps, n_elem,
+  stream_tiles<2, kStages2, GroupParams>(maps, n_elem,
       [&](size_t e0) { return fetch_group(s, z, e0, n_elem, group_shift); },
       [&](size_t e0, const uint4 (&raw)[2][4], const GroupParams& gp) {
     const bool live = e0 < n_elem;                      // uniform over the lanes of a group
@@ -303,12 +309,12 @@ __device__ __forceinline__ uint32_t bf162_min(uint32_t a, uint32_t b) {
 }
 
 template <int LPG>
-__global__ void __launch_bounds__(kThreadsS, 3)
+__global__ void __launch_bounds__(kThreadsS, kCtas1)
 minmax_stream_kernel(const __grid_constant__ CUtensorMap map_w, float* __restrict__ s, float* __restrict__ z,
                      size_t n_elem, float Q) {
   const CUtensorMap* const maps[1] = {&map_w};
   constexpr int group_shift = LPG == 1 ? 5 : LPG == 2 ? 6 : LPG == 4 ? 7 : 8;
-  stream_tiles<1, NoParams>(maps, n_elem, [](size_t) { return NoParams{}; },
+  stream_tiles<1, kStages1, NoParams>(maps, n_elem, [](size_t) { return NoParams{}; },
       [&](size_t e0, const uint4 (&raw)[1][4], const NoParams&) {
     // extrema on packed bf16 pairs (exact: comparisons only), widened to fp32 at the end
     uint32_t mx2 = 0xFF80FF80u, mn2 = 0x7F807F80u;      // (-inf, -inf) and (+inf, +inf) as bf16 pairs
@@ -343,39 +349,69 @@ minmax_stream_kernel(const __grid_constant__ CUtensorMap map_w, float* __restric
 // ------------------------------------------------------------------ quantise + pack (hand-off)
 // A lane turns its 32 weights into 32 codes = BITS consecutive 32-bit words of the
 // little-endian stream (code j of the lane at bits [BITS*j, BITS*j + BITS)).
+//
+// Only the clamped code is wanted here, not r or r - w/s, which allows a shorter
+// exact evaluation of Eq. 1 than quotient_round8.  With cz = 2^23 + zr (an
+// integer) t = fma(w, rs, cz) rounds w*rs + zr to an integer held in the low
+// mantissa bits of t whenever the sum is in [0, 2^23), and lands below 2^23
+// (code 0 after the clamp) when it is negative.  The code is DEFINED through
+// y0 = rn(w / s).  Take the two reciprocals rs_lo = rs (1 - 2^-16) and
+// rs_hi = rs (1 + 2^-16), rs good to 1 ulp: the exact products w*rs_lo and
+// w*rs_hi enclose y0 with a margin of 2^-17 |y0| on either side, and rounding is
+// monotone, so when t_lo == t_hi every value between the products, y0 among
+// them, rounds to the same integer; y0 itself cannot be an exact tie then, since
+// a tie strictly inside the interval would separate t_lo from t_hi.  (The
+// integer added before rounding changes which neighbour a tie goes to, but a tie
+// never reaches this branch.)  When they differ (the quotient is within about
+// 2^-16 |y0| of a rounding boundary: a few elements per thousand) the element
+// is redone with the defining sequence.  Two multiply-adds and one logic
+// operation per element, and the clamped t feeds the bit packing directly: its
+// low bits ARE the code.
 template <int BITS>
-__global__ void __launch_bounds__(kThreadsS, 3)
+__global__ void __launch_bounds__(kThreadsS, kCtas1)
 quantize_pack_stream_kernel(const __grid_constant__ CUtensorMap map_w, const float* __restrict__ s,
                             const float* __restrict__ z, uint8_t* __restrict__ packed, uint8_t* __restrict__ z8,
                             eqat_fp16* __restrict__ s16, size_t n_elem, int group_shift) {
   const CUtensorMap* const maps[1] = {&map_w};
   constexpr float Q = (float)((1 << BITS) - 1);
-  stream_tiles<1, GroupParams>(maps, n_elem,
+  constexpr float kTwo23 = 8388608.0f;
+  // sum over the 8 codes of a vector of the bit pattern of 2^23 shifted to the code's place (mod 2^32)
+  constexpr uint32_t kBias = (uint32_t)(0x4B000000ull * (((1ull << (8 * BITS)) - 1ull) / ((1ull << BITS) - 1ull)));
+  stream_tiles<1, kStages1, GroupParams>(maps, n_elem,
       [&](size_t e0) { return fetch_group(s, z, e0, n_elem, group_shift); },
       [&](size_t e0, const uint4 (&raw)[1][4], const GroupParams& gp) {
     if (e0 >= n_elem) return;
     const float sv = gp.s;
     const float zr = rintf(gp.z);
-    const float rs = group_rcp(sv, zr);
+    const float rs = group_rcp(sv, zr);                 // NaN: the whole group takes the defining sequence
+    const bool exact_only = !(fabsf(rs) >= 2.5e-38f);   // (also when rs_lo would lose bits to underflow)
+    const float rs_lo = rs * 0.9999847412109375f, rs_hi = rs * 1.0000152587890625f;
+    const float cz = kTwo23 + zr;
     uint32_t piece[4];                                  // vector u's 8 codes, code i at bits [BITS*i, BITS*i + BITS)
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      float w[8], r[8], rt[8];
+      float w[8], t[8];
       unpack8(raw[0][u], w);
-      quotient_round8(w, sv, rs, r, rt);
-      // The piece is sum_i code_i * 2^(BITS*i) with code_i = clamp(r_i + zr, 0, Q): evaluated by Horner's rule on the
-      // integer-valued floats (exact: below 2^24), with one conversion per 16 or 24 bits instead of an add, a mask,
-      // a shift and an or per code.
-      constexpr float kRadix = (float)(1 << BITS);
-      constexpr int kHalf = BITS == 4 ? 4 : 8;                                 // codes per conversion
-      piece[u] = 0u;
+      uint32_t differ = exact_only ? 1u : 0u;
 #pragma unroll
-      for (int h = 0; h < 8 / kHalf; ++h) {
-        float acc = fminf(fmaxf(r[h * kHalf + kHalf - 1] + zr, 0.0f), Q);
-#pragma unroll
-        for (int i = kHalf - 2; i >= 0; --i) acc = fmaf(acc, kRadix, fminf(fmaxf(r[h * kHalf + i] + zr, 0.0f), Q));
-        piece[u] |= __float2uint_rn(acc) << (h * BITS * kHalf);
+      for (int i = 0; i < 8; ++i) {
+        t[i] = fmaf(w[i], rs_lo, cz);
+        differ |= __float_as_uint(t[i]) ^ __float_as_uint(fmaf(w[i], rs_hi, cz));
       }
+      if (differ != 0u) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (exact_only || !(t[i] == fmaf(w[i], rs_hi, cz))) {
+            const float r = rintf(__fdiv_rn(w[i], sv));
+            t[i] = (r + zr) + kTwo23;
+          }
+        }
+      }
+      uint32_t acc = 0u;
+#pragma unroll
+      for (int i = 7; i >= 0; --i)
+        acc = (acc << BITS) + __float_as_uint(fminf(fmaxf(t[i], kTwo23), kTwo23 + Q));
+      piece[u] = acc - kBias;
     }
     if ((e0 & (((size_t)1 << group_shift) - 1)) == 0) {
       const size_t g = e0 >> group_shift;
@@ -455,7 +491,7 @@ int launch_fakequant_stream(const eqat_desc& d, const eqat_bf16* W, const float*
   const float Q = (float)((1 << d.bits) - 1);
   CUtensorMap mw;
   if (!weight_map(&mw, W, n_elem)) return EQAT_ERR_CUDA;
-  return launch_stream<fakequant_stream_kernel>(Ring<1>::kSmemBytes, n_elem, st, mw, s, z, What, n_elem,
+  return launch_stream<fakequant_stream_kernel>(Ring<1, kStages1>::kSmemBytes, n_elem, st, mw, s, z, What, n_elem,
                                                 group_shift_of(d.group), Q, (int)aligned32(What));
 }
 
@@ -466,7 +502,7 @@ int launch_ste_bwd_stream(const eqat_desc& d, const eqat_bf16* dWhat, const eqat
   const int lit = d.dz_mode == 1, wide = (int)aligned32(dW);
   CUtensorMap mg, mw;
   if (!weight_map(&mg, dWhat, n_elem) || !weight_map(&mw, W, n_elem)) return EQAT_ERR_CUDA;
-  constexpr int smem = Ring<2>::kSmemBytes;
+  constexpr int smem = Ring<2, kStages2>::kSmemBytes;
   switch (d.group) {
     case 32:  return launch_stream<ste_bwd_stream_kernel<1>>(smem, n_elem, st, mg, mw, s, z, dW, ds, dz, n_elem, Q, lit, wide);
     case 64:  return launch_stream<ste_bwd_stream_kernel<2>>(smem, n_elem, st, mg, mw, s, z, dW, ds, dz, n_elem, Q, lit, wide);
@@ -480,7 +516,7 @@ int launch_minmax_stream(const eqat_desc& d, const eqat_bf16* W, float* s, float
   const float Q = (float)((1 << d.bits) - 1);
   CUtensorMap mw;
   if (!weight_map(&mw, W, n_elem)) return EQAT_ERR_CUDA;
-  constexpr int smem = Ring<1>::kSmemBytes;
+  constexpr int smem = Ring<1, kStages1>::kSmemBytes;
   switch (d.group) {
     case 32:  return launch_stream<minmax_stream_kernel<1>>(smem, n_elem, st, mw, s, z, n_elem, Q);
     case 64:  return launch_stream<minmax_stream_kernel<2>>(smem, n_elem, st, mw, s, z, n_elem, Q);
@@ -495,7 +531,7 @@ int launch_quantize_pack_stream(const eqat_desc& d, const eqat_bf16* W, const fl
   const int gs = group_shift_of(d.group);
   CUtensorMap mw;
   if (!weight_map(&mw, W, n_elem)) return EQAT_ERR_CUDA;
-  constexpr int smem = Ring<1>::kSmemBytes;
+  constexpr int smem = Ring<1, kStages1>::kSmemBytes;
   switch (d.bits) {
     case 2:  return launch_stream<quantize_pack_stream_kernel<2>>(smem, n_elem, st, mw, s, z, packed, z8, s16, n_elem, gs);
     case 3:  return launch_stream<quantize_pack_stream_kernel<3>>(smem, n_elem, st, mw, s, z, packed, z8, s16, n_elem, gs);
