@@ -104,10 +104,11 @@ size_t eqat_workspace_bytes(const eqat_desc* d, int op) {
 
 int eqat_device_status(int* h_status, int* h_detail) {
   if (h_status == nullptr) return EQAT_ERR_NULL;
-  int st[2] = {0, 0}, det[2] = {0, 0};
+  int st[3] = {0, 0, 0}, det[3] = {0, 0, 0};
   EQAT_TRY(read_device_status(&st[0], &det[0]));      // GEMM kernels
   EQAT_TRY(read_stream_status(&st[1], &det[1]));      // staged streaming kernels
-  const int k = st[0] != EQAT_OK ? 0 : 1;
+  EQAT_TRY(read_gemv_status(&st[2], &det[2]));        // matrix-vector kernels
+  const int k = st[0] != EQAT_OK ? 0 : (st[1] != EQAT_OK ? 1 : 2);
   *h_status = st[k];
   if (h_detail != nullptr) *h_detail = det[k];
   return EQAT_OK;

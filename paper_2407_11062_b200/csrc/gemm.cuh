@@ -9,6 +9,10 @@ namespace eqat {
 // Tensor map of a bf16 matrix [outer, inner] row-major for copies of 64 elements (128 bytes) x box_outer rows
 // with the 128-byte swizzle (the driver's encoder is looked up once; false if it is missing or refuses).
 bool make_tmap_bf16(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer, uint32_t box_outer);
+// Tensor map of a byte matrix [outer, inner_bytes] row-major for copies of box_bytes (at most 128) x box_outer
+// rows with the 128-byte swizzle; bytes outside the matrix are delivered as zeros.
+bool make_tmap_u8(CUtensorMap* tm, const void* base, uint64_t inner_bytes, uint64_t outer, uint32_t box_bytes,
+                  uint32_t box_outer);
 
 // Y[T,out] = X[T,in] * What[out,in]^T
 int launch_dense_fwd(const eqat_desc& d, const eqat_bf16* X, const eqat_bf16* What, eqat_bf16* Y, cudaStream_t st);

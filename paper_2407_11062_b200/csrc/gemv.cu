@@ -15,7 +15,10 @@
 // For a unit with step size s and zero point z
 //     sum_j (q_j - z) s x_j = s (2^N * sum_j (1 + q_j/2^N) x_j - (2^N + z) * sum_j x_j),
 // all in fp32, so the dequantised weight is never rounded to bf16 here.
+#include <cuda.h>
+
 #include "common.cuh"
+#include "gemm.cuh"
 #include "gemv.cuh"
 #include "ptx.cuh"
 
@@ -266,12 +269,491 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
   }
 }
 
+
+// ====================================================================== 2-bit codes on tensor-core tiles
+// The kernel above spends three instructions per code and token on the ordinary
+// cores.  For 2-bit codes that is several times what the bytes allow, so they go
+// through warp-level matrix instructions instead (mma.sync m16n8k16, bf16 in,
+// fp32 out): 16 weight rows by 16 columns against up to 8 tokens per
+// instruction, with the weight fragment built in registers, one logic
+// operation per PAIR of codes.  (The paired-CTA tensor-memory path of gemm.cu
+// wants its operands expanded into shared memory, which is exactly the cost to
+// avoid here; and with at most a few tokens there is nothing for a 128-row
+// accumulator to amortise.)
+//
+// Fragment construction.  A 32-bit word of the stream holds 16 consecutive codes
+// of one row, code j at bits [2j, 2j + 2).  (w >> 2p) & 0x00030003 isolates codes
+// p and p + 8 in the two halves of a register; OR-ing 0x4300 into each half makes
+// them the bf16 numbers 128 + q.  For p = 1, 2 (mod 3) the shift is skipped: a
+// code left at bits 2-3 (4-5) of a half with 0x4200 (0x4100) above it is the
+// bf16 number 32 + q (8 + q).  Eight registers from ten operations.  The added
+// constants and the zero point are taken out again by a fifth instruction per
+// chunk: with xb = sum of bias * x and xs = sum of x over the chunk's 64 columns,
+//     sum (q - z) x = sum (bias + q) x - (xb - 128 xs) - (128 + z) xs,
+// and the fifth instruction multiplies weights -1 and -(128 + z) (the bf16
+// pattern 0xC300 | z) with xb - 128 xs and xs, each given as the sum of three
+// bf16 numbers (24 significant bits: an fp32 value split without loss), so the
+// correction is as exact as if it were done in fp32 and the accumulator of a
+// chunk only remains to be scaled by the row's step size.
+//
+// Mapping.  A task is 16 consecutive weight rows over the whole of K; persistent
+// CTAs take tasks round-robin.  The producer thread copies the task's codes into
+// a shared-memory ring as [16 rows x 128 bytes] boxes (cp.async.bulk.tensor,
+// 128-byte swizzle, bytes past the end of a row arrive as zeros), eight boxes
+// per stage.  Consumer warp w owns half of box w/2 of every stage: four chunks of
+// 16 bytes = 64 columns = the four words of the four lanes of a quad, so a
+// chunk lies in one quantisation group and its accumulator is scaled by one step
+// size per row.  Lane (g, q) of the warp holds rows g and g + 8 and, in
+// instruction m of a chunk, supplies codes 2m, 2m+8, 2m+1, 2m+9 of its word;
+// the activations are staged once per CTA in exactly that order, so a lane
+// fetches its fragment of X with one 8-byte load.  Zero points are one byte
+// each here (the fp16 variant goes through the kernel above).  The 16 warps'
+// partial sums of a task go through a double-buffered shared array to a reducer
+// warp, which adds them in a fixed order and stores Y while the consumers are
+// on the next task.
+constexpr int kTcWarps = 16;
+constexpr int kTcThreads = (kTcWarps + 2) * 32;        // + producer warp + reducer warp
+constexpr int kTcRows = 16;                            // weight rows per task
+constexpr int kTcBoxBytes = 128;
+constexpr int kTcBoxesPerStage = 8;
+constexpr int kTcBoxSmem = kTcRows * kTcBoxBytes;      // 2 KB
+constexpr int kTcStageBytes = kTcBoxesPerStage * kTcBoxSmem;   // 16 KB: 16 rows x 1024 bytes
+constexpr int kTcAhead = 3;                            // stages of lead of the parameter loads
+constexpr int kTcItems = 5;                            // instructions per chunk: four on codes, one correction
+constexpr int kTcMaxStages = 8;
+constexpr int kTcMinStages = 3;
+constexpr uint64_t kTcWaitLimitNs = 2000000000ull;
+constexpr size_t kTcSmemBudget = 225 * 1024;
+
+struct TcCtl {
+  uint64_t full[kTcMaxStages];
+  uint64_t empty[kTcMaxStages];
+  uint64_t part_ready[2];
+  uint64_t part_free[2];
+  int abort;
+};
+
+struct TcLayout {
+  size_t xb_off, part_off, ctl_off, total;             // byte offsets from the 1024-byte aligned ring base
+  int stages;
+};
+
+// Shared-memory plan for T tokens and in_features columns.
+__host__ __device__ inline TcLayout tc_layout(int T, int in_features, int stages) {
+  TcLayout L;
+  // chunks of 64 columns, counted up to the end of the last (possibly partial) 512-column box: the entries past
+  // in_features are zeros, so the compute loop needs no end-of-row case
+  const size_t chunks = (size_t)((in_features + 511) / 512) * 8;
+  L.stages = stages;
+  L.xb_off = (size_t)stages * kTcStageBytes;
+  L.part_off = L.xb_off + chunks * kTcItems * 4 * T * 8;             // permuted bf16 activations + correction terms
+  L.ctl_off = L.part_off + (size_t)2 * kTcWarps * kTcRows * kGemvMaxTokens * 4;
+  L.total = L.ctl_off + sizeof(TcCtl) + 1024 /*alignment slack*/;
+  return L;
+}
+
+inline int tc_stages_that_fit(int T, int in_features) {
+  for (int st = kTcMaxStages; st >= kTcMinStages; --st)
+    if (tc_layout(T, in_features, st).total <= kTcSmemBudget) return st;
+  return 0;
+}
+
+__device__ int g_gemv_status[2];   // [0] = eqat_status, [1] = WaitSite
+
+__device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, volatile int* abort, int site, uint32_t sleep_ns) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = ptx::globaltimer_ns();
+  uint32_t n = 0;
+  while (!ptx::mbar_try_wait(bar, parity)) {
+    if (sleep_ns != 0) __nanosleep(sleep_ns);
+    if ((++n & 31u) == 0u) {
+      if (*abort) return false;
+      if (ptx::globaltimer_ns() - t0 > kTcWaitLimitNs) {
+        *abort = 1;
+        atomicExch(&g_gemv_status[1], site);
+        atomicExch(&g_gemv_status[0], (int)EQAT_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+// (t & mask) | magic on both halves of a register.
+__device__ __forceinline__ uint32_t and_or(uint32_t t, uint32_t mask, uint32_t magic) {
+  uint32_t r;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(t), "r"(mask), "r"(magic));
+  return r;
+}
+
+// D += A * B, A 16x16 (row), B 16x8 (col), bf16 inputs, fp32 accumulators.
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// The eight registers (codes p and p + 8 as bf16 pairs, p = 0..7) of one 16-code word.
+__device__ __forceinline__ void expand_word2(uint32_t w, uint32_t (&P)[8]) {
+  const uint32_t t1 = w >> 6, t2 = w >> 12;
+  P[0] = and_or(w, 0x00030003u, 0x43004300u);
+  P[1] = and_or(w, 0x000C000Cu, 0x42004200u);
+  P[2] = and_or(w, 0x00300030u, 0x41004100u);
+  P[3] = and_or(t1, 0x00030003u, 0x43004300u);
+  P[4] = and_or(t1, 0x000C000Cu, 0x42004200u);
+  P[5] = and_or(t1, 0x00300030u, 0x41004100u);
+  P[6] = and_or(t2, 0x00030003u, 0x43004300u);
+  P[7] = and_or(t2, 0x000C000Cu, 0x42004200u);
+}
+// Constant that expand_word2 adds to code j (0..15) of a word.
+__host__ __device__ inline float tc_bias(int j) {
+  const int r = (j & 7) % 3;
+  return r == 0 ? 128.0f : (r == 1 ? 32.0f : 8.0f);
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16* __restrict__ X,
+                      const eqat_fp16* __restrict__ s16, const uint8_t* __restrict__ z8, eqat_bf16* __restrict__ Y,
+                      int out_features, int in_features, int group_shift, int groups_per_row, int T, int vec_params,
+                      int stages) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+  const uint32_t ring_addr = (raw_addr + 1023u) & ~1023u;          // boxes are 1024-byte aligned (swizzle period)
+  uint8_t* ring = smem_raw + (ring_addr - raw_addr);
+  const TcLayout L = tc_layout(T, in_features, stages);
+  uint2* xb = reinterpret_cast<uint2*>(ring + L.xb_off);           // [chunk][item][quad lane][token] -> 4 bf16
+  float* part = reinterpret_cast<float*>(ring + L.part_off);       // [2][warp][row][kGemvMaxTokens]
+  TcCtl* ctl = reinterpret_cast<TcCtl*>(ring + L.ctl_off);
+  volatile int* abort_flag = &ctl->abort;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_tasks = out_features / kTcRows;
+  const int chunks = in_features >> 6;
+  const int row_bytes = in_features >> 2;
+  const int n_boxes = (row_bytes + kTcBoxBytes - 1) / kTcBoxBytes;
+  const int task_stages = (n_boxes + kTcBoxesPerStage - 1) / kTcBoxesPerStage;
+  const int chunks_pad = n_boxes * 8;
+
+  // Consumers request their first loads before anything else: the first unit of the activations and the step
+  // sizes / zero points of the first stages.  They are first touches of their pages in this launch, and once the
+  // weight stream is running a small load waits behind megabytes of bulk copies.
+  const int units = T * chunks_pad * 4;                                // (token, chunk, quad lane): 16 columns each
+  auto unit_src = [&](int u) -> const uint4* {
+    const int uq = u & 3, cg = (u >> 2) % chunks_pad, t = (u >> 2) / chunks_pad;
+    return cg < chunks ? reinterpret_cast<const uint4*>(X + (size_t)t * in_features + (size_t)cg * 64 + uq * 16) : nullptr;
+  };
+  uint4 x_first[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+  if (warp < kTcWarps && (int)threadIdx.x < units) {
+    const uint4* src = unit_src(threadIdx.x);
+    if (src != nullptr) { x_first[0] = __ldg(src); x_first[1] = __ldg(src + 1); }
+  }
+
+  const int g = lane >> 2, q = lane & 3;
+  const int box = warp >> 1, chunk0 = (warp & 1) * 4;
+  // Step sizes (four fp16) and zero points (four bytes) of this lane's four chunks of stage k of a task, rows g
+  // and g + 8.  With groups of 64 and rows of parameters that keep their alignment (vec_params) the four chunks
+  // are four consecutive groups: one load per row and kind.
+  struct StageParams { uint2 s_lo, s_hi; uint32_t z_lo, z_hi; };
+  auto fetch = [&](int task, int k) {
+    StageParams sp;
+    sp.s_lo = sp.s_hi = make_uint2(0u, 0u);
+    sp.z_lo = sp.z_hi = 0u;
+    const int cg0 = (k * kTcBoxesPerStage + box) * 8 + chunk0;
+    if (task < n_tasks && cg0 < chunks) {
+      const size_t p_lo = (size_t)(task * kTcRows + g) * groups_per_row, p_hi = p_lo + (size_t)8 * groups_per_row;
+      if (vec_params) {                                   // chunks is a multiple of 4 here: all four exist
+        sp.s_lo = __ldg(reinterpret_cast<const uint2*>(s16 + p_lo + cg0));
+        sp.s_hi = __ldg(reinterpret_cast<const uint2*>(s16 + p_hi + cg0));
+        sp.z_lo = __ldg(reinterpret_cast<const uint32_t*>(z8 + p_lo + cg0));
+        sp.z_hi = __ldg(reinterpret_cast<const uint32_t*>(z8 + p_hi + cg0));
+      } else {
+        uint32_t sl[4] = {0u, 0u, 0u, 0u}, sh[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (cg0 + c < chunks) {
+            const int grp = ((cg0 + c) << 6) >> group_shift;
+            sl[c] = __ldg(s16 + p_lo + grp);
+            sh[c] = __ldg(s16 + p_hi + grp);
+            sp.z_lo |= (uint32_t)__ldg(z8 + p_lo + grp) << (8 * c);
+            sp.z_hi |= (uint32_t)__ldg(z8 + p_hi + grp) << (8 * c);
+          }
+        }
+        sp.s_lo = make_uint2(sl[0] | (sl[1] << 16), sl[2] | (sl[3] << 16));
+        sp.s_hi = make_uint2(sh[0] | (sh[1] << 16), sh[2] | (sh[3] << 16));
+      }
+    }
+    return sp;
+  };
+  // kTcAhead stages of lead (the ring alone keeps 128 KB per SM in flight, so one stage is not enough)
+  StageParams nx[kTcAhead];
+  int pf_task = blockIdx.x, pf_k = 0;                     // next (task, stage) to request
+  auto advance = [&]() {
+    if (++pf_k == task_stages) { pf_k = 0; pf_task += gridDim.x; }
+  };
+#pragma unroll
+  for (int i = 0; i < kTcAhead; ++i) {
+    nx[i] = StageParams{make_uint2(0u, 0u), make_uint2(0u, 0u), 0u, 0u};
+    if (warp < kTcWarps) { nx[i] = fetch(pf_task, pf_k); advance(); }
+  }
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), 1);
+      ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), kTcWarps);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(ptx::smem_addr(&ctl->part_ready[b]), kTcWarps);
+      ptx::mbar_init(ptx::smem_addr(&ctl->part_free[b]), 1);
+    }
+    ctl->abort = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+
+  if (warp == kTcWarps) {
+    // ---------------------------------------------------------------- producer
+    if (lane == 0) {
+      ptx::tma_prefetch_desc(&map_w);
+      int slot = 0;
+      uint32_t phase = 0;
+      size_t issued = 0;
+      bool ok = true;
+      for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x) {
+        for (int k = 0; k < task_stages; ++k) {
+          if (!tc_wait(ptx::smem_addr(&ctl->empty[slot]), phase ^ 1u, abort_flag, WAIT_STREAM_EMPTY, 32)) {
+            ok = false;
+            break;
+          }
+          const int nb = min(kTcBoxesPerStage, n_boxes - k * kTcBoxesPerStage);
+          const uint32_t full = ptx::smem_addr(&ctl->full[slot]);
+          ptx::mbar_expect_tx(full, (uint32_t)nb * kTcBoxSmem);     // bytes past the end of a row are zero-filled and counted
+          for (int b = 0; b < nb; ++b)
+            ptx::tma_load_2d(ring_addr + slot * kTcStageBytes + b * kTcBoxSmem, &map_w,
+                             (k * kTcBoxesPerStage + b) * kTcBoxBytes, task * kTcRows, full);
+          ++issued;
+          if (++slot == stages) { slot = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok || *abort_flag) {
+        // every copy this thread started must land before the CTA exits
+        const size_t first = issued > (size_t)stages ? issued - stages : 0;
+        for (size_t i = first; i < issued; ++i) {
+          const uint32_t bar = ptx::smem_addr(&ctl->full[i % stages]);
+          const uint32_t par = (uint32_t)((i / stages) & 1);
+          const uint64_t t0 = ptx::globaltimer_ns();
+          while (!ptx::mbar_try_wait(bar, par)) {
+            if (ptx::globaltimer_ns() - t0 > 50000000ull) {
+              atomicExch(&g_gemv_status[1], (int)WAIT_TEARDOWN);
+              break;
+            }
+          }
+        }
+      }
+    }
+  } else if (warp == kTcWarps + 1) {
+    // ---------------------------------------------------------------- reducer
+    int buf = 0;
+    uint32_t ready_phase[2] = {0u, 0u};
+    for (int task = blockIdx.x; task < n_tasks; task += gridDim.x) {
+      const bool got = tc_wait(ptx::smem_addr(&ctl->part_ready[buf]), ready_phase[buf], abort_flag, WAIT_EPI_ACC_FULL, 0);
+      if (!__all_sync(0xFFFFFFFFu, got)) break;
+      for (int idx = lane; idx < kTcRows * T; idx += 32) {
+        const int r = idx & (kTcRows - 1), n = idx >> 4;
+        float v = 0.0f;
+#pragma unroll
+        for (int wv = 0; wv < kTcWarps; ++wv)              // fixed order: deterministic
+          v += part[((buf * kTcWarps + wv) * kTcRows + r) * kGemvMaxTokens + n];
+        Y[(size_t)n * out_features + (size_t)task * kTcRows + r] = (eqat_bf16)(pack_bf16x2(v, 0.0f) & 0xFFFFu);
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->part_free[buf]));
+      ready_phase[buf] ^= 1u;
+      buf ^= 1;
+    }
+  } else {
+    // ---------------------------------------------------------------- consumers
+    // Activations, in fragment order (zeros past in_features): unit (t, chunk, quad lane) = the 16 columns of that
+    // lane's word.
+    {
+      const int tid = threadIdx.x;                                     // 0 .. 511
+      for (int u0 = tid - lane; u0 < units; u0 += kTcWarps * 32) {     // warp-uniform bounds: the sums shuffle
+        const int u = u0 + lane;
+        const bool valid = u < units;
+        float sb = 0.0f, sx = 0.0f;
+        if (valid) {
+          const int uq = u & 3, cg = (u >> 2) % chunks_pad, t = (u >> 2) / chunks_pad;
+          uint4 v0 = x_first[0], v1 = x_first[1];
+          if (u0 >= kTcWarps * 32) {                                   // later rounds load here
+            const uint4* src = unit_src(u);
+            v0 = v1 = make_uint4(0u, 0u, 0u, 0u);
+            if (src != nullptr) { v0 = __ldg(src); v1 = __ldg(src + 1); }
+          }
+          const uint32_t r[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+          uint32_t h[16];                                              // column j of the word as 16 bits
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { h[2 * i] = r[i] & 0xFFFFu; h[2 * i + 1] = r[i] >> 16; }
+          float sb4[4] = {0.0f, 0.0f, 0.0f, 0.0f}, sx4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {                               // fixed order, four short chains
+            const float xv = __uint_as_float(h[j] << 16);
+            sb4[j & 3] = fmaf(tc_bias(j), xv, sb4[j & 3]);
+            sx4[j & 3] += xv;
+          }
+          sb = (sb4[0] + sb4[1]) + (sb4[2] + sb4[3]);
+          sx = (sx4[0] + sx4[1]) + (sx4[2] + sx4[3]);
+#pragma unroll
+          for (int m = 0; m < 4; ++m)
+            xb[(((size_t)cg * kTcItems + m) * 4 + uq) * T + t] =
+                make_uint2(h[2 * m] | (h[2 * m + 8] << 16), h[2 * m + 1] | (h[2 * m + 9] << 16));
+        }
+        sb += __shfl_xor_sync(0xFFFFFFFFu, sb, 1); sx += __shfl_xor_sync(0xFFFFFFFFu, sx, 1);
+        sb += __shfl_xor_sync(0xFFFFFFFFu, sb, 2); sx += __shfl_xor_sync(0xFFFFFFFFu, sx, 2);
+        if (valid && (u & 3) == 0) {
+          // correction item of the chunk: xb - 128 xs and xs, each as three bf16 numbers (round to nearest, the
+          // remainders are exact in fp32), in the slots of quad lanes 0 and 1; lanes 2 and 3 supply zeros
+          const int cg = (u >> 2) % chunks_pad, t = (u >> 2) / chunks_pad;
+          float v[2] = {fmaf(-128.0f, sx, sb), sx};
+          uint32_t parts[2][3];
+#pragma unroll
+          for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int pce = 0; pce < 3; ++pce) {
+              const uint32_t hb = pack_bf16x2(v[i], 0.0f) & 0xFFFFu;
+              parts[i][pce] = hb;
+              v[i] -= __uint_as_float(hb << 16);
+            }
+          uint2* item = xb + ((size_t)cg * kTcItems + 4) * 4 * T + t;
+          item[0 * T] = make_uint2(parts[0][0] | (parts[0][1] << 16), parts[0][2] | (parts[1][0] << 16));
+          item[1 * T] = make_uint2(parts[1][1] | (parts[1][2] << 16), 0u);
+          item[2 * T] = make_uint2(0u, 0u);
+          item[3 * T] = make_uint2(0u, 0u);
+        }
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(kTcWarps * 32) : "memory");
+    }
+
+    // Correction weights by quad lane: lane 0 holds slots 0, 1 (-1, -1) and 8, 9 (-1, -(128 + z)), lane 1 slots
+    // 2, 3 (-(128 + z) twice), lanes 2 and 3 zeros.  0xBF80 = -1, 0xC300 | z = -(128 + z) for z < 128.
+    const uint32_t mask_a = q == 1 ? 0x007F007Fu : 0u, const_a = q == 0 ? 0xBF80BF80u : (q == 1 ? 0xC300C300u : 0u);
+    const uint32_t mask_b = q == 0 ? 0x007F0000u : 0u, const_b = q == 0 ? 0xC300BF80u : 0u;
+    const uint2* xb_lane = xb + (size_t)q * T + g;                     // + chunk and item offsets
+    int slot = 0, buf = 0;
+    uint32_t phase = 0, free_phase[2] = {0u, 0u};
+    bool alive = true;
+    for (int task = blockIdx.x; task < n_tasks && alive; task += gridDim.x) {
+      float tot[4] = {0.0f, 0.0f, 0.0f, 0.0f};                         // rows g, g + 8 x tokens 2q, 2q + 1
+      for (int k = 0; k < task_stages; ++k) {
+        const int gbox = k * kTcBoxesPerStage + box;
+        const bool have = gbox < n_boxes;
+        const StageParams sp = nx[0];
+#pragma unroll
+        for (int i = 0; i + 1 < kTcAhead; ++i) nx[i] = nx[i + 1];
+        nx[kTcAhead - 1] = fetch(pf_task, pf_k);
+        advance();
+        const bool got = tc_wait(ptx::smem_addr(&ctl->full[slot]), phase, abort_flag, WAIT_STREAM_FULL, 0);
+        if (!__all_sync(0xFFFFFFFFu, got)) { alive = false; break; }
+        uint32_t w_lo[4], w_hi[4];
+        if (have) {
+          // 16-byte piece c of row r sits at piece (c ^ (r & 7)); rows g and g + 8 share the pattern
+          const uint32_t row = ring_addr + slot * kTcStageBytes + box * kTcBoxSmem + g * kTcBoxBytes + q * 4;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint32_t a = row + ((uint32_t)((chunk0 + c) ^ g) << 4);
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w_lo[c]) : "r"(a) : "memory");
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w_hi[c]) : "r"(a + 8 * kTcBoxBytes) : "memory");
+          }
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->empty[slot]));   // the stage can be refilled now
+        if (++slot == stages) { slot = 0; phase ^= 1u; }
+        if (have) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {                                // four independent chains, no branches
+            const int cg = gbox * 8 + chunk0 + c;
+            uint32_t PL[8], PH[8];
+            expand_word2(w_lo[c], PL);
+            expand_word2(w_hi[c], PH);
+            const uint2* item = xb_lane + (size_t)cg * (kTcItems * 4) * T;
+            float D[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+              uint2 b = make_uint2(0u, 0u);
+              if (g < T) b = item[m * 4 * T];
+              mma_16816(D, PL[2 * m], PH[2 * m], PL[2 * m + 1], PH[2 * m + 1], b.x, b.y);
+            }
+            {
+              // correction: weights -1 and -(128 + z) against the split sums (see the header)
+              const uint32_t zz_lo = ((sp.z_lo >> (8 * c)) & 0xFFu) * 0x10001u;
+              const uint32_t zz_hi = ((sp.z_hi >> (8 * c)) & 0xFFu) * 0x10001u;
+              uint2 b = make_uint2(0u, 0u);
+              if (g < T) b = item[4 * 4 * T];
+              mma_16816(D, and_or(zz_lo, mask_a, const_a), and_or(zz_hi, mask_a, const_a), and_or(zz_lo, mask_b, const_b),
+                        and_or(zz_hi, mask_b, const_b), b.x, b.y);
+            }
+            const uint32_t s2_lo = c < 2 ? sp.s_lo.x : sp.s_lo.y, s2_hi = c < 2 ? sp.s_hi.x : sp.s_hi.y;
+            const float s_lo = __half2float(__ushort_as_half((unsigned short)((c & 1) ? (s2_lo >> 16) : (s2_lo & 0xFFFFu))));
+            const float s_hi = __half2float(__ushort_as_half((unsigned short)((c & 1) ? (s2_hi >> 16) : (s2_hi & 0xFFFFu))));
+            tot[0] = fmaf(s_lo, D[0], tot[0]);
+            tot[1] = fmaf(s_lo, D[1], tot[1]);
+            tot[2] = fmaf(s_hi, D[2], tot[2]);
+            tot[3] = fmaf(s_hi, D[3], tot[3]);
+          }
+        }
+      }
+      if (!alive) break;
+      const bool free_ok = tc_wait(ptx::smem_addr(&ctl->part_free[buf]), free_phase[buf] ^ 1u, abort_flag,
+                                   WAIT_MMA_ACC_EMPTY, 0);
+      if (!__all_sync(0xFFFFFFFFu, free_ok)) break;
+      float* pw = part + (size_t)((buf * kTcWarps + warp) * kTcRows) * kGemvMaxTokens;
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int n = 2 * q + e;
+        if (n < T) {
+          pw[g * kGemvMaxTokens + n] = tot[e];
+          pw[(g + 8) * kGemvMaxTokens + n] = tot[2 + e];
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->part_ready[buf]));
+      free_phase[buf] ^= 1u;
+      buf ^= 1;
+    }
+  }
+}
+
+int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
+              eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
+  static SmemOptIn opt_in;
+  if (!opt_in.ensure(packed_gemv_tc_kernel, (int)kTcSmemBudget)) return EQAT_ERR_CUDA;
+  CUtensorMap mw;
+  if (!make_tmap_u8(&mw, Wq, (uint64_t)d.in_features / 4, (uint64_t)d.out_features, kTcBoxBytes, kTcRows)) return EQAT_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return EQAT_ERR_CUDA;
+  const int T = (int)d.tokens, n_tasks = d.out_features / kTcRows, ng = d.in_features / d.group;
+  // four consecutive groups of a row with one load each: groups of 64, rows of parameters that stay 8-byte
+  // (step sizes) and 4-byte (zero points) aligned
+  const int vec_params = (d.group == 64 && ng % 4 == 0 && (reinterpret_cast<uintptr_t>(s16) & 7u) == 0 &&
+                          (reinterpret_cast<uintptr_t>(zq) & 3u) == 0) ? 1 : 0;
+  const TcLayout L = tc_layout(T, d.in_features, stages);
+  packed_gemv_tc_kernel<<<n_tasks < sms ? n_tasks : sms, kTcThreads, L.total, st>>>(
+      mw, X, s16, static_cast<const uint8_t*>(zq), Y, d.out_features, d.in_features, group_shift, ng, T, vec_params, stages);
+  return launch_status();
+}
+
 }  // namespace
+
+// 2-bit codes with byte zero points go through the tensor-core kernel whenever its shared-memory plan fits.
+static int tc_stages_for(const eqat_desc& d) {
+  if (d.bits != 2 || d.group < 64 || d.tokens < 1 || d.tokens > kGemvMaxTokens) return 0;
+  if (d.zero_point_format != EQAT_ZP_U8) return 0;
+  return tc_stages_that_fit((int)d.tokens, d.in_features);
+}
 
 bool packed_gemv_applies(const eqat_desc& d) {
   // a 64-code unit must lie inside one group: groups of 32 go through the tiled kernel
-  return d.tokens >= 1 && d.tokens <= kGemvMaxTokens && d.group >= 64 &&
-         smem_floats((int)d.tokens, d.in_features) * sizeof(float) <= kMaxSmem;
+  if (d.tokens < 1 || d.tokens > kGemvMaxTokens || d.group < 64) return false;
+  return tc_stages_for(d) > 0 || smem_floats((int)d.tokens, d.in_features) * sizeof(float) <= kMaxSmem;
 }
 
 int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
@@ -281,11 +763,24 @@ int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq
     group_shift = 0;
     while ((1 << group_shift) < d.group) ++group_shift;
   }
+  const int tc_stages = tc_stages_for(d);
+  if (tc_stages > 0) return launch_tc(d, X, Wq, s16, zq, Y, group_shift, tc_stages, st);
   switch (d.bits) {
     case 2: return launch_bits<2>(d, X, Wq, s16, zq, Y, group_shift, st);
     case 3: return launch_bits<3>(d, X, Wq, s16, zq, Y, group_shift, st);
     default: return launch_bits<4>(d, X, Wq, s16, zq, Y, group_shift, st);
   }
+}
+
+int read_gemv_status(int* status, int* detail) {
+  int h[2] = {0, 0};
+  if (cudaDeviceSynchronize() != cudaSuccess) return EQAT_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(h, g_gemv_status, sizeof(h)) != cudaSuccess) return EQAT_ERR_CUDA;
+  const int zero[2] = {0, 0};
+  if (cudaMemcpyToSymbol(g_gemv_status, zero, sizeof(zero)) != cudaSuccess) return EQAT_ERR_CUDA;
+  *status = h[0];
+  *detail = h[1];
+  return EQAT_OK;
 }
 
 }  // namespace eqat
