@@ -61,10 +61,10 @@ EXTRA_CONFIGS = {
 # files change (comments and white space aside) the figures are stale and `roofline.traffic` is reported as null.
 NCU_TRAFFIC = {
     "sources": ("gemm.cu", "ptx.cuh"),
-    "sources_sha256": "3b2106bc3b7354efc28822654a030b5243cf54848a42562f6390b2b582091a92",
-    "packed_fwd": {"qkvo": 139.26e6 + 93.10e6, "gate_up": 147.72e6 + 314.19e6, "down": 448.65e6 + 114.63e6},
-    "packed_bwd_dx": {"qkvo": 139.26e6 + 93.85e6, "gate_up": 449.56e6 + 114.69e6, "down": 147.73e6 + 315.56e6},
-    "packed_bwd_ds": {"qkvo": 416.23e6 + 0.85e6, "gate_up": 1306.73e6 + 3.00e6, "down": 1073.39e6 + 2.82e6},
+    "sources_sha256": "c66b5e131c34943e0c94211e2485da9bbaa818df051387a7c0c3eb6dce73c425",
+    "packed_fwd": {"qkvo": 141.4e6 + 100.7e6, "gate_up": 163.5e6 + 315.0e6, "down": 502.9e6 + 116.0e6},
+    "packed_bwd_dx": {"qkvo": 140.7e6 + 100.1e6, "gate_up": 514.8e6 + 115.9e6, "down": 154.1e6 + 316.4e6},
+    "packed_bwd_ds": {"qkvo": 416.2e6 + 4.5e6, "gate_up": 1306.3e6 + 2.7e6, "down": 1073.8e6 + 2.9e6},
 }
 
 
@@ -799,6 +799,7 @@ def run_ours(args):
             # the other workloads and the cold streaming figures (one GPU is enough for them: the path is replicated)
             out["configs"] = {name: run_extra_config(eqat, device, name, spec, peaks) for name, spec in EXTRA_CONFIGS.items()}
             out["block_ap_forms"] = run_block_ap_forms(eqat, device)
+            out["few_tokens"] = decode_leg(eqat, device, peaks, 10)
             out["streaming"] = {"w2g64": run_streaming_leg(eqat, device, peaks, 2, 64),
                                 "w4g128": run_streaming_leg(eqat, device, peaks, 4, 128)}
             alias = {"fakequant_weight": "fakequant_weight", "ste_bwd": "ste_bwd", "minmax_init": "minmax_init_cold",
@@ -849,18 +850,13 @@ def run_streaming_case(args):
     print(json.dumps(r), flush=True)
 
 
-def run_decode_case(args):
-    """Few-token packed forward (the matrix-vector kernel) on the block's three linear shapes: device time per
+def decode_leg(eqat, dev, peaks, iters):
+    """Few-token packed forward (the matrix-vector kernels) on the block's three linear shapes: device time per
     launch from a CUDA graph of launches over rotating weight copies (more than L2 in total), and the bandwidth that
     time means for the bytes one launch must read."""
-    torch.cuda.set_device(0)
-    from paper_2407_11062_b200.build import build_library
-    build_library()
-    from paper_2407_11062_b200 import binding as eqat
-    peaks = load_peaks()
-    dev = torch.device("cuda", 0)
     out = {"metric": "packed forward, few tokens", "unit": "us per launch", "bits": BITS, "group": GROUP,
-           "hbm_gbs_peak": peaks["hbm_gbs"], "cases": {}}
+           "hbm_gbs_peak": peaks["hbm_gbs"],
+           "method": "CUDA graph of one launch per weight copy (copies total > 2 x L2), replayed back to back", "cases": {}}
     for lin in LINEARS["7b"]:
         o, i = lin.out_features, lin.in_features
         ng = i // GROUP
@@ -873,27 +869,22 @@ def run_decode_case(args):
             X = torch.randn(T, i, device=dev).to(torch.bfloat16)
             Y = torch.empty(T, o, dtype=torch.bfloat16, device=dev)
             d = eqat.make_desc(BITS, GROUP, o, i, T)
-            side = torch.cuda.Stream()
-            with torch.cuda.stream(side):
-                for P in Ps[:3]:
-                    eqat.qlinear_packed_fwd(d, X, P, s16, z8, Y)       # warm-up, outside the capture
-                side.synchronize()
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=side):
-                    for P in Ps:
-                        eqat.qlinear_packed_fwd(d, X, P, s16, z8, Y)
-                g.replay(); side.synchronize()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(side)
-                for _ in range(args.case_iters):
-                    g.replay()
-                e1.record(side)
-                side.synchronize()
-            us = e0.elapsed_time(e1) * 1e3 / (args.case_iters * copies)
+            us = time_rotation([lambda P=P: eqat.qlinear_packed_fwd(d, X, P, s16, z8, Y) for P in Ps], iters)
             nbytes = wbytes + o * ng * 3 + T * (i + o) * 2
             out["cases"][f"{lin.name}/T{T}"] = {"us": us, "bytes": nbytes, "gbs": nbytes / us / 1e3,
                                                  "frac_of_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
         del Ps
+        torch.cuda.empty_cache()
+    return out
+
+
+def run_decode_case(args):
+    """The few-token forward leg alone (for profiler captures and kernel work)."""
+    torch.cuda.set_device(0)
+    from paper_2407_11062_b200.build import build_library
+    build_library()
+    from paper_2407_11062_b200 import binding as eqat
+    out = decode_leg(eqat, torch.device("cuda", 0), load_peaks(), args.case_iters)
     assert eqat.device_status() == (0, 0)
     print(json.dumps(out), flush=True)
 

@@ -107,7 +107,8 @@ int eqat_device_status(int* h_status, int* h_detail);
  * EQAT_ERR_TIMEOUT in the device status word, abandons its work and returns
  * normally.  This call enqueues one warp that waits, with a limit of 1 ms, on a
  * barrier that nothing ever signals, through the very wait routine of the GEMM
- * kernels (which = 0) or of the streaming kernels (which = 1); afterwards
+ * kernels (which = 0), of the streaming kernels (which = 1) or of the
+ * few-token forward kernel (which = 2); afterwards
  * eqat_device_status() must report EQAT_ERR_TIMEOUT once and EQAT_OK from then
  * on.  It touches no tensor. */
 int eqat_selftest_wait_expiry(int which, void* stream);

@@ -117,6 +117,7 @@ int eqat_device_status(int* h_status, int* h_detail) {
 int eqat_selftest_wait_expiry(int which, void* stream) {
   if (which == 0) return launch_wait_expiry_gemm(as_stream(stream));
   if (which == 1) return launch_wait_expiry_stream(as_stream(stream));
+  if (which == 2) return launch_wait_expiry_gemv(as_stream(stream));
   return EQAT_ERR_UNSUPPORTED;
 }
 

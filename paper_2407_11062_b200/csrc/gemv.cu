@@ -360,7 +360,8 @@ inline int tc_stages_that_fit(int T, int in_features) {
 
 __device__ int g_gemv_status[2];   // [0] = eqat_status, [1] = WaitSite
 
-__device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, volatile int* abort, int site, uint32_t sleep_ns) {
+__device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, volatile int* abort, int site, uint32_t sleep_ns,
+                                        uint64_t limit_ns = kTcWaitLimitNs) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = ptx::globaltimer_ns();
   uint32_t n = 0;
@@ -368,7 +369,7 @@ __device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, volatile 
     if (sleep_ns != 0) __nanosleep(sleep_ns);
     if ((++n & 31u) == 0u) {
       if (*abort) return false;
-      if (ptx::globaltimer_ns() - t0 > kTcWaitLimitNs) {
+      if (ptx::globaltimer_ns() - t0 > limit_ns) {
         *abort = 1;
         atomicExch(&g_gemv_status[1], site);
         atomicExch(&g_gemv_status[0], (int)EQAT_ERR_TIMEOUT);
@@ -722,6 +723,19 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
   }
 }
 
+// The give-up path of tc_wait alone: one warp, a barrier nothing signals, a short limit.
+__global__ void tc_wait_expiry_kernel(uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_word;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_addr(&bar), 1);
+    abort_word = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  (void)tc_wait(ptx::smem_addr(&bar), 0u, &abort_word, WAIT_SELFTEST, 0, limit_ns);
+}
+
 int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
               eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
   static SmemOptIn opt_in;
@@ -770,6 +784,11 @@ int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq
     case 3: return launch_bits<3>(d, X, Wq, s16, zq, Y, group_shift, st);
     default: return launch_bits<4>(d, X, Wq, s16, zq, Y, group_shift, st);
   }
+}
+
+int launch_wait_expiry_gemv(cudaStream_t st) {
+  tc_wait_expiry_kernel<<<1, 32, 0, st>>>(1000000ull);   // 1 ms
+  return launch_status();
 }
 
 int read_gemv_status(int* status, int* detail) {

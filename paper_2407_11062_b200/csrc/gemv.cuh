@@ -14,6 +14,8 @@ bool packed_gemv_applies(const eqat_desc& d);
 int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
                        const void* zq, eqat_bf16* Y, cudaStream_t st);
 
+// Self-test of the matrix-vector kernel's bounded wait (one warp, 1 ms, a barrier nothing signals).
+int launch_wait_expiry_gemv(cudaStream_t st);
 // Reads and clears the status word of the matrix-vector kernels ({status, wait site}); synchronises.
 int read_gemv_status(int* status, int* detail);
 

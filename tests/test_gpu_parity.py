@@ -499,6 +499,10 @@ def test_few_token_forward_agrees_with_tiled_forward(eqat):
     (320, 1408, 1100, 2, 1408),     # one group per row with in_features not a power of two: 5.5 column tiles
     (192, 640, 3, 4, 640),          # one group per row through the few-token kernel
     (192, 640, 3, 2, 32),           # groups of 32 with few tokens: the tiled kernel
+    (128, 1152, 3, 2, 1152),        # 2-bit codes, one group per row, few tokens: the tensor-core matrix-vector kernel
+    (192, 768, 2, 2, 128),          # the same kernel with groups of 128 (two 64-column chunks per group) ...
+    (80 * 16, 4608, 1, 2, 256),     # ... and of 256; 80 row-blocks of 16 over several stages of the ring, 9 boxes per row
+    (2432, 512, 4, 2, 64),          # more row-blocks than SMs: every CTA takes a second task, parameters loaded as vectors
 ])
 def test_e2e_ragged(eqat, out, in_f, tokens, bits, group):
     cfg = small_cfg(f"e2er_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens)
@@ -593,7 +597,7 @@ def test_packed_weight_aligned_to_16_bytes_only(eqat, bits, tokens):
     assert rel_err(torch_to_f64(res[1][0]), O.linear_fwd(f32(Xb), What_o)) <= TOL
 
 
-@pytest.mark.parametrize("which,name", [(0, "GEMM kernels"), (1, "streaming kernels")])
+@pytest.mark.parametrize("which,name", [(0, "GEMM kernels"), (1, "streaming kernels"), (2, "matrix-vector kernel")])
 def test_a_bounded_wait_runs_out_cleanly(eqat, which, name):
     """One warp waits 1 ms for a barrier that nothing signals, through the kernels' own wait routine: the kernel
     must end normally, the status word must say TIMEOUT with the self-test's site code exactly once, and the
