@@ -865,7 +865,7 @@ def decode_leg(eqat, dev, peaks, iters):
         Ps = [torch.randint(0, 256, (o, i * BITS // 8), dtype=torch.uint8, device=dev) for _ in range(copies)]
         z8 = torch.randint(0, 1 << BITS, (o, ng), dtype=torch.uint8, device=dev)
         s16 = (torch.rand(o, ng, device=dev) * 0.01 + 0.001).half()
-        for T in (1, 4):
+        for T in (1, 4, 8):
             X = torch.randn(T, i, device=dev).to(torch.bfloat16)
             Y = torch.empty(T, o, dtype=torch.bfloat16, device=dev)
             d = eqat.make_desc(BITS, GROUP, o, i, T)

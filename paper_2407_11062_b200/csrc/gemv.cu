@@ -311,6 +311,7 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // partial sums of a task go through a double-buffered shared array to a reducer
 // warp, which adds them in a fixed order and stores Y while the consumers are
 // on the next task.
+constexpr int kTcMaxTokens = 8;                         // the instruction has eight token columns
 constexpr int kTcWarps = 16;
 constexpr int kTcThreads = (kTcWarps + 2) * 32;        // + producer warp + reducer warp
 constexpr int kTcRows = 16;                            // weight rows per task
@@ -347,7 +348,7 @@ __host__ __device__ inline TcLayout tc_layout(int T, int in_features, int stages
   L.stages = stages;
   L.xb_off = (size_t)stages * kTcStageBytes;
   L.part_off = L.xb_off + chunks * kTcItems * 4 * T * 8;             // permuted bf16 activations + correction terms
-  L.ctl_off = L.part_off + (size_t)2 * kTcWarps * kTcRows * kGemvMaxTokens * 4;
+  L.ctl_off = L.part_off + (size_t)2 * kTcWarps * kTcRows * kTcMaxTokens * 4;
   L.total = L.ctl_off + sizeof(TcCtl) + 1024 /*alignment slack*/;
   return L;
 }
@@ -425,7 +426,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
   uint8_t* ring = smem_raw + (ring_addr - raw_addr);
   const TcLayout L = tc_layout(T, in_features, stages);
   uint2* xb = reinterpret_cast<uint2*>(ring + L.xb_off);           // [chunk][item][quad lane][token] -> 4 bf16
-  float* part = reinterpret_cast<float*>(ring + L.part_off);       // [2][warp][row][kGemvMaxTokens]
+  float* part = reinterpret_cast<float*>(ring + L.part_off);       // [2][warp][row][kTcMaxTokens]
   TcCtl* ctl = reinterpret_cast<TcCtl*>(ring + L.ctl_off);
   volatile int* abort_flag = &ctl->abort;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -564,7 +565,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
         float v = 0.0f;
 #pragma unroll
         for (int wv = 0; wv < kTcWarps; ++wv)              // fixed order: deterministic
-          v += part[((buf * kTcWarps + wv) * kTcRows + r) * kGemvMaxTokens + n];
+          v += part[((buf * kTcWarps + wv) * kTcRows + r) * kTcMaxTokens + n];
         Y[(size_t)n * out_features + (size_t)task * kTcRows + r] = (eqat_bf16)(pack_bf16x2(v, 0.0f) & 0xFFFFu);
       }
       __syncwarp();
@@ -706,13 +707,13 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
       const bool free_ok = tc_wait(ptx::smem_addr(&ctl->part_free[buf]), free_phase[buf] ^ 1u, abort_flag,
                                    WAIT_MMA_ACC_EMPTY, 0);
       if (!__all_sync(0xFFFFFFFFu, free_ok)) break;
-      float* pw = part + (size_t)((buf * kTcWarps + warp) * kTcRows) * kGemvMaxTokens;
+      float* pw = part + (size_t)((buf * kTcWarps + warp) * kTcRows) * kTcMaxTokens;
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         const int n = 2 * q + e;
         if (n < T) {
-          pw[g * kGemvMaxTokens + n] = tot[e];
-          pw[(g + 8) * kGemvMaxTokens + n] = tot[2 + e];
+          pw[g * kTcMaxTokens + n] = tot[e];
+          pw[(g + 8) * kTcMaxTokens + n] = tot[2 + e];
         }
       }
       __syncwarp();
@@ -759,15 +760,16 @@ int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const e
 
 // 2-bit codes with byte zero points go through the tensor-core kernel whenever its shared-memory plan fits.
 static int tc_stages_for(const eqat_desc& d) {
-  if (d.bits != 2 || d.group < 64 || d.tokens < 1 || d.tokens > kGemvMaxTokens) return 0;
+  if (d.bits != 2 || d.group < 64 || d.tokens < 1 || d.tokens > kTcMaxTokens) return 0;
   if (d.zero_point_format != EQAT_ZP_U8) return 0;
   return tc_stages_that_fit((int)d.tokens, d.in_features);
 }
 
 bool packed_gemv_applies(const eqat_desc& d) {
   // a 64-code unit must lie inside one group: groups of 32 go through the tiled kernel
-  if (d.tokens < 1 || d.tokens > kGemvMaxTokens || d.group < 64) return false;
-  return tc_stages_for(d) > 0 || smem_floats((int)d.tokens, d.in_features) * sizeof(float) <= kMaxSmem;
+  if (d.tokens < 1 || d.group < 64) return false;
+  if (tc_stages_for(d) > 0) return true;                 // up to eight tokens
+  return d.tokens <= kGemvMaxTokens && smem_floats((int)d.tokens, d.in_features) * sizeof(float) <= kMaxSmem;
 }
 
 int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,

@@ -462,9 +462,10 @@ def test_e2e_small(eqat, bits, group, real_z):
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
-@pytest.mark.parametrize("tokens", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("tokens", [1, 2, 3, 4, 5, 7, 8, 9])
 def test_e2e_few_tokens(eqat, bits, tokens):
-    """Decode-sized batches: up to four tokens take the matrix-vector forward kernel, five the tiled one.
+    """Decode-sized batches: up to four tokens (eight for 2-bit codes) take a matrix-vector forward kernel, more the
+    tiled one.
     640 = 10 units of 64 columns, fewer than the sixteen warps of a CTA (some get none); 1408 = 22 (one or two each)."""
     group = 64 if bits == 2 else 128
     cfg = small_cfg(f"gemv_{bits}_{tokens}", 448, 640 if group == 64 else 1408, bits, group, tokens, "student_t4", 0.02, 0.01)
@@ -472,9 +473,9 @@ def test_e2e_few_tokens(eqat, bits, tokens):
 
 
 def test_few_token_forward_agrees_with_tiled_forward(eqat):
-    """The same rows through both forward kernels (4 tokens alone, and as the first rows of a 5-token batch)."""
-    cfg = small_cfg("gemv_vs_gemm", 512, 1024, 2, 64, 5)
-    r5 = run_e2e(eqat, cfg, cfg.linears[0], 5)
+    """The same rows through both forward kernels (4 tokens alone, and as the first rows of a 9-token batch)."""
+    cfg = small_cfg("gemv_vs_gemm", 512, 1024, 2, 64, 9)
+    r5 = run_e2e(eqat, cfg, cfg.linears[0], 9)
     cfg4 = small_cfg("gemv_vs_gemm", 512, 1024, 2, 64, 4)
     Wb = weight_for(cfg4, cfg4.linears[0])
     assert np.array_equal(Wb, weight_for(cfg, cfg.linears[0]))
