@@ -57,7 +57,21 @@ def variants(W32, bits, group):
 @pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("group", [32, 64, 128, 256, 512])
 def test_minmax_fakequant_ste_pack(eqat, bits, group):
-    out, in_f = 192, 512                      # 98304 elements: several blocks and a ragged last block
+    check_streaming_kernels(eqat, bits, group, 192, 512)      # 98304 elements: twelve tiles of 8192
+
+
+@pytest.mark.parametrize("out,in_f,bits,group", [
+    (1, 128, 2, 64),          # two 128-byte rows: far less than one tile of the copy engine, four live lanes
+    (3, 384, 3, 128),         # 1152 elements, 36 live lanes
+    (1, 256, 4, 256),         # a single group spread over eight lanes
+    (65, 8320, 2, 32),        # 66 tiles and a ragged last one (540800 = 66 * 8192 + 128 elements), groups of 32
+    (7, 1152, 2, 1152),       # one group per row, rows that are no power of two (the long-group kernels)
+])
+def test_streaming_kernels_tiny_and_ragged(eqat, out, in_f, bits, group):
+    check_streaming_kernels(eqat, bits, group, out, in_f)
+
+
+def check_streaming_kernels(eqat, bits, group, out, in_f):
     cfg = small_cfg(f"ew_{bits}_{group}", out, in_f, bits, group, 0, "student_t4", 0.02, 0.01)
     Wb = weight_for(cfg, cfg.linears[0]); W32 = f32(Wb)
     d = eqat.make_desc(bits, group, out, in_f)
@@ -503,6 +517,8 @@ def test_few_token_forward_agrees_with_tiled_forward(eqat):
     (128, 1152, 3, 2, 1152),        # 2-bit codes, one group per row, few tokens: the tensor-core matrix-vector kernel
     (192, 768, 2, 2, 128),          # the same kernel with groups of 128 (two 64-column chunks per group) ...
     (80 * 16, 4608, 1, 2, 256),     # ... and of 256; 80 row-blocks of 16 over several stages of the ring, 9 boxes per row
+    (64, 128, 1, 2, 64),            # rows of 32 bytes: a quarter of the copy engine's 128-byte box
+    (64, 256, 8, 2, 128),           # eight tokens, the most the matrix-vector kernel takes
     (2432, 512, 4, 2, 64),          # more row-blocks than SMs: every CTA takes a second task, parameters loaded as vectors
 ])
 def test_e2e_ragged(eqat, out, in_f, tokens, bits, group):
