@@ -264,6 +264,16 @@ def test_quotients_far_out_of_range_and_zero_points_off_the_grid(eqat):
     What_o = bf16_round(((q_o - np.repeat(z, group, 1)).astype(np.float32) * np.repeat(s, group, 1)).astype(np.float32))
     bad = np.argwhere(torch_to_f64(What) != What_o.astype(np.float64))
     assert bad.size == 0, (bad[:5], [(W32[i, j], s[i, j // group], z[i, j // group]) for i, j in bad[:5]])
+    # the hand-off takes the same decisions (its exactness test is a different one: two bracketing reciprocals)
+    P = torch.empty(out, in_f * bits // 8, dtype=torch.uint8, device="cuda")
+    z8 = torch.empty(out, in_f // group, dtype=torch.uint8, device="cuda")
+    s16 = torch.empty(out, in_f // group, dtype=torch.float16, device="cuda")
+    eqat.eqat_quantize_pack(d, bits_to_torch(Wb), dev(s), dev(z), P, z8, s16)
+    codes = torch.empty(out, in_f, dtype=torch.uint8, device="cuda")
+    eqat.eqat_unpack(d, P, codes)
+    badq = np.argwhere(codes.cpu().numpy() != q_o.astype(np.uint8))
+    assert badq.size == 0, (badq[:5], [(W32[i, j], s[i, j // group], z[i, j // group]) for i, j in badq[:5]])
+    assert np.array_equal(z8.cpu().numpy(), np.clip(z, 0, (1 << bits) - 1).astype(np.uint8))
     G = np.ones_like(W32); dW = torch.empty_like(What)
     ds = torch.empty(out, in_f // group, device="cuda")
     eqat.eqat_ste_bwd(d, bits_to_torch(to_bf16_bits(G)), bits_to_torch(Wb), dev(s), dev(z), dW, ds, None)
