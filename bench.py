@@ -823,7 +823,8 @@ def run_kernel_case(args):
     mode = args.case_mode
     wl = BlockWorkload(eqat, torch.device("cuda", 0), seed=1, model=args.case_model, bits=args.case_bits, group=args.case_group,
                        t_block_ap=args.case_tokens if mode in ("both", "block_ap") else 0,
-                       t_e2e=args.case_tokens if mode in ("both", "e2e_qp") else 0, handoff=(mode == "both"))
+                       t_e2e=args.case_tokens if mode in ("both", "e2e_qp") else 0, handoff=(mode == "both"),
+                       store_w_hat=not args.case_no_w_hat)
     wl.layers = [L for L in wl.layers if L["shape"] == args.case_shape][:1]
     assert wl.layers, f"no linear named {args.case_shape} in model {args.case_model}"
     for _ in range(2):
@@ -902,6 +903,8 @@ def main():
     ap.add_argument("--case-group", type=int, default=GROUP)
     ap.add_argument("--case-mode", default="both", choices=["both", "block_ap", "e2e_qp"])
     ap.add_argument("--case-iters", type=int, default=2)
+    ap.add_argument("--case-no-w-hat", action="store_true",
+                    help="kernel case: Block-AP without a stored W_hat (Eq. 1-2 inside the forward and dX GEMMs)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
