@@ -527,6 +527,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
             ok = false;
             break;
           }
+          ptx::fence_proxy_async_smem();                            // consumers' reads of this stage before the copies' writes
           const int nb = min(kTcBoxesPerStage, n_boxes - k * kTcBoxesPerStage);
           const uint32_t full = ptx::smem_addr(&ctl->full[slot]);
           ptx::mbar_expect_tx(full, (uint32_t)nb * kTcBoxSmem);     // bytes past the end of a row are zero-filled and counted
@@ -666,6 +667,9 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w_hi[c]) : "r"(a + 8 * kTcBoxBytes) : "memory");
           }
         }
+        // The stage's next user is a copy of the asynchronous proxy, which the barrier alone does not order after
+        // these generic-proxy reads: the readers fence here, the producer again between its wait and the copy.
+        ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->empty[slot]));   // the stage can be refilled now
         if (++slot == stages) { slot = 0; phase ^= 1u; }

@@ -132,6 +132,7 @@ __device__ __forceinline__ void stream_tiles(const CUtensorMap* const (&maps)[NI
           ok = false;
           break;
         }
+        ptx::fence_proxy_async_smem();                             // consumers' reads of this stage before the copy's writes
         const uint32_t full = ptx::smem_addr(&ctl->full[stage]);
         ptx::mbar_expect_tx(full, NIN * kTileBytes);               // rows past the end are zero-filled and counted
 #pragma unroll
@@ -176,6 +177,11 @@ __device__ __forceinline__ void stream_tiles(const CUtensorMap* const (&maps)[NI
       for (int i = 0; i < NIN; ++i)
 #pragma unroll
         for (int u = 0; u < 4; ++u) raw[i][u] = ptx::lds_128(st + i * kTileBytes + (((c0 + u) ^ sx) << 4));
+      // The stage is handed back before the compute.  Its next user is a copy of the asynchronous proxy, which
+      // is not ordered after these generic-proxy reads by the barrier alone: without a proxy fence on the way
+      // a few lanes read rows of the tile four steps ahead (seen on 8192 x 8192 weights with three CTAs per SM).
+      // The readers fence here, and the producer fences again between its wait and the copy.
+      ptx::fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->empty[stage]));   // the stage can be refilled now
       if (++stage == R::kStages) { stage = 0; phase ^= 1u; }

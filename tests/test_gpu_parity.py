@@ -282,6 +282,51 @@ def test_quotients_far_out_of_range_and_zero_points_off_the_grid(eqat):
     assert dW_o.sum() > 1000 and (dW_o == 0).sum() > 1000                  # both branches well populated
 
 
+def test_streaming_kernels_repeat_bit_for_bit_on_a_large_weight(eqat):
+    """Nine or more tiles per CTA, so every stage of the shared-memory ring is reused several times while the
+    consumers run ahead of one another.  A stage that is refilled before all of its readers are done (the
+    copy engine's writes are not ordered after ordinary reads without a proxy fence) shows up as a few stale
+    rows in some launches, so every kernel is launched a dozen times and must reproduce its first result bit
+    for bit; the first result is checked against the oracle on sampled rows."""
+    out, in_f, bits, group = 4096, 8192, 2, 64
+    ng = in_f // group
+    g = torch.Generator(device="cuda"); g.manual_seed(20240711)
+    Wd = (torch.randn(out, in_f, device="cuda", generator=g) * 0.02).to(torch.bfloat16)
+    Gd = (torch.randn(out, in_f, device="cuda", generator=g) * 0.01).to(torch.bfloat16)
+    d = eqat.make_desc(bits, group, out, in_f)
+
+    def run():
+        s = torch.empty(out, ng, device="cuda"); z = torch.empty(out, ng, device="cuda")
+        eqat.eqat_minmax_init(d, Wd, s, z)
+        What = torch.empty(out, in_f, dtype=torch.bfloat16, device="cuda"); dW = torch.empty_like(What)
+        ds = torch.empty(out, ng, device="cuda"); dz = torch.empty(out, ng, device="cuda")
+        P = torch.empty(out, in_f * bits // 8, dtype=torch.uint8, device="cuda")
+        z8 = torch.empty(out, ng, dtype=torch.uint8, device="cuda")
+        s16 = torch.empty(out, ng, dtype=torch.float16, device="cuda")
+        eqat.eqat_fakequant_weight(d, Wd, s, z, What)
+        eqat.eqat_ste_bwd(d, Gd, Wd, s, z, dW, ds, dz)
+        eqat.eqat_quantize_pack(d, Wd, s, z, P, z8, s16)
+        torch.cuda.synchronize()
+        return dict(s=s, z=z, What=What, dW=dW, ds=ds, dz=dz, P=P)
+
+    first = run()
+    for _ in range(12):
+        again = run()
+        for k, v in again.items():
+            assert torch.equal(v.view(torch.uint8), first[k].view(torch.uint8)), k
+    rows = np.unique(np.concatenate([np.arange(0, out, 97), [out - 1]]))
+    W32 = Wd[rows].float().cpu().numpy()
+    s_o, z_o = O.minmax_init(W32, bits, group)
+    assert np.array_equal(first["s"][rows].cpu().numpy(), s_o) and np.array_equal(first["z"][rows].cpu().numpy(), z_o)
+    What_o = O.fake_quant_weight(W32, s_o, z_o, bits, group)              # the oracle's value, to one bf16 ulp
+    assert (np.abs(torch_to_f64(first["What"][rows]) - What_o) <= np.abs(What_o) * 2.0 ** -7 + 1e-30).all()
+    P_o, _, _ = O.quantize_pack(W32, s_o, z_o, bits, group)
+    assert np.array_equal(first["P"][rows].cpu().numpy(), P_o)
+    dW_o, ds_o, _ = O.ste_bwd(Gd[rows].float().cpu().numpy(), W32, s_o, z_o, bits, group)
+    assert np.array_equal(torch_to_f64(first["dW"][rows]), dW_o)
+    assert rel_err(torch_to_f64(first["ds"][rows]), ds_o) <= TOL
+
+
 # --------------------------------------------------------------------------- Block-AP layer
 def workspace_for(eqat, d):
     """Scratch of the Block-AP backward: none (NULL) when the group is reduced inside the GEMM."""
@@ -511,6 +556,33 @@ def test_few_token_forward_agrees_with_tiled_forward(eqat):
     eqat.qlinear_packed_fwd(d, X4, dev(P_o), s16d, dev(z8_o), Y4)
     torch.cuda.synchronize()
     assert rel_err(torch_to_f64(Y4), torch_to_f64(r5["Y"][:4])) <= TOL
+
+
+def test_few_token_forward_is_deterministic(eqat):
+    """More row-blocks than SMs, several stages per row-block: the partial sums of the sixteen warps are added in
+    a fixed order by one warp, so repeated launches must agree bit for bit (also while other work runs beside them)."""
+    out, in_f, T = 2432, 5120, 3
+    g = torch.Generator(device="cuda"); g.manual_seed(11)
+    P = torch.randint(0, 256, (out, in_f // 4), dtype=torch.uint8, device="cuda", generator=g)
+    z8 = torch.randint(0, 4, (out, in_f // 64), dtype=torch.uint8, device="cuda", generator=g)
+    s16 = (torch.rand(out, in_f // 64, device="cuda", generator=g) * 0.01 + 0.001).half()
+    X = torch.randn(T, in_f, device="cuda", generator=g).to(torch.bfloat16)
+    d = eqat.make_desc(2, 64, out, in_f, T)
+    ref = torch.empty(T, out, dtype=torch.bfloat16, device="cuda")
+    eqat.qlinear_packed_fwd(d, X, P, s16, z8, ref)
+    side = torch.cuda.Stream()
+    noise = torch.empty(1 << 26, device="cuda")
+    for _ in range(5):
+        with torch.cuda.stream(side):
+            noise.normal_()                                # unrelated traffic on another stream
+        Y = torch.full_like(ref, float("nan"))
+        eqat.qlinear_packed_fwd(d, X, P, s16, z8, Y)
+        torch.cuda.synchronize()
+        assert torch.equal(Y.view(torch.int16), ref.view(torch.int16))
+    # and it is the right answer
+    q = O.unpack_rows(P.cpu().numpy(), 2, in_f)
+    What_o = O.dequantize(q, s16.cpu().numpy().astype(np.float32), z8.cpu().numpy(), 64)
+    assert rel_err(torch_to_f64(ref), O.linear_fwd(torch_to_f64(X), What_o)) <= TOL
 
 
 @pytest.mark.parametrize("out,in_f,tokens,bits,group", [
