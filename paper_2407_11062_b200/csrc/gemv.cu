@@ -1,14 +1,19 @@
 // Packed-weight forward for a handful of tokens (decode-time inference):
-//     Y[T,out] = X[T,in] * dequant(Wq)^T,   T <= 4,
+//     Y[T,out] = X[T,in] * dequant(Wq)^T,
 // the matrix-vector case of the E2E-QP forward (Eq. 2 on frozen codes).  The
-// 256-row tensor-core tiles of gemm.cu would be almost empty here; the work is
-// one pass over the packed weight, so the kernel is a stream over its bytes.
+// 512-row tensor-memory tiles of gemm.cu would be almost empty here; the work is
+// one pass over the packed weight, so the kernels are streams over its bytes.
+// Two kernels: the first (below) runs on the ordinary cores and takes every bit
+// width and zero-point format for up to four tokens; the second (further down)
+// builds weight fragments for warp-level matrix instructions and takes 2-bit
+// codes with byte zero points for up to eight tokens.
 //
-// Mapping: a CTA owns 32 consecutive weight rows, lane = row, and its 16 warps
-// split the row into contiguous runs of 64-code units.  All lanes of a warp are
-// on the same columns, so the activations are read from shared memory as
-// broadcasts (one wavefront per 16-byte load); each warp stages the columns of
-// its own units there as fp32, together with their sum over every 64-column unit.
+// First kernel.  Mapping: a CTA owns 32 consecutive weight rows, lane = row, and
+// its 16 warps split the row into contiguous runs of 64-code units.  All lanes
+// of a warp are on the same columns, so the activations are read from shared
+// memory as broadcasts (one wavefront per 16-byte load); each warp stages the
+// columns of its own units there as fp32, together with their sum over every
+// 64-column unit.
 //
 // Arithmetic: a code q is dropped into the top mantissa bits of the float 1.0,
 // giving 1 + q/2^N with two logic operations and no int-to-float conversion.
