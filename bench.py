@@ -592,6 +592,40 @@ def run_block_ap_forms(eqat, device, steps=10):
     return out
 
 
+def run_block_driver(eqat, device, steps=10):
+    """The headline block (without the hand-off) through the library's block-level entry points, one C call per
+    phase and step, beside the same work as one call per linear and pass: same kernels, so the difference is what
+    the host spends on crossing the boundary."""
+    wl = BlockWorkload(eqat, device, seed=5, handoff=False)
+    ap, e2e = [], []
+    for L in wl.layers:
+        S = wl.shapes[L["shape"]]
+        ap.append(dict(desc=S["d_ap"], X=S["X"][: wl.t_ap], dY=S["dY"][: wl.t_ap], W=L["W"], s=L["s"], z=L["z"],
+                       Y=S["Y"][: wl.t_ap], W_hat=S["What"], dX=S["dX"][: wl.t_ap], dW=S["dW"], ds=S["ds"], dz=S["dz"],
+                       workspace=S["ws"]))
+        e2e.append(dict(desc=S["d_e2e"], X=S["X"][: wl.t_e2e], dY=S["dY"][: wl.t_e2e], Wq_packed=L["P"], s16=L["s16"],
+                        z=L["z8"], Y=S["Y"][: wl.t_e2e], dX=S["dX"][: wl.t_e2e], ds=S["ds2"], dz=None, workspace=None))
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / steps
+
+    ms_layer = timed(lambda: wl.step())
+    ms_block = timed(lambda: (eqat.eqat_block_ap_step(ap), eqat.eqat_e2e_qp_step(e2e)))
+    f = sum(wl.flops())
+    return {"calls": "eqat_block_ap_step + eqat_e2e_qp_step over the 7 linears", "ms_per_step": ms_block,
+            "tflops": f / (ms_block * 1e-3) / 1e12, "per_linear_calls_ms_per_step": ms_layer,
+            "per_linear_calls_tflops": f / (ms_layer * 1e-3) / 1e12}
+
+
 def time_rotation(calls, rounds):
     """Device time per launch (us) of `calls` issued in order, `rounds` times over: one pass is captured in a CUDA
     graph (so the host's launch cost is not in the figure) and replayed between a pair of events on its stream."""
@@ -800,6 +834,7 @@ def run_ours(args):
             out["configs"] = {name: run_extra_config(eqat, device, name, spec, peaks) for name, spec in EXTRA_CONFIGS.items()}
             out["block_ap_forms"] = run_block_ap_forms(eqat, device)
             out["few_tokens"] = decode_leg(eqat, device, peaks, 10)
+            out["block_driver"] = run_block_driver(eqat, device)
             out["streaming"] = {"w2g64": run_streaming_leg(eqat, device, peaks, 2, 64),
                                 "w4g128": run_streaming_leg(eqat, device, peaks, 4, 128)}
             alias = {"fakequant_weight": "fakequant_weight", "ste_bwd": "ste_bwd", "minmax_init": "minmax_init_cold",

@@ -254,6 +254,57 @@ int qlinear_packed_bwd_ds(const eqat_desc* desc, const eqat_bf16* X, const eqat_
                           const uint8_t* Wq_packed, const void* z, const eqat_fp16* s16,
                           float* ds, float* dz, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------ whole blocks */
+
+/* Both phases of the paper work on one transformer block at a time (Block-AP,
+ * Sec. 3.2: "training of all parameters" of a block; E2E-QP, Sec. 3.3: every
+ * quantised linear of the network with frozen codes), so a training step calls
+ * the layer entry points above once per linear of the block (seven in a Llama
+ * decoder block).  The two calls below take the block's linears as a HOST array
+ * and do exactly that, in array order, on one stream:
+ *   eqat_block_ap_step : qlinear_fakequant_fwd, then qlinear_fakequant_bwd
+ *   eqat_e2e_qp_step   : qlinear_packed_fwd, qlinear_packed_bwd_dx,
+ *                        qlinear_packed_bwd_ds
+ * Every linear is validated on the host before the first launch: on an error
+ * nothing has been enqueued, the status is that of the first offending linear
+ * and *h_failed (may be NULL) receives its index.  The fields have the meaning
+ * of the same-named arguments of the layer entry points (W_hat, dz, workspace
+ * optional as there).  The arrays are read during the call and not retained. */
+typedef struct {
+  eqat_desc desc;
+  const eqat_bf16* X;         /* [T,in]                          */
+  const eqat_bf16* dY;        /* [T,out]                         */
+  const eqat_bf16* W;         /* [out,in] latent weight          */
+  const float* s;             /* [out,in/g]                      */
+  const float* z;             /* [out,in/g]                      */
+  eqat_bf16* Y;               /* [T,out]   (out)                 */
+  eqat_bf16* W_hat;           /* [out,in]  (out, may be NULL)    */
+  eqat_bf16* dX;              /* [T,in]    (out)                 */
+  eqat_bf16* dW;              /* [out,in]  (out)                 */
+  float* ds;                  /* [out,in/g] (out)                */
+  float* dz;                  /* [out,in/g] (out, may be NULL)   */
+  void* workspace;            /* eqat_workspace_bytes(EQAT_OP_FAKEQUANT_BWD), may be NULL if 0 */
+  size_t workspace_bytes;
+} eqat_block_ap_linear;
+
+typedef struct {
+  eqat_desc desc;
+  const eqat_bf16* X;         /* [T,in]                          */
+  const eqat_bf16* dY;        /* [T,out]                         */
+  const uint8_t* Wq_packed;   /* [out, in*N/8]                   */
+  const eqat_fp16* s16;       /* [out,in/g]                      */
+  const void* z;              /* [out,in/g] uint8 or fp16 (desc.zero_point_format) */
+  eqat_bf16* Y;               /* [T,out]   (out)                 */
+  eqat_bf16* dX;              /* [T,in]    (out)                 */
+  float* ds;                  /* [out,in/g] (out)                */
+  float* dz;                  /* [out,in/g] (out, may be NULL)   */
+  void* workspace;            /* eqat_workspace_bytes(EQAT_OP_PACKED_BWD_DS), may be NULL if 0 */
+  size_t workspace_bytes;
+} eqat_e2e_qp_linear;
+
+int eqat_block_ap_step(const eqat_block_ap_linear* h_linears, int count, int* h_failed, void* stream);
+int eqat_e2e_qp_step(const eqat_e2e_qp_linear* h_linears, int count, int* h_failed, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

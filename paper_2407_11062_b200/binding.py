@@ -34,6 +34,18 @@ class eqat_desc(Structure):
                 ("tokens", c_int64), ("dz_mode", c_int32), ("zero_point_format", c_int32)]
 
 
+class eqat_block_ap_linear(Structure):
+    _fields_ = [("desc", eqat_desc), ("X", c_void_p), ("dY", c_void_p), ("W", c_void_p), ("s", c_void_p), ("z", c_void_p),
+                ("Y", c_void_p), ("W_hat", c_void_p), ("dX", c_void_p), ("dW", c_void_p), ("ds", c_void_p),
+                ("dz", c_void_p), ("workspace", c_void_p), ("workspace_bytes", c_size_t)]
+
+
+class eqat_e2e_qp_linear(Structure):
+    _fields_ = [("desc", eqat_desc), ("X", c_void_p), ("dY", c_void_p), ("Wq_packed", c_void_p), ("s16", c_void_p),
+                ("z", c_void_p), ("Y", c_void_p), ("dX", c_void_p), ("ds", c_void_p), ("dz", c_void_p),
+                ("workspace", c_void_p), ("workspace_bytes", c_size_t)]
+
+
 def _load():
     if not os.path.exists(_LIB_PATH):
         raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2407_11062_b200.build` "
@@ -60,6 +72,8 @@ def _load():
         "qlinear_packed_fwd": (c_int, [D, P, P, P, P, P, P]),
         "qlinear_packed_bwd_dx": (c_int, [D, P, P, P, P, P, P]),
         "qlinear_packed_bwd_ds": (c_int, [D, P, P, P, P, P, P, P, P, c_size_t, P]),
+        "eqat_block_ap_step": (c_int, [POINTER(eqat_block_ap_linear), c_int, POINTER(c_int), P]),
+        "eqat_e2e_qp_step": (c_int, [POINTER(eqat_e2e_qp_linear), c_int, POINTER(c_int), P]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -189,3 +203,40 @@ def qlinear_packed_bwd_ds(desc, X, dY, Wq_packed, z8, s16, ds, dz=None, workspac
     _check(lib.qlinear_packed_bwd_ds(ctypes.byref(desc), _ptr(X), _ptr(dY), _ptr(Wq_packed), _ptr(z8), _ptr(s16),
                                      _ptr(ds), _ptr(dz), _ptr(workspace), nbytes, _stream()),
            "qlinear_packed_bwd_ds")
+
+
+def _addr(t):
+    p = _ptr(t)
+    return None if p is None else p.value
+
+
+def _nbytes(t):
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def _run_block(fn, struct, rows, where):
+    arr = (struct * len(rows))(*rows)
+    failed = c_int(-1)
+    rc = fn(arr, len(rows), ctypes.byref(failed), _stream())
+    if rc != EQAT_OK:
+        raise EqatError(rc, f"{where} (linear {failed.value})")
+
+
+def eqat_block_ap_step(linears):
+    """Block-AP forward + backward of every linear of a block in one call.  `linears`: dicts with desc, X, dY, W,
+    s, z, Y, W_hat (or None), dX, dW, ds, dz (or None), workspace (or None)."""
+    rows = [eqat_block_ap_linear(L["desc"], _addr(L["X"]), _addr(L["dY"]), _addr(L["W"]), _addr(L["s"]), _addr(L["z"]),
+                                 _addr(L["Y"]), _addr(L.get("W_hat")), _addr(L["dX"]), _addr(L["dW"]), _addr(L["ds"]),
+                                 _addr(L.get("dz")), _addr(L.get("workspace")), _nbytes(L.get("workspace")))
+            for L in linears]
+    _run_block(lib.eqat_block_ap_step, eqat_block_ap_linear, rows, "eqat_block_ap_step")
+
+
+def eqat_e2e_qp_step(linears):
+    """E2E-QP forward, dX and ds (dz) of every linear of a block in one call.  `linears`: dicts with desc, X, dY,
+    Wq_packed, s16, z, Y, dX, ds, dz (or None), workspace (or None)."""
+    rows = [eqat_e2e_qp_linear(L["desc"], _addr(L["X"]), _addr(L["dY"]), _addr(L["Wq_packed"]), _addr(L["s16"]),
+                               _addr(L["z"]), _addr(L["Y"]), _addr(L["dX"]), _addr(L["ds"]), _addr(L.get("dz")),
+                               _addr(L.get("workspace")), _nbytes(L.get("workspace")))
+            for L in linears]
+    _run_block(lib.eqat_e2e_qp_step, eqat_e2e_qp_linear, rows, "eqat_e2e_qp_step")

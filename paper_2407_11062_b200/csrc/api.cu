@@ -62,6 +62,53 @@ int check_ptrs(P... ptrs) {
 
 inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
 
+// Host-side validation of the layer entry points, one function each, so that the block-level calls can check
+// every linear before the first launch.
+int v_fakequant_fwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* W, const float* s, const float* z,
+                    const eqat_bf16* Y, const eqat_bf16* W_hat) {
+  int rc = check_gemm_desc(d, false);
+  if (rc != EQAT_OK) return rc;
+  if ((rc = check_ptrs(X, W, s, z, Y)) != EQAT_OK) return rc;
+  if (W_hat == nullptr) return latent_group_ok(d) ? EQAT_OK : EQAT_ERR_UNSUPPORTED;
+  return aligned16(W_hat) ? EQAT_OK : EQAT_ERR_ALIGN;
+}
+
+int v_fakequant_bwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* dY, const eqat_bf16* W, const float* s,
+                    const float* z, const eqat_bf16* W_hat, const eqat_bf16* dX, const eqat_bf16* dW, const float* ds,
+                    const float* dz, const void* workspace, size_t workspace_bytes) {
+  int rc = check_gemm_desc(d, false);
+  if (rc != EQAT_OK) return rc;
+  if ((rc = check_ptrs(X, dY, W, s, z, dX, dW, ds)) != EQAT_OK) return rc;
+  if (dz != nullptr && !aligned16(dz)) return EQAT_ERR_ALIGN;
+  if (W_hat != nullptr && !aligned16(W_hat)) return EQAT_ERR_ALIGN;
+  if (W_hat == nullptr && !latent_group_ok(d)) return EQAT_ERR_UNSUPPORTED;
+  if (d->group > kMaxFusedSteGroup) {
+    const size_t need = (size_t)d->out_features * d->in_features * sizeof(eqat_bf16);
+    if (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+      return EQAT_ERR_WORKSPACE;
+  }
+  return EQAT_OK;
+}
+
+int v_packed_fwd(const eqat_desc* d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* z,
+                 const eqat_bf16* Y) {
+  const int rc = check_gemm_desc(d, true);
+  return rc != EQAT_OK ? rc : check_ptrs(X, Wq, s16, z, Y);
+}
+
+int v_packed_bwd_ds(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* dY, const uint8_t* Wq, const void* z,
+                    const eqat_fp16* s16, const float* ds, const float* dz, const void* workspace,
+                    size_t workspace_bytes) {
+  int rc = check_gemm_desc(d, true);
+  if (rc != EQAT_OK) return rc;
+  if ((rc = check_ptrs(X, dY, Wq, z, ds)) != EQAT_OK) return rc;
+  if (dz != nullptr && (rc = check_ptrs(dz, s16)) != EQAT_OK) return rc;
+  const size_t need = packed_ds_workspace_bytes(*d);
+  if (need != 0 && (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0))
+    return EQAT_ERR_WORKSPACE;
+  return EQAT_OK;
+}
+
 #define EQAT_TRY(expr)            \
   do {                            \
     const int rc__ = (expr);      \
@@ -136,14 +183,9 @@ int eqat_fakequant_weight(const eqat_desc* d, const eqat_bf16* W, const float* s
 
 int qlinear_fakequant_fwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* W, const float* s, const float* z,
                           eqat_bf16* Y, eqat_bf16* W_hat, void* stream) {
-  EQAT_TRY(check_gemm_desc(d, false));
-  EQAT_TRY(check_ptrs(X, W, s, z, Y));
-  if (W_hat == nullptr) {
-    // W_hat is not wanted: fake-quantise each tile of W inside the GEMM, after it has reached shared memory
-    if (!latent_group_ok(d)) return EQAT_ERR_UNSUPPORTED;
-    return launch_latent_fwd(*d, X, W, s, z, Y, as_stream(stream));
-  }
-  if (!aligned16(W_hat)) return EQAT_ERR_ALIGN;
+  EQAT_TRY(v_fakequant_fwd(d, X, W, s, z, Y, W_hat));
+  // W_hat not wanted: fake-quantise each tile of W inside the GEMM, after it has reached shared memory
+  if (W_hat == nullptr) return launch_latent_fwd(*d, X, W, s, z, Y, as_stream(stream));
   EQAT_TRY(launch_fakequant(*d, W, s, z, W_hat, as_stream(stream)));
   return launch_dense_fwd(*d, X, W_hat, Y, as_stream(stream));
 }
@@ -159,20 +201,11 @@ int eqat_ste_bwd(const eqat_desc* d, const eqat_bf16* dW_hat, const eqat_bf16* W
 int qlinear_fakequant_bwd(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* dY, const eqat_bf16* W,
                           const float* s, const float* z, const eqat_bf16* W_hat, eqat_bf16* dX, eqat_bf16* dW,
                           float* ds, float* dz, void* workspace, size_t workspace_bytes, void* stream) {
-  EQAT_TRY(check_gemm_desc(d, false));
-  EQAT_TRY(check_ptrs(X, dY, W, s, z, dX, dW, ds));
-  if (dz != nullptr && !aligned16(dz)) return EQAT_ERR_ALIGN;
-  if (W_hat != nullptr && !aligned16(W_hat)) return EQAT_ERR_ALIGN;
-  if (W_hat == nullptr && !latent_group_ok(d)) return EQAT_ERR_UNSUPPORTED;
+  EQAT_TRY(v_fakequant_bwd(d, X, dY, W, s, z, W_hat, dX, dW, ds, dz, workspace, workspace_bytes));
   // A group that fits inside one output tile is reduced in the weight-gradient GEMM's epilogue and needs no
   // scratch; a longer one (channel-wise quantisation) spans tiles, so its gradient goes through the workspace
   // and a second kernel.
   const bool fused = d->group <= kMaxFusedSteGroup;
-  if (!fused) {
-    const size_t need = (size_t)d->out_features * d->in_features * sizeof(eqat_bf16);
-    if (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
-      return EQAT_ERR_WORKSPACE;
-  }
   eqat_bf16* dW_hat = static_cast<eqat_bf16*>(workspace);
   cudaStream_t st = as_stream(stream);
   if (W_hat != nullptr) EQAT_TRY(launch_dense_dx(*d, dY, W_hat, dX, st));
@@ -217,8 +250,7 @@ int eqat_unpack_zeros(const eqat_desc* d, const uint8_t* z_packed, uint8_t* z8, 
 
 int qlinear_packed_fwd(const eqat_desc* d, const eqat_bf16* X, const uint8_t* Wq_packed, const eqat_fp16* s16,
                        const void* z, eqat_bf16* Y, void* stream) {
-  EQAT_TRY(check_gemm_desc(d, true));
-  EQAT_TRY(check_ptrs(X, Wq_packed, s16, z, Y));
+  EQAT_TRY(v_packed_fwd(d, X, Wq_packed, s16, z, Y));
   // a handful of tokens (decoding): one pass over the packed weight instead of near-empty tensor-core tiles
   if (packed_gemv_applies(*d)) return launch_packed_gemv(*d, X, Wq_packed, s16, z, Y, as_stream(stream));
   return launch_packed_fwd(*d, X, Wq_packed, s16, z, Y, as_stream(stream));
@@ -226,21 +258,71 @@ int qlinear_packed_fwd(const eqat_desc* d, const eqat_bf16* X, const uint8_t* Wq
 
 int qlinear_packed_bwd_dx(const eqat_desc* d, const eqat_bf16* dY, const uint8_t* Wq_packed, const eqat_fp16* s16,
                           const void* z, eqat_bf16* dX, void* stream) {
-  EQAT_TRY(check_gemm_desc(d, true));
-  EQAT_TRY(check_ptrs(dY, Wq_packed, s16, z, dX));
+  EQAT_TRY(v_packed_fwd(d, dY, Wq_packed, s16, z, dX));          // same shape of check: one activation in, one out
   return launch_packed_dx(*d, dY, Wq_packed, s16, z, dX, as_stream(stream));
 }
 
 int qlinear_packed_bwd_ds(const eqat_desc* d, const eqat_bf16* X, const eqat_bf16* dY, const uint8_t* Wq_packed,
                           const void* z, const eqat_fp16* s16, float* ds, float* dz, void* workspace,
                           size_t workspace_bytes, void* stream) {
-  EQAT_TRY(check_gemm_desc(d, true));
-  EQAT_TRY(check_ptrs(X, dY, Wq_packed, z, ds));
-  if (dz != nullptr) EQAT_TRY(check_ptrs(dz, s16));
-  const size_t need = packed_ds_workspace_bytes(*d);
-  if (need != 0 && (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0))
-    return EQAT_ERR_WORKSPACE;
+  EQAT_TRY(v_packed_bwd_ds(d, X, dY, Wq_packed, z, s16, ds, dz, workspace, workspace_bytes));
   return launch_packed_ds(*d, X, dY, Wq_packed, z, s16, ds, dz, workspace, as_stream(stream));
+}
+
+int eqat_block_ap_step(const eqat_block_ap_linear* L, int count, int* h_failed, void* stream) {
+  if (h_failed != nullptr) *h_failed = -1;
+  if (L == nullptr) return EQAT_ERR_NULL;
+  if (count <= 0) return EQAT_ERR_SHAPE;
+  for (int i = 0; i < count; ++i) {                         // everything is checked before anything is launched
+    int rc = v_fakequant_fwd(&L[i].desc, L[i].X, L[i].W, L[i].s, L[i].z, L[i].Y, L[i].W_hat);
+    if (rc == EQAT_OK)
+      rc = v_fakequant_bwd(&L[i].desc, L[i].X, L[i].dY, L[i].W, L[i].s, L[i].z, L[i].W_hat, L[i].dX, L[i].dW, L[i].ds,
+                           L[i].dz, L[i].workspace, L[i].workspace_bytes);
+    if (rc != EQAT_OK) {
+      if (h_failed != nullptr) *h_failed = i;
+      return rc;
+    }
+  }
+  for (int i = 0; i < count; ++i) {
+    int rc = qlinear_fakequant_fwd(&L[i].desc, L[i].X, L[i].W, L[i].s, L[i].z, L[i].Y, L[i].W_hat, stream);
+    if (rc == EQAT_OK)
+      rc = qlinear_fakequant_bwd(&L[i].desc, L[i].X, L[i].dY, L[i].W, L[i].s, L[i].z, L[i].W_hat, L[i].dX, L[i].dW,
+                                 L[i].ds, L[i].dz, L[i].workspace, L[i].workspace_bytes, stream);
+    if (rc != EQAT_OK) {                                    // only the runtime can still refuse (EQAT_ERR_CUDA)
+      if (h_failed != nullptr) *h_failed = i;
+      return rc;
+    }
+  }
+  return EQAT_OK;
+}
+
+int eqat_e2e_qp_step(const eqat_e2e_qp_linear* L, int count, int* h_failed, void* stream) {
+  if (h_failed != nullptr) *h_failed = -1;
+  if (L == nullptr) return EQAT_ERR_NULL;
+  if (count <= 0) return EQAT_ERR_SHAPE;
+  for (int i = 0; i < count; ++i) {
+    int rc = v_packed_fwd(&L[i].desc, L[i].X, L[i].Wq_packed, L[i].s16, L[i].z, L[i].Y);
+    if (rc == EQAT_OK) rc = v_packed_fwd(&L[i].desc, L[i].dY, L[i].Wq_packed, L[i].s16, L[i].z, L[i].dX);
+    if (rc == EQAT_OK)
+      rc = v_packed_bwd_ds(&L[i].desc, L[i].X, L[i].dY, L[i].Wq_packed, L[i].z, L[i].s16, L[i].ds, L[i].dz,
+                           L[i].workspace, L[i].workspace_bytes);
+    if (rc != EQAT_OK) {
+      if (h_failed != nullptr) *h_failed = i;
+      return rc;
+    }
+  }
+  for (int i = 0; i < count; ++i) {
+    int rc = qlinear_packed_fwd(&L[i].desc, L[i].X, L[i].Wq_packed, L[i].s16, L[i].z, L[i].Y, stream);
+    if (rc == EQAT_OK) rc = qlinear_packed_bwd_dx(&L[i].desc, L[i].dY, L[i].Wq_packed, L[i].s16, L[i].z, L[i].dX, stream);
+    if (rc == EQAT_OK)
+      rc = qlinear_packed_bwd_ds(&L[i].desc, L[i].X, L[i].dY, L[i].Wq_packed, L[i].z, L[i].s16, L[i].ds, L[i].dz,
+                                 L[i].workspace, L[i].workspace_bytes, stream);
+    if (rc != EQAT_OK) {
+      if (h_failed != nullptr) *h_failed = i;
+      return rc;
+    }
+  }
+  return EQAT_OK;
 }
 
 }  // extern "C"

@@ -696,6 +696,68 @@ def test_packed_weight_aligned_to_16_bytes_only(eqat, bits, tokens):
     assert rel_err(torch_to_f64(res[1][0]), O.linear_fwd(f32(Xb), What_o)) <= TOL
 
 
+def test_block_level_calls_equal_the_layer_calls(eqat):
+    """eqat_block_ap_step and eqat_e2e_qp_step over three linears of different shapes (one with one group per row,
+    which needs both kinds of scratch): bit for bit what the layer entry points give, called one by one."""
+    specs = [(256, 512, 300, 64), (192, 384, 300, 128), (128, 640, 300, 640)]
+    bits = 2
+    ap_rows, e2e_rows, expect = [], [], []
+    for k, (out, in_f, T, group) in enumerate(specs):
+        cfg = small_cfg(f"blk_{k}", out, in_f, bits, group, T, "student_t4", 0.02, 0.01)
+        lin = cfg.linears[0]
+        ng = in_f // group
+        W32 = f32(weight_for(cfg, lin)); Xb, dYb = activations_for(cfg, lin, T)
+        s, z = O.minmax_init(W32, bits, group)
+        P_o, z8_o, s16_o = O.quantize_pack(W32, s, z, bits, group)
+        Wd, Xd, dYd, sd, zd = bits_to_torch(weight_for(cfg, lin)), bits_to_torch(Xb), bits_to_torch(dYb), dev(s), dev(z)
+        Pd, z8d = dev(P_o), dev(z8_o)
+        s16d = torch.from_numpy(s16_o.view(np.int16)).view(torch.float16).cuda()
+        d = eqat.make_desc(bits, group, out, in_f, T)
+        bf = torch.bfloat16
+
+        def outs_ap():
+            n = eqat.workspace_bytes(d, eqat.EQAT_OP_FAKEQUANT_BWD)
+            return dict(Y=torch.empty(T, out, dtype=bf, device="cuda"), W_hat=torch.empty(out, in_f, dtype=bf, device="cuda"),
+                        dX=torch.empty(T, in_f, dtype=bf, device="cuda"), dW=torch.empty(out, in_f, dtype=bf, device="cuda"),
+                        ds=torch.empty(out, ng, device="cuda"), dz=torch.empty(out, ng, device="cuda"),
+                        workspace=torch.empty(n, dtype=torch.uint8, device="cuda") if n else None)
+
+        def outs_e2e():
+            n = eqat.workspace_bytes(d, eqat.EQAT_OP_PACKED_BWD_DS)
+            return dict(Y=torch.empty(T, out, dtype=bf, device="cuda"), dX=torch.empty(T, in_f, dtype=bf, device="cuda"),
+                        ds=torch.empty(out, ng, device="cuda"), dz=torch.empty(out, ng, device="cuda"),
+                        workspace=torch.empty(n, dtype=torch.uint8, device="cuda") if n else None)
+
+        a, b = outs_ap(), outs_ap()
+        eqat.qlinear_fakequant_fwd(d, Xd, Wd, sd, zd, a["Y"], a["W_hat"])
+        eqat.qlinear_fakequant_bwd(d, Xd, dYd, Wd, sd, zd, a["W_hat"], a["dX"], a["dW"], a["ds"], a["dz"], a["workspace"])
+        ap_rows.append(dict(desc=d, X=Xd, dY=dYd, W=Wd, s=sd, z=zd, **b))
+        c, e = outs_e2e(), outs_e2e()
+        eqat.qlinear_packed_fwd(d, Xd, Pd, s16d, z8d, c["Y"])
+        eqat.qlinear_packed_bwd_dx(d, dYd, Pd, s16d, z8d, c["dX"])
+        eqat.qlinear_packed_bwd_ds(d, Xd, dYd, Pd, z8d, s16d, c["ds"], c["dz"], c["workspace"])
+        e2e_rows.append(dict(desc=d, X=Xd, dY=dYd, Wq_packed=Pd, s16=s16d, z=z8d, **e))
+        expect.append((a, c))
+    eqat.eqat_block_ap_step(ap_rows)
+    eqat.eqat_e2e_qp_step(e2e_rows)
+    torch.cuda.synchronize()
+    for (a, c), got_ap, got_e2e in zip(expect, ap_rows, e2e_rows):
+        for k in ("Y", "W_hat", "dX", "dW", "ds", "dz"):
+            assert torch.equal(got_ap[k], a[k]), k
+        for k in ("Y", "dX", "ds", "dz"):
+            assert torch.equal(got_e2e[k], c[k]), k
+    # a fault in the last linear: reported with its index, and nothing has run (the first linear's outputs keep
+    # the pattern they are given here)
+    ap_rows[0]["Y"].fill_(7.0)
+    broken = [dict(r) for r in ap_rows]
+    broken[2]["dW"] = None
+    with pytest.raises(eqat.EqatError, match="linear 2") as err:
+        eqat.eqat_block_ap_step(broken)
+    assert err.value.status == eqat.EQAT_ERR_NULL
+    torch.cuda.synchronize()
+    assert bool((ap_rows[0]["Y"] == 7.0).all())
+
+
 @pytest.mark.parametrize("which,name", [(0, "GEMM kernels"), (1, "streaming kernels"), (2, "matrix-vector kernel")])
 def test_a_bounded_wait_runs_out_cleanly(eqat, which, name):
     """One warp waits 1 ms for a barrier that nothing signals, through the kernels' own wait routine: the kernel

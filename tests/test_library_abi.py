@@ -95,3 +95,42 @@ def test_null_and_misaligned_pointers(eqat):
     assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(dc), *args, ok, 16, None) == eqat.EQAT_ERR_WORKSPACE
     assert eqat.lib.qlinear_fakequant_bwd(ctypes.byref(dc), *args, ctypes.c_void_p(0x1010), 1 << 20, None) == eqat.EQAT_ERR_WORKSPACE
     assert eqat.lib.eqat_selftest_wait_expiry(7, None) == eqat.EQAT_ERR_UNSUPPORTED
+
+
+def test_block_level_calls_validate_every_linear_before_anything_runs(eqat):
+    """eqat_block_ap_step / eqat_e2e_qp_step: a fault in the LAST linear of the array is reported with its index and
+    with the status the layer entry point would give; the pointers of the earlier (valid) linears are fake, so a
+    launch on them before the check of the last one would not go unnoticed on a machine with a GPU, and on this
+    one no launch is possible at all."""
+    ok = 0x1000
+    d = eqat.make_desc(2, 64, 512, 512, 256)
+
+    def ap(**kw):
+        f = dict(desc=d, X=ok, dY=ok, W=ok, s=ok, z=ok, Y=ok, W_hat=ok, dX=ok, dW=ok, ds=ok, dz=ok, workspace=None,
+                 workspace_bytes=0)
+        f.update(kw)
+        return eqat.eqat_block_ap_linear(**f)
+
+    def e2e(**kw):
+        f = dict(desc=d, X=ok, dY=ok, Wq_packed=ok, s16=ok, z=ok, Y=ok, dX=ok, ds=ok, dz=None, workspace=None,
+                 workspace_bytes=0)
+        f.update(kw)
+        return eqat.eqat_e2e_qp_linear(**f)
+
+    failed = ctypes.c_int(-5)
+    for rows, fn, struct, want in (
+            ([ap(), ap(), ap(dW=None)], eqat.lib.eqat_block_ap_step, eqat.eqat_block_ap_linear, (eqat.EQAT_ERR_NULL, 2)),
+            ([ap(), ap(Y=0x1004)], eqat.lib.eqat_block_ap_step, eqat.eqat_block_ap_linear, (eqat.EQAT_ERR_ALIGN, 1)),
+            ([ap(), ap(desc=eqat.make_desc(2, 512, 512, 512, 256))], eqat.lib.eqat_block_ap_step,
+             eqat.eqat_block_ap_linear, (eqat.EQAT_ERR_WORKSPACE, 1)),              # channel-wise without scratch
+            ([e2e(), e2e(), e2e(), e2e(ds=None)], eqat.lib.eqat_e2e_qp_step, eqat.eqat_e2e_qp_linear,
+             (eqat.EQAT_ERR_NULL, 3)),
+            ([e2e(), e2e(desc=eqat.make_desc(5, 64, 512, 512, 256))], eqat.lib.eqat_e2e_qp_step,
+             eqat.eqat_e2e_qp_linear, (eqat.EQAT_ERR_UNSUPPORTED, 1)),
+            ([e2e(), e2e(dz=ok, s16=None)], eqat.lib.eqat_e2e_qp_step, eqat.eqat_e2e_qp_linear, (eqat.EQAT_ERR_NULL, 1))):
+        arr = (struct * len(rows))(*rows)
+        rc = fn(arr, len(rows), ctypes.byref(failed), None)
+        assert (rc, failed.value) == want
+    assert eqat.lib.eqat_block_ap_step(None, 1, None, None) == eqat.EQAT_ERR_NULL
+    arr = (eqat.eqat_e2e_qp_linear * 1)(e2e())
+    assert eqat.lib.eqat_e2e_qp_step(arr, 0, None, None) == eqat.EQAT_ERR_SHAPE
