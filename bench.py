@@ -61,10 +61,10 @@ EXTRA_CONFIGS = {
 # files change (comments and white space aside) the figures are stale and `roofline.traffic` is reported as null.
 NCU_TRAFFIC = {
     "sources": ("gemm.cu", "ptx.cuh"),
-    "sources_sha256": "c66b5e131c34943e0c94211e2485da9bbaa818df051387a7c0c3eb6dce73c425",
-    "packed_fwd": {"qkvo": 141.4e6 + 100.7e6, "gate_up": 163.5e6 + 315.0e6, "down": 502.9e6 + 116.0e6},
-    "packed_bwd_dx": {"qkvo": 140.7e6 + 100.1e6, "gate_up": 514.8e6 + 115.9e6, "down": 154.1e6 + 316.4e6},
-    "packed_bwd_ds": {"qkvo": 416.2e6 + 4.5e6, "gate_up": 1306.3e6 + 2.7e6, "down": 1073.8e6 + 2.9e6},
+    "sources_sha256": "80fde187933896517192d9f4487bb958fba6b2499e62d11aadddd993f376ce5e",
+    "packed_fwd": {"qkvo": 141.3e6 + 96.9e6, "gate_up": 163.8e6 + 315.0e6, "down": 503.9e6 + 116.0e6},
+    "packed_bwd_dx": {"qkvo": 140.5e6 + 96.6e6, "gate_up": 514.8e6 + 116.0e6, "down": 153.7e6 + 315.5e6},
+    "packed_bwd_ds": {"qkvo": 416.2e6 + 0.8e6, "gate_up": 1306.4e6 + 2.8e6, "down": 1073.4e6 + 2.8e6},
 }
 
 

@@ -211,6 +211,26 @@ struct GroupValues {
   __device__ __forceinline__ GroupValues(float s, float z) : sp(s * (1.0f / 65536.0f)), cz(-(128.0f + z) * s) {}
   __device__ __forceinline__ float operator()(uint32_t xbits) const { return fmaf(__uint_as_float(xbits), sp, cz); }
 };
+// 3-bit codes are not byte-aligned, and a shift per code costs as much as the multiply-add that follows it.  A
+// code may instead sit at any mantissa position p as long as the constants follow it: with x = 2^23 + 2^p * q,
+// fma(x, s / 2^p, -(2^(23-p) + z) * s) = (q - z) * s, exact while (2^(23-p) + z) * s is (p >= 11 for 11-bit s and
+// z < 8).  Three consecutive codes of the stream land on p = 12, 15, 18 with ONE shift of the word (or of two
+// words, for a code that straddles them), so a triple costs one shift instead of three.
+template <>
+struct GroupValues<3> {
+  float sp[3], cz[3];
+  __device__ __forceinline__ GroupValues() : sp{0.0f, 0.0f, 0.0f}, cz{0.0f, 0.0f, 0.0f} {}
+  __device__ __forceinline__ GroupValues(float s, float z) {
+    sp[0] = s * (1.0f / 4096.0f);   cz[0] = -(2048.0f + z) * s;
+    sp[1] = s * (1.0f / 32768.0f);  cz[1] = -(256.0f + z) * s;
+    sp[2] = s * (1.0f / 262144.0f); cz[2] = -(32.0f + z) * s;
+  }
+  // code of slot k (0..2) of a triple, still at bits [12 + 3k, 15 + 3k) of `win`
+  __device__ __forceinline__ float at(int k, uint32_t win) const {
+    return fmaf(__uint_as_float((win & (7u << (12 + 3 * k))) | 0x4B000000u), sp[k], cz[k]);
+  }
+};
+
 template <>
 struct GroupValues<2> {
   uint32_t lut01, lut23;
@@ -261,23 +281,26 @@ __device__ __forceinline__ void dequant_half32(const uint32_t (&w)[BITS], const 
       store_chunk(row_sx, 4 * h + i, v);
     }
   } else {
+    // 32 codes = 3 words = 96 bits, code j at bit 3j.  Triple m (codes 3m .. 3m+2) is brought to bits 12..20 of a
+    // register by one shift of the stream: the 32-bit window that starts at bit 9m - 12.
+    float v[32];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {                       // 32 codes = 3 words
-      float v[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const int bit = 3 * (8 * c + e), word = bit >> 5, off = bit & 31;
-        uint32_t t;
-        if (off <= 16) {
-          t = w[word] << (16 - off);
-        } else {
-          const uint32_t hi = (off + 3 > 32) ? w[word + 1] : 0u;
-          t = __funnelshift_r(w[word], hi, off - 16);
-        }
-        v[e] = f((t & 0x00070000u) | kMagic);
+    for (int m = 0; m < 11; ++m) {
+      const int start = 9 * m - 12;
+      uint32_t win;
+      if (start < 0) {
+        win = w[0] << (-start);
+      } else {
+        const int word = start >> 5, sh = start & 31;
+        const uint32_t hi = word + 1 < 3 ? w[word + 1 < 3 ? word + 1 : 2] : 0u;
+        win = sh == 0 ? w[word] : __funnelshift_r(w[word], hi, sh);
       }
-      store_chunk(row_sx, 4 * h + c, v);
+#pragma unroll
+      for (int k = 0; k < 3; ++k)
+        if (3 * m + k < 32) v[3 * m + k] = f.at(k, win);
     }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) store_chunk(row_sx, 4 * h + c, *reinterpret_cast<const float(*)[8]>(v + 8 * c));
   }
 }
 
