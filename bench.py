@@ -886,14 +886,14 @@ def run_streaming_case(args):
     print(json.dumps(r), flush=True)
 
 
-def decode_leg(eqat, dev, peaks, iters):
-    """Few-token packed forward (the matrix-vector kernels) on the block's three linear shapes: device time per
+def decode_leg(eqat, dev, peaks, iters, model="7b"):
+    """Few-token packed forward (the matrix-vector kernels) on the linear shapes of one block: device time per
     launch from a CUDA graph of launches over rotating weight copies (more than L2 in total), and the bandwidth that
     time means for the bytes one launch must read."""
     out = {"metric": "packed forward, few tokens", "unit": "us per launch", "bits": BITS, "group": GROUP,
-           "hbm_gbs_peak": peaks["hbm_gbs"],
+           "model": model, "hbm_gbs_peak": peaks["hbm_gbs"],
            "method": "CUDA graph of one launch per weight copy (copies total > 2 x L2), replayed back to back", "cases": {}}
-    for lin in LINEARS["7b"]:
+    for lin in LINEARS[model]:
         o, i = lin.out_features, lin.in_features
         ng = i // GROUP
         wbytes = o * i * BITS // 8
@@ -901,7 +901,7 @@ def decode_leg(eqat, dev, peaks, iters):
         Ps = [torch.randint(0, 256, (o, i * BITS // 8), dtype=torch.uint8, device=dev) for _ in range(copies)]
         z8 = torch.randint(0, 1 << BITS, (o, ng), dtype=torch.uint8, device=dev)
         s16 = (torch.rand(o, ng, device=dev) * 0.01 + 0.001).half()
-        for T in (1, 4, 8):
+        for T in (1, 4, 8, 16):
             X = torch.randn(T, i, device=dev).to(torch.bfloat16)
             Y = torch.empty(T, o, dtype=torch.bfloat16, device=dev)
             d = eqat.make_desc(BITS, GROUP, o, i, T)
@@ -920,7 +920,7 @@ def run_decode_case(args):
     from paper_2407_11062_b200.build import build_library
     build_library()
     from paper_2407_11062_b200 import binding as eqat
-    out = decode_leg(eqat, torch.device("cuda", 0), load_peaks(), args.case_iters)
+    out = decode_leg(eqat, torch.device("cuda", 0), load_peaks(), args.case_iters, args.case_model)
     assert eqat.device_status() == (0, 0)
     print(json.dumps(out), flush=True)
 
@@ -929,7 +929,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--kernel-case", action="store_true", help="run one linear shape a few times (for profilers)")
     ap.add_argument("--decode-case", action="store_true",
-                    help="time the few-token packed forward on the block's linear shapes (uses --case-iters)")
+                    help="time the few-token packed forward on the linear shapes of --case-model (uses --case-iters)")
     ap.add_argument("--streaming-case", action="store_true", help="the cold streaming-kernel leg alone")
     ap.add_argument("--case-model", default="7b", choices=sorted(LINEARS))
     ap.add_argument("--case-shape", default="qkvo")

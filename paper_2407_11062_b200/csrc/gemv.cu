@@ -6,7 +6,8 @@
 // Two kernels: the first (below) runs on the ordinary cores and takes every bit
 // width and zero-point format for up to four tokens; the second (further down)
 // builds weight fragments for warp-level matrix instructions and takes 2-bit
-// codes with byte zero points for up to eight tokens.
+// codes with byte zero points for up to eight tokens per launch (more tokens,
+// or rows too long for the staged activations, go out as several launches).
 //
 // First kernel.  Mapping: a CTA owns 32 consecutive weight rows, lane = row, and
 // its 16 warps split the row into contiguous runs of 64-code units.  All lanes
@@ -317,6 +318,7 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // warp, which adds them in a fixed order and stores Y while the consumers are
 // on the next task.
 constexpr int kTcMaxTokens = 8;                         // the instruction has eight token columns
+constexpr int kTcMaxTotalTokens = 32;                   // more go out as several launches over slices of the tokens
 constexpr int kTcWarps = 16;
 constexpr int kTcThreads = (kTcWarps + 2) * 32;        // + producer warp + reducer warp
 constexpr int kTcRows = 16;                            // weight rows per task
@@ -329,7 +331,7 @@ constexpr int kTcItems = 5;                            // instructions per chunk
 constexpr int kTcMaxStages = 8;
 constexpr int kTcMinStages = 3;
 constexpr uint64_t kTcWaitLimitNs = 2000000000ull;
-constexpr size_t kTcSmemBudget = 225 * 1024;
+constexpr size_t kTcSmemBudget = 227 * 1024;             // the most a CTA can be given (eight tokens of 8192 columns need 225.2 KB)
 
 struct TcCtl {
   uint64_t full[kTcMaxStages];
@@ -385,6 +387,11 @@ __device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, volatile 
   }
   return true;
 }
+
+// Programmatic dependent launch: let the next launch of the stream start / wait until the launches before this one
+// have completed and their writes are visible (both do nothing in a launch without the attribute).
+__device__ __forceinline__ void grid_dependents_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // (t & mask) | magic on both halves of a register.
 __device__ __forceinline__ uint32_t and_or(uint32_t t, uint32_t mask, uint32_t magic) {
@@ -442,7 +449,26 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
   const int task_stages = (n_boxes + kTcBoxesPerStage - 1) / kTcBoxesPerStage;
   const int chunks_pad = n_boxes * 8;
 
-  // Consumers request their first loads before anything else: the first unit of the activations and the step
+  // Launched with programmatic stream serialisation: the next launch of the stream may start as soon as every
+  // CTA of this grid has got here, and a CTA of this grid may be running while the launch before it still is.
+  // Nothing before the wait below touches global memory (the barriers live in this CTA's shared memory); the
+  // wait returns once the earlier grids have completed and their writes are visible.
+  grid_dependents_launch();
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), 1);
+      ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), kTcWarps);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(ptx::smem_addr(&ctl->part_ready[b]), kTcWarps);
+      ptx::mbar_init(ptx::smem_addr(&ctl->part_free[b]), 1);
+    }
+    ctl->abort = 0;
+    ptx::fence_mbar_init();
+  }
+  grid_dependency_wait();
+
+  // Consumers request their first loads before the rest of the set-up: the first unit of the activations and the step
   // sizes / zero points of the first stages.  They are first touches of their pages in this launch, and once the
   // weight stream is running a small load waits behind megabytes of bulk copies.
   const int units = T * chunks_pad * 4;                                // (token, chunk, quad lane): 16 columns each
@@ -504,18 +530,6 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
     if (warp < kTcWarps) { nx[i] = fetch(pf_task, pf_k); advance(); }
   }
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) {
-      ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), 1);
-      ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), kTcWarps);
-    }
-    for (int b = 0; b < 2; ++b) {
-      ptx::mbar_init(ptx::smem_addr(&ctl->part_ready[b]), kTcWarps);
-      ptx::mbar_init(ptx::smem_addr(&ctl->part_free[b]), 1);
-    }
-    ctl->abort = 0;
-    ptx::fence_mbar_init();
-  }
   __syncthreads();
 
   if (warp == kTcWarps) {
@@ -760,24 +774,60 @@ int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const e
   const int vec_params = (d.group == 64 && ng % 4 == 0 && (reinterpret_cast<uintptr_t>(s16) & 7u) == 0 &&
                           (reinterpret_cast<uintptr_t>(zq) & 3u) == 0) ? 1 : 0;
   const TcLayout L = tc_layout(T, d.in_features, stages);
-  packed_gemv_tc_kernel<<<n_tasks < sms ? n_tasks : sms, kTcThreads, L.total, st>>>(
-      mw, X, s16, static_cast<const uint8_t*>(zq), Y, d.out_features, d.in_features, group_shift, ng, T, vec_params, stages);
+  // Programmatic stream serialisation: back-to-back launches of this kernel overlap the tail of one grid with the
+  // CTA start-up of the next (the kernel waits for its predecessors before its first global access).  After a
+  // kernel that never signals its dependents the launch behaves like an ordinary one.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(n_tasks < sms ? n_tasks : sms));
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = L.total;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, packed_gemv_tc_kernel, mw, X, s16, static_cast<const uint8_t*>(zq), Y, d.out_features,
+                         d.in_features, group_shift, ng, T, vec_params, stages) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return EQAT_ERR_CUDA;
+  }
   return launch_status();
 }
 
 }  // namespace
 
-// 2-bit codes with byte zero points go through the tensor-core kernel whenever its shared-memory plan fits.
-static int tc_stages_for(const eqat_desc& d) {
-  if (d.bits != 2 || d.group < 64 || d.tokens < 1 || d.tokens > kTcMaxTokens) return 0;
-  if (d.zero_point_format != EQAT_ZP_U8) return 0;
-  return tc_stages_that_fit((int)d.tokens, d.in_features);
+// 2-bit codes with byte zero points go through the tensor-core kernel: in one launch when the shared-memory plan
+// fits all tokens, otherwise (long rows, or more than eight tokens) as several launches over slices of the tokens,
+// each of which streams the packed weight once more.  That is taken only while it is clearly cheaper than the
+// tiled kernel of gemm.cu.  Cost model (from timings on the Llama-2 7B and 70B shapes): a launch of this kernel
+// takes about 4 us + 0.5 us per token + the packed weight at 1.6 TB/s; the tiled kernel takes about 1 us per 64
+// input columns for any token count below a full row-tile, because the K loop of a tile is serial.
+struct TcPlan {
+  int launches, slice;                                   // slice = tokens per launch (the last one may have fewer)
+};
+
+static TcPlan tc_plan(const eqat_desc& d) {
+  const TcPlan none{0, 0};
+  if (d.bits != 2 || d.group < 64 || d.tokens < 1 || d.tokens > kTcMaxTotalTokens) return none;
+  if (d.zero_point_format != EQAT_ZP_U8) return none;
+  const int T = (int)d.tokens;
+  int fit = T < kTcMaxTokens ? T : kTcMaxTokens;
+  while (fit >= 1 && tc_stages_that_fit(fit, d.in_features) == 0) --fit;
+  if (fit < 1) return none;
+  const int launches = (T + fit - 1) / fit, slice = (T + launches - 1) / launches;
+  if (launches > 1) {
+    const double weight_mb = (double)d.out_features * d.in_features / 4.0 / 1.0e6;
+    const double few_us = launches * (4.0 + 0.5 * slice + weight_mb / 1.6), tiled_us = d.in_features / 64.0;
+    if (few_us >= 0.8 * tiled_us) return none;
+  }
+  return TcPlan{launches, slice};
 }
 
 bool packed_gemv_applies(const eqat_desc& d) {
   // a 64-code unit must lie inside one group: groups of 32 go through the tiled kernel
   if (d.tokens < 1 || d.group < 64) return false;
-  if (tc_stages_for(d) > 0) return true;                 // up to eight tokens
+  if (tc_plan(d).launches > 0) return true;
   return d.tokens <= kGemvMaxTokens && smem_floats((int)d.tokens, d.in_features) * sizeof(float) <= kMaxSmem;
 }
 
@@ -788,8 +838,17 @@ int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq
     group_shift = 0;
     while ((1 << group_shift) < d.group) ++group_shift;
   }
-  const int tc_stages = tc_stages_for(d);
-  if (tc_stages > 0) return launch_tc(d, X, Wq, s16, zq, Y, group_shift, tc_stages, st);
+  const TcPlan plan = tc_plan(d);
+  if (plan.launches > 0) {
+    for (int t0 = 0; t0 < (int)d.tokens; t0 += plan.slice) {
+      eqat_desc part = d;
+      part.tokens = (int)d.tokens - t0 < plan.slice ? (int)d.tokens - t0 : plan.slice;
+      const int rc = launch_tc(part, X + (size_t)t0 * d.in_features, Wq, s16, zq, Y + (size_t)t0 * d.out_features,
+                               group_shift, tc_stages_that_fit((int)part.tokens, d.in_features), st);
+      if (rc != EQAT_OK) return rc;
+    }
+    return EQAT_OK;
+  }
   switch (d.bits) {
     case 2: return launch_bits<2>(d, X, Wq, s16, zq, Y, group_shift, st);
     case 3: return launch_bits<3>(d, X, Wq, s16, zq, Y, group_shift, st);

@@ -8,8 +8,9 @@ namespace eqat {
 constexpr int kGemvMaxTokens = 4;
 
 // True when a small-batch kernel handles this problem: groups of at least 64 elements and either 2-bit codes with
-// byte zero points and at most eight tokens (tensor-core kernel), or at most kGemvMaxTokens tokens, groups of at least 64
-// elements and activations (as fp32) that fit in the shared memory of one CTA.
+// byte zero points and at most 32 tokens (tensor-core kernel, at most eight tokens per launch; several launches only
+// while they are cheaper than the tiled kernel), or at most kGemvMaxTokens tokens and activations (as fp32) that fit
+// in the shared memory of one CTA.
 bool packed_gemv_applies(const eqat_desc& d);
 // Y[T,out] = X[T,in] * dequant(Wq)^T for a problem packed_gemv_applies() accepted
 int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,

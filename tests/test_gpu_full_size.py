@@ -10,7 +10,7 @@ each sampled block by its norm and element by element (helpers.contraction_bound
 always covers the last row-tile and the last column-tile of Y and dX (last 256 tokens x last 256 outputs /
 inputs), where a ragged edge would show; and whole-tensor identities that hold at any size tie the rest together:
   <dY, Y> = <dX, X>  (adjoint),  sum s*ds = <dY, Y>  (Y is linear in s).
-The E2E-QP cases also push the first one and four tokens through the forward alone (decoding).
+The E2E-QP cases also push the first 1, 4, 8 and 20 tokens through the forward alone (decoding).
 """
 import numpy as np
 import pytest
@@ -181,9 +181,10 @@ def test_full_size(eqat, cfg_name, lin_name, mode):
         assert abs(a - b) <= tol_abs
         euler = float((s16.double() * ds.double()).sum())
         assert abs(euler - a) <= tol_abs
-        # decoding: the first one and four tokens alone (the matrix-vector kernel where its activations fit in shared
-        # memory, the tiled kernel otherwise), against the oracle and against the same rows of the full batch
-        for t_few in (1, 4):
+        # decoding: the first one, four, eight and twenty tokens alone (the matrix-vector kernels where their
+        # activations fit in shared memory, whole or in slices of the tokens; the tiled kernel otherwise), against the
+        # oracle and against the same rows of the full batch
+        for t_few in (1, 4, 8, 20):
             d_few = eqat.make_desc(bits, g, out, in_f, t_few)
             Y_few = torch.empty(t_few, out, dtype=torch.bfloat16, device="cuda")
             eqat.qlinear_packed_fwd(d_few, Xd[:t_few].contiguous(), P, s16, z8, Y_few)

@@ -534,7 +534,7 @@ def test_e2e_small(eqat, bits, group, real_z):
 @pytest.mark.parametrize("tokens", [1, 2, 3, 4, 5, 7, 8, 9])
 def test_e2e_few_tokens(eqat, bits, tokens):
     """Decode-sized batches: up to four tokens (eight for 2-bit codes) take a matrix-vector forward kernel, more the
-    tiled one.
+    tiled one (rows this short are not worth several launches).
     640 = 10 units of 64 columns, fewer than the sixteen warps of a CTA (some get none); 1408 = 22 (one or two each)."""
     group = 64 if bits == 2 else 128
     cfg = small_cfg(f"gemv_{bits}_{tokens}", 448, 640 if group == 64 else 1408, bits, group, tokens, "student_t4", 0.02, 0.01)
@@ -585,6 +585,63 @@ def test_few_token_forward_is_deterministic(eqat):
     assert rel_err(torch_to_f64(ref), O.linear_fwd(torch_to_f64(X), What_o)) <= TOL
 
 
+def few_token_problem(out, in_f, tokens, seed):
+    g = torch.Generator(device="cuda"); g.manual_seed(seed)
+    P = torch.randint(0, 256, (out, in_f // 4), dtype=torch.uint8, device="cuda", generator=g)
+    z8 = torch.randint(1, 3, (out, in_f // 64), dtype=torch.uint8, device="cuda", generator=g)
+    s16 = (torch.rand(out, in_f // 64, device="cuda", generator=g) * 0.004 + 0.012).half()
+    X = torch.randn(tokens, in_f, device="cuda", generator=g).to(torch.bfloat16)
+    return P, z8, s16, X
+
+
+def test_few_token_forward_does_not_depend_on_the_slicing(eqat):
+    """Thirteen tokens go out as two launches (seven and six tokens); every token's row must be bit for bit what the
+    token gives alone, and what it gives in a batch of eight (one launch)."""
+    out, in_f, T = 1280, 4096, 13
+    P, z8, s16, X = few_token_problem(out, in_f, T, 21)
+    guard = Guarded()
+    Y = guard.empty(T, out, dtype=torch.bfloat16)
+    eqat.qlinear_packed_fwd(eqat.make_desc(2, 64, out, in_f, T), X, P, s16, z8, Y)
+    Y8 = guard.empty(8, out, dtype=torch.bfloat16)
+    eqat.qlinear_packed_fwd(eqat.make_desc(2, 64, out, in_f, 8), X[:8].contiguous(), P, s16, z8, Y8)
+    guard.check()
+    assert torch.equal(Y8.view(torch.int16), Y[:8].view(torch.int16))
+    d1 = eqat.make_desc(2, 64, out, in_f, 1)
+    for t in range(T):
+        y = torch.empty(1, out, dtype=torch.bfloat16, device="cuda")
+        eqat.qlinear_packed_fwd(d1, X[t:t + 1].contiguous(), P, s16, z8, y)
+        torch.cuda.synchronize()
+        assert torch.equal(y.view(torch.int16), Y[t:t + 1].view(torch.int16)), t
+    q = O.unpack_rows(P.cpu().numpy(), 2, in_f)
+    What_o = O.dequantize(q, s16.cpu().numpy().astype(np.float32), z8.cpu().numpy(), 64)
+    assert rel_err(torch_to_f64(Y), O.linear_fwd(torch_to_f64(X), What_o)) <= TOL
+
+
+@pytest.mark.parametrize("tokens", [1, 8, 12])
+def test_few_token_forwards_back_to_back_keep_their_order(eqat, tokens):
+    """Twelve layers in a row, each reading what the one before wrote, issued without a pause (the launches may
+    overlap their start-up with the tail of the launch before) and again with a synchronise after every call."""
+    n = 4096
+    Ps = [few_token_problem(n, n, tokens, 30 + i)[0] for i in range(12)]
+    _, z8, s16, X0 = few_token_problem(n, n, tokens, 29)
+    d = eqat.make_desc(2, 64, n, n, tokens)
+
+    def chain(pause):
+        bufs = [X0.clone(), torch.zeros_like(X0)]
+        for i, P in enumerate(Ps):
+            eqat.qlinear_packed_fwd(d, bufs[i & 1], P, s16, z8, bufs[(i + 1) & 1])
+            if pause:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        return bufs[len(Ps) & 1].clone()
+
+    ref = chain(True)
+    assert torch.isfinite(ref.float()).all() and float(ref.float().abs().max()) > 1e-3
+    for _ in range(10):
+        assert torch.equal(chain(False).view(torch.int16), ref.view(torch.int16))
+    assert eqat.device_status() == (0, 0)
+
+
 @pytest.mark.parametrize("out,in_f,tokens,bits,group", [
     (192, 384, 300, 2, 64),
     (64, 128, 1, 4, 128),
@@ -602,6 +659,10 @@ def test_few_token_forward_is_deterministic(eqat):
     (64, 128, 1, 2, 64),            # rows of 32 bytes: a quarter of the copy engine's 128-byte box
     (64, 256, 8, 2, 128),           # eight tokens, the most the matrix-vector kernel takes
     (2432, 512, 4, 2, 64),          # more row-blocks than SMs: every CTA takes a second task, parameters loaded as vectors
+    (64, 11008, 8, 2, 64),          # eight tokens whose staged activations do not fit: two launches of four
+    (128, 4096, 13, 2, 64),         # more than eight tokens: slices of seven and six
+    (128, 8192, 31, 2, 128),        # five slices (7, 7, 7, 7, 3)
+    (64, 28672, 4, 2, 64),          # the longest rows of the 70B block: two tokens per launch
 ])
 def test_e2e_ragged(eqat, out, in_f, tokens, bits, group):
     cfg = small_cfg(f"e2er_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens)
