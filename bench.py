@@ -890,9 +890,11 @@ def decode_leg(eqat, dev, peaks, iters, model="7b"):
     """Few-token packed forward (the matrix-vector kernels) on the linear shapes of one block: device time per
     launch from a CUDA graph of launches over rotating weight copies (more than L2 in total), and the bandwidth that
     time means for the bytes one launch must read."""
-    out = {"metric": "packed forward, few tokens", "unit": "us per launch", "bits": BITS, "group": GROUP,
+    out = {"metric": "packed forward, few tokens", "unit": "us per call", "bits": BITS, "group": GROUP,
            "model": model, "hbm_gbs_peak": peaks["hbm_gbs"],
-           "method": "CUDA graph of one launch per weight copy (copies total > 2 x L2), replayed back to back", "cases": {}}
+           "method": "CUDA graph of one call per weight copy (copies total > 2 x L2), replayed back to back; a call "
+                     "is one kernel launch for up to 8 tokens where the staged activations fit, else one per token slice",
+           "cases": {}}
     for lin in LINEARS[model]:
         o, i = lin.out_features, lin.in_features
         ng = i // GROUP
