@@ -886,27 +886,27 @@ def run_streaming_case(args):
     print(json.dumps(r), flush=True)
 
 
-def decode_leg(eqat, dev, peaks, iters, model="7b"):
+def decode_leg(eqat, dev, peaks, iters, model="7b", bits=BITS, group=GROUP):
     """Few-token packed forward (the matrix-vector kernels) on the linear shapes of one block: device time per
     launch from a CUDA graph of launches over rotating weight copies (more than L2 in total), and the bandwidth that
     time means for the bytes one launch must read."""
-    out = {"metric": "packed forward, few tokens", "unit": "us per call", "bits": BITS, "group": GROUP,
+    out = {"metric": "packed forward, few tokens", "unit": "us per call", "bits": bits, "group": group,
            "model": model, "hbm_gbs_peak": peaks["hbm_gbs"],
            "method": "CUDA graph of one call per weight copy (copies total > 2 x L2), replayed back to back; a call "
                      "is one kernel launch for up to 8 tokens where the staged activations fit, else one per token slice",
            "cases": {}}
     for lin in LINEARS[model]:
         o, i = lin.out_features, lin.in_features
-        ng = i // GROUP
-        wbytes = o * i * BITS // 8
+        ng = i // group
+        wbytes = o * i * bits // 8
         copies = max(4, int(320e6 // wbytes))
-        Ps = [torch.randint(0, 256, (o, i * BITS // 8), dtype=torch.uint8, device=dev) for _ in range(copies)]
-        z8 = torch.randint(0, 1 << BITS, (o, ng), dtype=torch.uint8, device=dev)
+        Ps = [torch.randint(0, 256, (o, i * bits // 8), dtype=torch.uint8, device=dev) for _ in range(copies)]
+        z8 = torch.randint(0, 1 << bits, (o, ng), dtype=torch.uint8, device=dev)
         s16 = (torch.rand(o, ng, device=dev) * 0.01 + 0.001).half()
         for T in (1, 4, 8, 16):
             X = torch.randn(T, i, device=dev).to(torch.bfloat16)
             Y = torch.empty(T, o, dtype=torch.bfloat16, device=dev)
-            d = eqat.make_desc(BITS, GROUP, o, i, T)
+            d = eqat.make_desc(bits, group, o, i, T)
             us = time_rotation([lambda P=P: eqat.qlinear_packed_fwd(d, X, P, s16, z8, Y) for P in Ps], iters)
             nbytes = wbytes + o * ng * 3 + T * (i + o) * 2
             out["cases"][f"{lin.name}/T{T}"] = {"us": us, "bytes": nbytes, "gbs": nbytes / us / 1e3,
@@ -922,7 +922,8 @@ def run_decode_case(args):
     from paper_2407_11062_b200.build import build_library
     build_library()
     from paper_2407_11062_b200 import binding as eqat
-    out = decode_leg(eqat, torch.device("cuda", 0), load_peaks(), args.case_iters, args.case_model)
+    out = decode_leg(eqat, torch.device("cuda", 0), load_peaks(), args.case_iters, args.case_model, args.case_bits,
+                     args.case_group)
     assert eqat.device_status() == (0, 0)
     print(json.dumps(out), flush=True)
 

@@ -229,7 +229,7 @@ int eqat_unpack_zeros(const eqat_desc* desc, const uint8_t* z_packed, uint8_t* z
  * shared memory inside the GEMM (Eq. 2; Sec. 3.3).  With one to four tokens
  * (decoding) and groups of at least 64 a matrix-vector kernel streams the
  * packed weight instead and does not round (W_int - z) * s to bf16.  For 2-bit
- * codes with byte zero points that kernel takes up to eight tokens per launch,
+ * and 4-bit codes with byte zero points it takes up to eight tokens per launch,
  * and up to 32 tokens go through it in slices (one pass over the packed weight
  * per slice) while that is cheaper than the tiled kernel; a token's result
  * does not depend on how the tokens were sliced.

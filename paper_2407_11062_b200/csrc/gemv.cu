@@ -276,9 +276,9 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 }
 
 
-// ====================================================================== 2-bit codes on tensor-core tiles
+// ====================================================================== 2-bit and 4-bit codes on tensor-core tiles
 // The kernel above spends three instructions per code and token on the ordinary
-// cores.  For 2-bit codes that is several times what the bytes allow, so they go
+// cores.  That is several times what the bytes allow, so 2-bit and 4-bit codes go
 // through warp-level matrix instructions instead (mma.sync m16n8k16, bf16 in,
 // fp32 out): 16 weight rows by 16 columns against up to 8 tokens per
 // instruction, with the weight fragment built in registers, one logic
@@ -287,8 +287,9 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // avoid here; and with at most a few tokens there is nothing for a 128-row
 // accumulator to amortise.)
 //
-// Fragment construction.  A 32-bit word of the stream holds 16 consecutive codes
-// of one row, code j at bits [2j, 2j + 2).  (w >> 2p) & 0x00030003 isolates codes
+// Fragment construction, 2-bit codes (4-bit codes: expand_words4, one shift and
+// one logic operation per pair of codes, constant 128 throughout).  A 32-bit word
+// of the stream holds 16 consecutive codes of one row, code j at bits [2j, 2j + 2).  (w >> 2p) & 0x00030003 isolates codes
 // p and p + 8 in the two halves of a register; OR-ing 0x4300 into each half makes
 // them the bf16 numbers 128 + q.  For p = 1, 2 (mod 3) the shift is skipped: a
 // code left at bits 2-3 (4-5) of a half with 0x4200 (0x4100) above it is the
@@ -306,11 +307,13 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // CTAs take tasks round-robin.  The producer thread copies the task's codes into
 // a shared-memory ring as [16 rows x 128 bytes] boxes (cp.async.bulk.tensor,
 // 128-byte swizzle, bytes past the end of a row arrive as zeros), eight boxes
-// per stage.  Consumer warp w owns half of box w/2 of every stage: four chunks of
-// 16 bytes = 64 columns = the four words of the four lanes of a quad, so a
+// per stage (sixteen for 4-bit codes).  Consumer warp w owns half of box w/2 of every stage: four chunks of
+// 16 bytes = 64 columns = the four words of the four lanes of a quad (4-bit
+// codes: two chunks of 32 bytes, two words per lane), so a
 // chunk lies in one quantisation group and its accumulator is scaled by one step
 // size per row.  Lane (g, q) of the warp holds rows g and g + 8 and, in
-// instruction m of a chunk, supplies codes 2m, 2m+8, 2m+1, 2m+9 of its word;
+// instruction m of a chunk, supplies codes 2m, 2m+8, 2m+1, 2m+9 of its word
+// (tc_column gives the order for either width);
 // the activations are staged once per CTA in exactly that order, so a lane
 // fetches its fragment of X with one 8-byte load.  Zero points are one byte
 // each here (the fp16 variant goes through the kernel above).  The 16 warps'
@@ -323,13 +326,15 @@ constexpr int kTcWarps = 16;
 constexpr int kTcThreads = (kTcWarps + 2) * 32;        // + producer warp + reducer warp
 constexpr int kTcRows = 16;                            // weight rows per task
 constexpr int kTcBoxBytes = 128;
-constexpr int kTcBoxesPerStage = 8;
+// Boxes per stage: every consumer warp has four chunks of a stage, i.e. half a box of 2-bit codes (8 boxes,
+// 16 KB per stage) or a whole box of 4-bit codes (16 boxes, 32 KB per stage).
+__host__ __device__ constexpr int tc_boxes_per_stage(int bits) { return 4 * bits; }
 constexpr int kTcBoxSmem = kTcRows * kTcBoxBytes;      // 2 KB
-constexpr int kTcStageBytes = kTcBoxesPerStage * kTcBoxSmem;   // 16 KB: 16 rows x 1024 bytes
+__host__ __device__ constexpr int tc_stage_bytes(int bits) { return tc_boxes_per_stage(bits) * kTcBoxSmem; }
 constexpr int kTcAhead = 3;                            // stages of lead of the parameter loads
 constexpr int kTcItems = 5;                            // instructions per chunk: four on codes, one correction
 constexpr int kTcMaxStages = 8;
-constexpr int kTcMinStages = 3;
+__host__ __device__ constexpr int tc_min_stages(int bits) { return bits == 2 ? 3 : 2; }   // 48 KB / 64 KB in flight
 constexpr uint64_t kTcWaitLimitNs = 2000000000ull;
 constexpr size_t kTcSmemBudget = 227 * 1024;             // the most a CTA can be given (eight tokens of 8192 columns need 225.2 KB)
 
@@ -346,23 +351,24 @@ struct TcLayout {
   int stages;
 };
 
-// Shared-memory plan for T tokens and in_features columns.
-__host__ __device__ inline TcLayout tc_layout(int T, int in_features, int stages) {
+// Shared-memory plan for T tokens and in_features columns of `bits`-bit codes.
+__host__ __device__ inline TcLayout tc_layout(int T, int in_features, int stages, int bits) {
   TcLayout L;
-  // chunks of 64 columns, counted up to the end of the last (possibly partial) 512-column box: the entries past
-  // in_features are zeros, so the compute loop needs no end-of-row case
-  const size_t chunks = (size_t)((in_features + 511) / 512) * 8;
+  // chunks of 64 columns, counted up to the end of the last (possibly partial) 128-byte box (512 columns of 2-bit
+  // codes, 256 of 4-bit codes): the entries past in_features are zeros, so the compute loop needs no end-of-row case
+  const int box_cols = kTcBoxBytes * 8 / bits;
+  const size_t chunks = (size_t)((in_features + box_cols - 1) / box_cols) * (box_cols / 64);
   L.stages = stages;
-  L.xb_off = (size_t)stages * kTcStageBytes;
+  L.xb_off = (size_t)stages * tc_stage_bytes(bits);
   L.part_off = L.xb_off + chunks * kTcItems * 4 * T * 8;             // permuted bf16 activations + correction terms
   L.ctl_off = L.part_off + (size_t)2 * kTcWarps * kTcRows * kTcMaxTokens * 4;
   L.total = L.ctl_off + sizeof(TcCtl) + 1024 /*alignment slack*/;
   return L;
 }
 
-inline int tc_stages_that_fit(int T, int in_features) {
-  for (int st = kTcMaxStages; st >= kTcMinStages; --st)
-    if (tc_layout(T, in_features, st).total <= kTcSmemBudget) return st;
+inline int tc_stages_that_fit(int T, int in_features, int bits) {
+  for (int st = kTcMaxStages; st >= tc_min_stages(bits); --st)
+    if (tc_layout(T, in_features, st, bits).total <= kTcSmemBudget) return st;
   return 0;
 }
 
@@ -421,22 +427,41 @@ __device__ __forceinline__ void expand_word2(uint32_t w, uint32_t (&P)[8]) {
   P[6] = and_or(t2, 0x00030003u, 0x43004300u);
   P[7] = and_or(t2, 0x000C000Cu, 0x42004200u);
 }
-// Constant that expand_word2 adds to code j (0..15) of a word.
-__host__ __device__ inline float tc_bias(int j) {
-  const int r = (j & 7) % 3;
-  return r == 0 ? 128.0f : (r == 1 ? 32.0f : 8.0f);
+// 4-bit codes: a word holds eight, code j at bits [4j, 4j + 4).  A lane's two words (16 consecutive columns)
+// give the registers (code p, code p + 4) of each word, all with the constant 128; the codes fill the low four
+// mantissa bits, so there is no room to skip a shift.
+__device__ __forceinline__ void expand_words4(uint32_t w0, uint32_t w1, uint32_t (&P)[8]) {
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    P[p] = and_or(w0 >> (4 * p), 0x000F000Fu, 0x43004300u);
+    P[4 + p] = and_or(w1 >> (4 * p), 0x000F000Fu, 0x43004300u);
+  }
+}
+// Which of a lane's 16 columns sits in half `half` (0 = low) of register r (0..7) of the expansion.
+template <int BITS>
+__host__ __device__ constexpr int tc_column(int r, int half) {
+  return BITS == 2 ? r + 8 * half : (r < 4 ? r + 4 * half : r + 4 + 4 * half);
+}
+// Constant that the expansion adds to column j (0..15) of a lane.
+template <int BITS>
+__host__ __device__ constexpr float tc_bias(int j) {
+  return BITS == 4 ? 128.0f : ((j & 7) % 3 == 0 ? 128.0f : ((j & 7) % 3 == 1 ? 32.0f : 8.0f));
 }
 
+template <int BITS, int PARAM_MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16* __restrict__ X,
                       const eqat_fp16* __restrict__ s16, const uint8_t* __restrict__ z8, eqat_bf16* __restrict__ Y,
-                      int out_features, int in_features, int group_shift, int groups_per_row, int T, int vec_params,
-                      int stages) {
+                      int out_features, int in_features, int group_shift, int groups_per_row, int T, int stages) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_addr(smem_raw);
   const uint32_t ring_addr = (raw_addr + 1023u) & ~1023u;          // boxes are 1024-byte aligned (swizzle period)
   uint8_t* ring = smem_raw + (ring_addr - raw_addr);
-  const TcLayout L = tc_layout(T, in_features, stages);
+  constexpr int kChunksPerBox = kTcBoxBytes * 8 / BITS / 64;        // 64-column chunks of a row per box: 8 or 4
+  constexpr int kChunksPerWarp = 4;                                 // half a box (2-bit codes) or a box (4-bit codes)
+  constexpr int kBoxesPerStage = tc_boxes_per_stage(BITS);
+  constexpr int kStageBytes = tc_stage_bytes(BITS);
+  const TcLayout L = tc_layout(T, in_features, stages, BITS);
   uint2* xb = reinterpret_cast<uint2*>(ring + L.xb_off);           // [chunk][item][quad lane][token] -> 4 bf16
   float* part = reinterpret_cast<float*>(ring + L.part_off);       // [2][warp][row][kTcMaxTokens]
   TcCtl* ctl = reinterpret_cast<TcCtl*>(ring + L.ctl_off);
@@ -444,10 +469,10 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tasks = out_features / kTcRows;
   const int chunks = in_features >> 6;
-  const int row_bytes = in_features >> 2;
+  const int row_bytes = in_features * BITS / 8;
   const int n_boxes = (row_bytes + kTcBoxBytes - 1) / kTcBoxBytes;
-  const int task_stages = (n_boxes + kTcBoxesPerStage - 1) / kTcBoxesPerStage;
-  const int chunks_pad = n_boxes * 8;
+  const int task_stages = (n_boxes + kBoxesPerStage - 1) / kBoxesPerStage;
+  const int chunks_pad = n_boxes * kChunksPerBox;
 
   // Launched with programmatic stream serialisation: the next launch of the stream may start as soon as every
   // CTA of this grid has got here, and a CTA of this grid may be running while the launch before it still is.
@@ -483,27 +508,43 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
   }
 
   const int g = lane >> 2, q = lane & 3;
-  const int box = warp >> 1, chunk0 = (warp & 1) * 4;
-  // Step sizes (four fp16) and zero points (four bytes) of this lane's four chunks of stage k of a task, rows g
-  // and g + 8.  With groups of 64 and rows of parameters that keep their alignment (vec_params) the four chunks
-  // are four consecutive groups: one load per row and kind.
+  const int box = BITS == 2 ? warp >> 1 : warp, chunk0 = BITS == 2 ? (warp & 1) * kChunksPerWarp : 0;
+  // Step sizes (fp16) and zero points (bytes) of this lane's four chunks of stage k of a task, rows g and g + 8,
+  // in up to four slots.  The four chunks are 256 consecutive columns starting at a multiple of 256: four groups
+  // of 64 (mode 1), two groups of 128 (mode 2) or part of one larger group (mode 3), fetched with one load per row
+  // and kind where the rows of parameters keep the alignment for it; mode 0 fetches chunk by chunk.  Chunk c uses
+  // slot c >> kSlotShift.  The loaded registers are not touched before the stage is computed (three stages later):
+  // an instruction on them here would wait for the load.
   struct StageParams { uint2 s_lo, s_hi; uint32_t z_lo, z_hi; };
+  constexpr int kSlotShift = PARAM_MODE == 2 ? 1 : (PARAM_MODE == 3 ? 2 : 0);
   auto fetch = [&](int task, int k) {
     StageParams sp;
     sp.s_lo = sp.s_hi = make_uint2(0u, 0u);
     sp.z_lo = sp.z_hi = 0u;
-    const int cg0 = (k * kTcBoxesPerStage + box) * 8 + chunk0;
+    const int cg0 = (k * kBoxesPerStage + box) * kChunksPerBox + chunk0;
     if (task < n_tasks && cg0 < chunks) {
       const size_t p_lo = (size_t)(task * kTcRows + g) * groups_per_row, p_hi = p_lo + (size_t)8 * groups_per_row;
-      if (vec_params) {                                   // chunks is a multiple of 4 here: all four exist
+      if constexpr (PARAM_MODE == 1) {                    // the row has a multiple of four groups: all four exist
         sp.s_lo = __ldg(reinterpret_cast<const uint2*>(s16 + p_lo + cg0));
         sp.s_hi = __ldg(reinterpret_cast<const uint2*>(s16 + p_hi + cg0));
         sp.z_lo = __ldg(reinterpret_cast<const uint32_t*>(z8 + p_lo + cg0));
         sp.z_hi = __ldg(reinterpret_cast<const uint32_t*>(z8 + p_hi + cg0));
+      } else if constexpr (PARAM_MODE == 2) {             // an even number of groups per row: both exist
+        const int g0 = cg0 >> 1;
+        sp.s_lo.x = __ldg(reinterpret_cast<const uint32_t*>(s16 + p_lo + g0));
+        sp.s_hi.x = __ldg(reinterpret_cast<const uint32_t*>(s16 + p_hi + g0));
+        sp.z_lo = __ldg(reinterpret_cast<const uint16_t*>(z8 + p_lo + g0));
+        sp.z_hi = __ldg(reinterpret_cast<const uint16_t*>(z8 + p_hi + g0));
+      } else if constexpr (PARAM_MODE == 3) {
+        const int grp = (cg0 << 6) >> group_shift;
+        sp.s_lo.x = __ldg(s16 + p_lo + grp);
+        sp.s_hi.x = __ldg(s16 + p_hi + grp);
+        sp.z_lo = __ldg(z8 + p_lo + grp);
+        sp.z_hi = __ldg(z8 + p_hi + grp);
       } else {
         uint32_t sl[4] = {0u, 0u, 0u, 0u}, sh[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < kChunksPerWarp; ++c) {
           if (cg0 + c < chunks) {
             const int grp = ((cg0 + c) << 6) >> group_shift;
             sl[c] = __ldg(s16 + p_lo + grp);
@@ -547,12 +588,12 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
             break;
           }
           ptx::fence_proxy_async_smem();                            // consumers' reads of this stage before the copies' writes
-          const int nb = min(kTcBoxesPerStage, n_boxes - k * kTcBoxesPerStage);
+          const int nb = min(kBoxesPerStage, n_boxes - k * kBoxesPerStage);
           const uint32_t full = ptx::smem_addr(&ctl->full[slot]);
           ptx::mbar_expect_tx(full, (uint32_t)nb * kTcBoxSmem);     // bytes past the end of a row are zero-filled and counted
           for (int b = 0; b < nb; ++b)
-            ptx::tma_load_2d(ring_addr + slot * kTcStageBytes + b * kTcBoxSmem, &map_w,
-                             (k * kTcBoxesPerStage + b) * kTcBoxBytes, task * kTcRows, full);
+            ptx::tma_load_2d(ring_addr + slot * kStageBytes + b * kTcBoxSmem, &map_w,
+                             (k * kBoxesPerStage + b) * kTcBoxBytes, task * kTcRows, full);
           ++issued;
           if (++slot == stages) { slot = 0; phase ^= 1u; }
         }
@@ -619,7 +660,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
 #pragma unroll
           for (int j = 0; j < 16; ++j) {                               // fixed order, four short chains
             const float xv = __uint_as_float(h[j] << 16);
-            sb4[j & 3] = fmaf(tc_bias(j), xv, sb4[j & 3]);
+            sb4[j & 3] = fmaf(tc_bias<BITS>(j), xv, sb4[j & 3]);
             sx4[j & 3] += xv;
           }
           sb = (sb4[0] + sb4[1]) + (sb4[2] + sb4[3]);
@@ -627,7 +668,8 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
 #pragma unroll
           for (int m = 0; m < 4; ++m)
             xb[(((size_t)cg * kTcItems + m) * 4 + uq) * T + t] =
-                make_uint2(h[2 * m] | (h[2 * m + 8] << 16), h[2 * m + 1] | (h[2 * m + 9] << 16));
+                make_uint2(h[tc_column<BITS>(2 * m, 0)] | (h[tc_column<BITS>(2 * m, 1)] << 16),
+                           h[tc_column<BITS>(2 * m + 1, 0)] | (h[tc_column<BITS>(2 * m + 1, 1)] << 16));
         }
         sb += __shfl_xor_sync(0xFFFFFFFFu, sb, 1); sx += __shfl_xor_sync(0xFFFFFFFFu, sx, 1);
         sb += __shfl_xor_sync(0xFFFFFFFFu, sb, 2); sx += __shfl_xor_sync(0xFFFFFFFFu, sx, 2);
@@ -666,7 +708,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
     for (int task = blockIdx.x; task < n_tasks && alive; task += gridDim.x) {
       float tot[4] = {0.0f, 0.0f, 0.0f, 0.0f};                         // rows g, g + 8 x tokens 2q, 2q + 1
       for (int k = 0; k < task_stages; ++k) {
-        const int gbox = k * kTcBoxesPerStage + box;
+        const int gbox = k * kBoxesPerStage + box;
         const bool have = gbox < n_boxes;
         const StageParams sp = nx[0];
 #pragma unroll
@@ -675,15 +717,22 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
         advance();
         const bool got = tc_wait(ptx::smem_addr(&ctl->full[slot]), phase, abort_flag, WAIT_STREAM_FULL, 0);
         if (!__all_sync(0xFFFFFFFFu, got)) { alive = false; break; }
-        uint32_t w_lo[4], w_hi[4];
+        uint32_t w_lo[kChunksPerWarp][BITS / 2], w_hi[kChunksPerWarp][BITS / 2];   // a lane's 16 codes per row and chunk
         if (have) {
           // 16-byte piece c of row r sits at piece (c ^ (r & 7)); rows g and g + 8 share the pattern
-          const uint32_t row = ring_addr + slot * kTcStageBytes + box * kTcBoxSmem + g * kTcBoxBytes + q * 4;
+          const uint32_t row = ring_addr + slot * kStageBytes + box * kTcBoxSmem + g * kTcBoxBytes;
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const uint32_t a = row + ((uint32_t)((chunk0 + c) ^ g) << 4);
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w_lo[c]) : "r"(a) : "memory");
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w_hi[c]) : "r"(a + 8 * kTcBoxBytes) : "memory");
+          for (int c = 0; c < kChunksPerWarp; ++c) {
+            if constexpr (BITS == 2) {                                 // word q of the chunk's one piece
+              const uint32_t a = row + ((uint32_t)((chunk0 + c) ^ g) << 4) + q * 4;
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w_lo[c][0]) : "r"(a) : "memory");
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w_hi[c][0]) : "r"(a + 8 * kTcBoxBytes) : "memory");
+            } else {                                                   // words 2q, 2q + 1 of the chunk's two pieces
+              const uint32_t a = row + ((uint32_t)(((chunk0 + c) * 2 + (q >> 1)) ^ g) << 4) + (q & 1) * 8;
+              asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(w_lo[c][0]), "=r"(w_lo[c][1]) : "r"(a) : "memory");
+              asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(w_hi[c][0]), "=r"(w_hi[c][1])
+                           : "r"(a + 8 * kTcBoxBytes) : "memory");
+            }
           }
         }
         // The stage's next user is a copy of the asynchronous proxy, which the barrier alone does not order after
@@ -694,11 +743,16 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
         if (++slot == stages) { slot = 0; phase ^= 1u; }
         if (have) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {                                // four independent chains, no branches
-            const int cg = gbox * 8 + chunk0 + c;
+          for (int c = 0; c < kChunksPerWarp; ++c) {                   // independent chains, no branches
+            const int cg = gbox * kChunksPerBox + chunk0 + c;
             uint32_t PL[8], PH[8];
-            expand_word2(w_lo[c], PL);
-            expand_word2(w_hi[c], PH);
+            if constexpr (BITS == 2) {
+              expand_word2(w_lo[c][0], PL);
+              expand_word2(w_hi[c][0], PH);
+            } else {
+              expand_words4(w_lo[c][0], w_lo[c][1], PL);
+              expand_words4(w_hi[c][0], w_hi[c][1], PH);
+            }
             const uint2* item = xb_lane + (size_t)cg * (kTcItems * 4) * T;
             float D[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
@@ -709,16 +763,17 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
             }
             {
               // correction: weights -1 and -(128 + z) against the split sums (see the header)
-              const uint32_t zz_lo = ((sp.z_lo >> (8 * c)) & 0xFFu) * 0x10001u;
-              const uint32_t zz_hi = ((sp.z_hi >> (8 * c)) & 0xFFu) * 0x10001u;
+              const uint32_t zz_lo = ((sp.z_lo >> (8 * (c >> kSlotShift))) & 0xFFu) * 0x10001u;
+              const uint32_t zz_hi = ((sp.z_hi >> (8 * (c >> kSlotShift))) & 0xFFu) * 0x10001u;
               uint2 b = make_uint2(0u, 0u);
               if (g < T) b = item[4 * 4 * T];
               mma_16816(D, and_or(zz_lo, mask_a, const_a), and_or(zz_hi, mask_a, const_a), and_or(zz_lo, mask_b, const_b),
                         and_or(zz_hi, mask_b, const_b), b.x, b.y);
             }
-            const uint32_t s2_lo = c < 2 ? sp.s_lo.x : sp.s_lo.y, s2_hi = c < 2 ? sp.s_hi.x : sp.s_hi.y;
-            const float s_lo = __half2float(__ushort_as_half((unsigned short)((c & 1) ? (s2_lo >> 16) : (s2_lo & 0xFFFFu))));
-            const float s_hi = __half2float(__ushort_as_half((unsigned short)((c & 1) ? (s2_hi >> 16) : (s2_hi & 0xFFFFu))));
+            const int slot = c >> kSlotShift;                          // a constant once the loop is unrolled
+            const uint32_t s2_lo = slot < 2 ? sp.s_lo.x : sp.s_lo.y, s2_hi = slot < 2 ? sp.s_hi.x : sp.s_hi.y;
+            const float s_lo = __half2float(__ushort_as_half((unsigned short)((slot & 1) ? (s2_lo >> 16) : (s2_lo & 0xFFFFu))));
+            const float s_hi = __half2float(__ushort_as_half((unsigned short)((slot & 1) ? (s2_hi >> 16) : (s2_hi & 0xFFFFu))));
             tot[0] = fmaf(s_lo, D[0], tot[0]);
             tot[1] = fmaf(s_lo, D[1], tot[1]);
             tot[2] = fmaf(s_hi, D[2], tot[2]);
@@ -760,20 +815,18 @@ __global__ void tc_wait_expiry_kernel(uint64_t limit_ns) {
   (void)tc_wait(ptx::smem_addr(&bar), 0u, &abort_word, WAIT_SELFTEST, 0, limit_ns);
 }
 
-int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
-              eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
+template <int BITS, int PARAM_MODE>
+int launch_tc_mode(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
+                   eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
   static SmemOptIn opt_in;
-  if (!opt_in.ensure(packed_gemv_tc_kernel, (int)kTcSmemBudget)) return EQAT_ERR_CUDA;
+  if (!opt_in.ensure(packed_gemv_tc_kernel<BITS, PARAM_MODE>, (int)kTcSmemBudget)) return EQAT_ERR_CUDA;
   CUtensorMap mw;
-  if (!make_tmap_u8(&mw, Wq, (uint64_t)d.in_features / 4, (uint64_t)d.out_features, kTcBoxBytes, kTcRows)) return EQAT_ERR_CUDA;
+  if (!make_tmap_u8(&mw, Wq, (uint64_t)d.in_features * BITS / 8, (uint64_t)d.out_features, kTcBoxBytes, kTcRows))
+    return EQAT_ERR_CUDA;
   const int sms = sm_count();
   if (sms <= 0) return EQAT_ERR_CUDA;
   const int T = (int)d.tokens, n_tasks = d.out_features / kTcRows, ng = d.in_features / d.group;
-  // four consecutive groups of a row with one load each: groups of 64, rows of parameters that stay 8-byte
-  // (step sizes) and 4-byte (zero points) aligned
-  const int vec_params = (d.group == 64 && ng % 4 == 0 && (reinterpret_cast<uintptr_t>(s16) & 7u) == 0 &&
-                          (reinterpret_cast<uintptr_t>(zq) & 3u) == 0) ? 1 : 0;
-  const TcLayout L = tc_layout(T, d.in_features, stages);
+  const TcLayout L = tc_layout(T, d.in_features, stages, BITS);
   // Programmatic stream serialisation: back-to-back launches of this kernel overlap the tail of one grid with the
   // CTA start-up of the next (the kernel waits for its predecessors before its first global access).  After a
   // kernel that never signals its dependents the launch behaves like an ordinary one.
@@ -787,38 +840,55 @@ int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const e
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, packed_gemv_tc_kernel, mw, X, s16, static_cast<const uint8_t*>(zq), Y, d.out_features,
-                         d.in_features, group_shift, ng, T, vec_params, stages) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, packed_gemv_tc_kernel<BITS, PARAM_MODE>, mw, X, s16, static_cast<const uint8_t*>(zq), Y,
+                         d.out_features, d.in_features, group_shift, ng, T, stages) != cudaSuccess) {
     (void)cudaGetLastError();
     return EQAT_ERR_CUDA;
   }
   return launch_status();
 }
 
+template <int BITS>
+int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
+              eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
+  // how a lane fetches the parameters of its 256 columns of a stage (see the kernel): one load per row and kind
+  // where the rows of step sizes and zero points keep the alignment those loads need, chunk by chunk otherwise
+  const uintptr_t s_addr = reinterpret_cast<uintptr_t>(s16), z_addr = reinterpret_cast<uintptr_t>(zq);
+  const int ng = d.in_features / d.group;
+  if (d.group == 64 && ng % 4 == 0 && (s_addr & 7u) == 0 && (z_addr & 3u) == 0)
+    return launch_tc_mode<BITS, 1>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
+  if (d.group == 128 && ng % 2 == 0 && (s_addr & 3u) == 0 && (z_addr & 1u) == 0)
+    return launch_tc_mode<BITS, 2>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
+  if (d.group >= 256) return launch_tc_mode<BITS, 3>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
+  return launch_tc_mode<BITS, 0>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
+}
+
 }  // namespace
 
-// 2-bit codes with byte zero points go through the tensor-core kernel: in one launch when the shared-memory plan
-// fits all tokens, otherwise (long rows, or more than eight tokens) as several launches over slices of the tokens,
-// each of which streams the packed weight once more.  That is taken only while it is clearly cheaper than the
-// tiled kernel of gemm.cu.  Cost model (from timings on the Llama-2 7B and 70B shapes): a launch of this kernel
-// takes about 4 us + 0.5 us per token + the packed weight at 1.6 TB/s; the tiled kernel takes about 1 us per 64
-// input columns for any token count below a full row-tile, because the K loop of a tile is serial.
+// 2-bit and 4-bit codes with byte zero points go through the tensor-core kernel: in one launch when the
+// shared-memory plan fits all tokens, otherwise (long rows, or more than eight tokens) as several launches over
+// slices of the tokens, each of which streams the packed weight once more.  That is taken only while it is clearly
+// cheaper than the tiled kernel of gemm.cu.  Cost model (from timings on the Llama-2 7B and 70B shapes): a launch
+// of this kernel takes about 4 us + 0.5 us per token + the packed weight at 1.6 TB/s (2-bit codes) or 2.5 TB/s
+// (4-bit codes); the tiled kernel takes about 1 us (1.2 us) per 64 input columns for any token count below a full
+// row-tile, because the K loop of a tile is serial.
 struct TcPlan {
   int launches, slice;                                   // slice = tokens per launch (the last one may have fewer)
 };
 
 static TcPlan tc_plan(const eqat_desc& d) {
   const TcPlan none{0, 0};
-  if (d.bits != 2 || d.group < 64 || d.tokens < 1 || d.tokens > kTcMaxTotalTokens) return none;
+  if ((d.bits != 2 && d.bits != 4) || d.group < 64 || d.tokens < 1 || d.tokens > kTcMaxTotalTokens) return none;
   if (d.zero_point_format != EQAT_ZP_U8) return none;
   const int T = (int)d.tokens;
   int fit = T < kTcMaxTokens ? T : kTcMaxTokens;
-  while (fit >= 1 && tc_stages_that_fit(fit, d.in_features) == 0) --fit;
+  while (fit >= 1 && tc_stages_that_fit(fit, d.in_features, d.bits) == 0) --fit;
   if (fit < 1) return none;
   const int launches = (T + fit - 1) / fit, slice = (T + launches - 1) / launches;
   if (launches > 1) {
-    const double weight_mb = (double)d.out_features * d.in_features / 4.0 / 1.0e6;
-    const double few_us = launches * (4.0 + 0.5 * slice + weight_mb / 1.6), tiled_us = d.in_features / 64.0;
+    const double weight_mb = (double)d.out_features * d.in_features * d.bits / 8.0 / 1.0e6;
+    const double stream_tbs = d.bits == 2 ? 1.6 : 2.5, tiled_us = d.in_features / 64.0 * (d.bits == 2 ? 1.0 : 1.2);
+    const double few_us = launches * (4.0 + 0.5 * slice + weight_mb / stream_tbs);
     if (few_us >= 0.8 * tiled_us) return none;
   }
   return TcPlan{launches, slice};
@@ -843,8 +913,11 @@ int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq
     for (int t0 = 0; t0 < (int)d.tokens; t0 += plan.slice) {
       eqat_desc part = d;
       part.tokens = (int)d.tokens - t0 < plan.slice ? (int)d.tokens - t0 : plan.slice;
-      const int rc = launch_tc(part, X + (size_t)t0 * d.in_features, Wq, s16, zq, Y + (size_t)t0 * d.out_features,
-                               group_shift, tc_stages_that_fit((int)part.tokens, d.in_features), st);
+      const int stages = tc_stages_that_fit((int)part.tokens, d.in_features, d.bits);
+      const eqat_bf16* Xs = X + (size_t)t0 * d.in_features;
+      eqat_bf16* Ys = Y + (size_t)t0 * d.out_features;
+      const int rc = d.bits == 2 ? launch_tc<2>(part, Xs, Wq, s16, zq, Ys, group_shift, stages, st)
+                                 : launch_tc<4>(part, Xs, Wq, s16, zq, Ys, group_shift, stages, st);
       if (rc != EQAT_OK) return rc;
     }
     return EQAT_OK;

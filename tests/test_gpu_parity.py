@@ -533,8 +533,8 @@ def test_e2e_small(eqat, bits, group, real_z):
 @pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("tokens", [1, 2, 3, 4, 5, 7, 8, 9])
 def test_e2e_few_tokens(eqat, bits, tokens):
-    """Decode-sized batches: up to four tokens (eight for 2-bit codes) take a matrix-vector forward kernel, more the
-    tiled one (rows this short are not worth several launches).
+    """Decode-sized batches: up to four tokens (eight for 2-bit and 4-bit codes) take a matrix-vector forward kernel,
+    more the tiled one (rows this short are not worth several launches).
     640 = 10 units of 64 columns, fewer than the sixteen warps of a CTA (some get none); 1408 = 22 (one or two each)."""
     group = 64 if bits == 2 else 128
     cfg = small_cfg(f"gemv_{bits}_{tokens}", 448, 640 if group == 64 else 1408, bits, group, tokens, "student_t4", 0.02, 0.01)
@@ -558,16 +558,17 @@ def test_few_token_forward_agrees_with_tiled_forward(eqat):
     assert rel_err(torch_to_f64(Y4), torch_to_f64(r5["Y"][:4])) <= TOL
 
 
-def test_few_token_forward_is_deterministic(eqat):
+@pytest.mark.parametrize("bits,group", [(2, 64), (4, 128), (4, 64)])
+def test_few_token_forward_is_deterministic(eqat, bits, group):
     """More row-blocks than SMs, several stages per row-block: the partial sums of the sixteen warps are added in
     a fixed order by one warp, so repeated launches must agree bit for bit (also while other work runs beside them)."""
     out, in_f, T = 2432, 5120, 3
     g = torch.Generator(device="cuda"); g.manual_seed(11)
-    P = torch.randint(0, 256, (out, in_f // 4), dtype=torch.uint8, device="cuda", generator=g)
-    z8 = torch.randint(0, 4, (out, in_f // 64), dtype=torch.uint8, device="cuda", generator=g)
-    s16 = (torch.rand(out, in_f // 64, device="cuda", generator=g) * 0.01 + 0.001).half()
+    P = torch.randint(0, 256, (out, in_f * bits // 8), dtype=torch.uint8, device="cuda", generator=g)
+    z8 = torch.randint(0, 1 << bits, (out, in_f // group), dtype=torch.uint8, device="cuda", generator=g)
+    s16 = (torch.rand(out, in_f // group, device="cuda", generator=g) * 0.01 + 0.001).half()
     X = torch.randn(T, in_f, device="cuda", generator=g).to(torch.bfloat16)
-    d = eqat.make_desc(2, 64, out, in_f, T)
+    d = eqat.make_desc(bits, group, out, in_f, T)
     ref = torch.empty(T, out, dtype=torch.bfloat16, device="cuda")
     eqat.qlinear_packed_fwd(d, X, P, s16, z8, ref)
     side = torch.cuda.Stream()
@@ -580,51 +581,54 @@ def test_few_token_forward_is_deterministic(eqat):
         torch.cuda.synchronize()
         assert torch.equal(Y.view(torch.int16), ref.view(torch.int16))
     # and it is the right answer
-    q = O.unpack_rows(P.cpu().numpy(), 2, in_f)
-    What_o = O.dequantize(q, s16.cpu().numpy().astype(np.float32), z8.cpu().numpy(), 64)
+    q = O.unpack_rows(P.cpu().numpy(), bits, in_f)
+    What_o = O.dequantize(q, s16.cpu().numpy().astype(np.float32), z8.cpu().numpy(), group)
     assert rel_err(torch_to_f64(ref), O.linear_fwd(torch_to_f64(X), What_o)) <= TOL
 
 
-def few_token_problem(out, in_f, tokens, seed):
+def few_token_problem(out, in_f, tokens, seed, bits=2, group=64):
+    """Random packed bytes (every code value equally likely), zero points near the middle of the code range."""
     g = torch.Generator(device="cuda"); g.manual_seed(seed)
-    P = torch.randint(0, 256, (out, in_f // 4), dtype=torch.uint8, device="cuda", generator=g)
-    z8 = torch.randint(1, 3, (out, in_f // 64), dtype=torch.uint8, device="cuda", generator=g)
-    s16 = (torch.rand(out, in_f // 64, device="cuda", generator=g) * 0.004 + 0.012).half()
+    Q = (1 << bits) - 1
+    P = torch.randint(0, 256, (out, in_f * bits // 8), dtype=torch.uint8, device="cuda", generator=g)
+    z8 = torch.randint(Q // 2, Q // 2 + 2, (out, in_f // group), dtype=torch.uint8, device="cuda", generator=g)
+    s16 = ((torch.rand(out, in_f // group, device="cuda", generator=g) * 0.004 + 0.012) * 3 / Q).half()
     X = torch.randn(tokens, in_f, device="cuda", generator=g).to(torch.bfloat16)
     return P, z8, s16, X
 
 
-def test_few_token_forward_does_not_depend_on_the_slicing(eqat):
+@pytest.mark.parametrize("bits,group", [(2, 64), (4, 128)])
+def test_few_token_forward_does_not_depend_on_the_slicing(eqat, bits, group):
     """Thirteen tokens go out as two launches (seven and six tokens); every token's row must be bit for bit what the
     token gives alone, and what it gives in a batch of eight (one launch)."""
     out, in_f, T = 1280, 4096, 13
-    P, z8, s16, X = few_token_problem(out, in_f, T, 21)
+    P, z8, s16, X = few_token_problem(out, in_f, T, 21, bits, group)
     guard = Guarded()
     Y = guard.empty(T, out, dtype=torch.bfloat16)
-    eqat.qlinear_packed_fwd(eqat.make_desc(2, 64, out, in_f, T), X, P, s16, z8, Y)
+    eqat.qlinear_packed_fwd(eqat.make_desc(bits, group, out, in_f, T), X, P, s16, z8, Y)
     Y8 = guard.empty(8, out, dtype=torch.bfloat16)
-    eqat.qlinear_packed_fwd(eqat.make_desc(2, 64, out, in_f, 8), X[:8].contiguous(), P, s16, z8, Y8)
+    eqat.qlinear_packed_fwd(eqat.make_desc(bits, group, out, in_f, 8), X[:8].contiguous(), P, s16, z8, Y8)
     guard.check()
     assert torch.equal(Y8.view(torch.int16), Y[:8].view(torch.int16))
-    d1 = eqat.make_desc(2, 64, out, in_f, 1)
+    d1 = eqat.make_desc(bits, group, out, in_f, 1)
     for t in range(T):
         y = torch.empty(1, out, dtype=torch.bfloat16, device="cuda")
         eqat.qlinear_packed_fwd(d1, X[t:t + 1].contiguous(), P, s16, z8, y)
         torch.cuda.synchronize()
         assert torch.equal(y.view(torch.int16), Y[t:t + 1].view(torch.int16)), t
-    q = O.unpack_rows(P.cpu().numpy(), 2, in_f)
-    What_o = O.dequantize(q, s16.cpu().numpy().astype(np.float32), z8.cpu().numpy(), 64)
+    q = O.unpack_rows(P.cpu().numpy(), bits, in_f)
+    What_o = O.dequantize(q, s16.cpu().numpy().astype(np.float32), z8.cpu().numpy(), group)
     assert rel_err(torch_to_f64(Y), O.linear_fwd(torch_to_f64(X), What_o)) <= TOL
 
 
-@pytest.mark.parametrize("tokens", [1, 8, 12])
-def test_few_token_forwards_back_to_back_keep_their_order(eqat, tokens):
+@pytest.mark.parametrize("bits,group,tokens", [(2, 64, 1), (2, 64, 8), (2, 64, 12), (4, 128, 3), (4, 128, 12)])
+def test_few_token_forwards_back_to_back_keep_their_order(eqat, bits, group, tokens):
     """Twelve layers in a row, each reading what the one before wrote, issued without a pause (the launches may
     overlap their start-up with the tail of the launch before) and again with a synchronise after every call."""
     n = 4096
-    Ps = [few_token_problem(n, n, tokens, 30 + i)[0] for i in range(12)]
-    _, z8, s16, X0 = few_token_problem(n, n, tokens, 29)
-    d = eqat.make_desc(2, 64, n, n, tokens)
+    Ps = [few_token_problem(n, n, tokens, 30 + i, bits, group)[0] for i in range(12)]
+    _, z8, s16, X0 = few_token_problem(n, n, tokens, 29, bits, group)
+    d = eqat.make_desc(bits, group, n, n, tokens)
 
     def chain(pause):
         bufs = [X0.clone(), torch.zeros_like(X0)]
@@ -648,7 +652,8 @@ def test_few_token_forwards_back_to_back_keep_their_order(eqat, tokens):
     (320, 640, 129, 3, 128),
     (1024, 256, 520, 2, 64),
     (64, 11008, 4, 2, 64),          # few-token kernel with more than 48 KB of staged activations
-    (64, 28672, 2, 4, 128),         # activations too large to stage: two tokens through the tiled kernel
+    (64, 28672, 2, 4, 128),         # the longest rows of the 70B block, 4-bit codes: two tokens fit one launch
+    (64, 28672, 3, 3, 128),         # activations too large to stage on the ordinary cores: the tiled kernel
     (448, 1408, 700, 3, 32),        # groups of 32, nothing a multiple of a tile
     (320, 1408, 1100, 2, 1408),     # one group per row with in_features not a power of two: 5.5 column tiles
     (192, 640, 3, 4, 640),          # one group per row through the few-token kernel
@@ -663,6 +668,10 @@ def test_few_token_forwards_back_to_back_keep_their_order(eqat, tokens):
     (128, 4096, 13, 2, 64),         # more than eight tokens: slices of seven and six
     (128, 8192, 31, 2, 128),        # five slices (7, 7, 7, 7, 3)
     (64, 28672, 4, 2, 64),          # the longest rows of the 70B block: two tokens per launch
+    (64, 11008, 8, 4, 128),         # 4-bit codes: 43 boxes of 256 columns per row, two launches of four tokens
+    (128, 4096, 13, 4, 64),         # 4-bit codes, groups of 64 (one group per chunk), slices of seven and six
+    (80 * 16, 2304, 5, 4, 256),     # 4-bit codes, groups of 256, nine boxes per row, 80 row-blocks
+    (64, 128, 2, 4, 64),            # rows of 64 bytes: half a box, two chunks, two groups
 ])
 def test_e2e_ragged(eqat, out, in_f, tokens, bits, group):
     cfg = small_cfg(f"e2er_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens)
