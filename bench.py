@@ -886,7 +886,7 @@ def run_streaming_case(args):
     print(json.dumps(r), flush=True)
 
 
-def decode_leg(eqat, dev, peaks, iters, model="7b", bits=BITS, group=GROUP):
+def decode_leg(eqat, dev, peaks, iters, model="7b", bits=BITS, group=GROUP, only_shape=None, tokens=(1, 4, 8, 16)):
     """Few-token packed forward (the matrix-vector kernels) on the linear shapes of one block: device time per
     launch from a CUDA graph of launches over rotating weight copies (more than L2 in total), and the bandwidth that
     time means for the bytes one launch must read."""
@@ -896,6 +896,8 @@ def decode_leg(eqat, dev, peaks, iters, model="7b", bits=BITS, group=GROUP):
                      "is one kernel launch for up to 8 tokens where the staged activations fit, else one per token slice",
            "cases": {}}
     for lin in LINEARS[model]:
+        if only_shape is not None and lin.name != only_shape:
+            continue
         o, i = lin.out_features, lin.in_features
         ng = i // group
         wbytes = o * i * bits // 8
@@ -903,7 +905,7 @@ def decode_leg(eqat, dev, peaks, iters, model="7b", bits=BITS, group=GROUP):
         Ps = [torch.randint(0, 256, (o, i * bits // 8), dtype=torch.uint8, device=dev) for _ in range(copies)]
         z8 = torch.randint(0, 1 << bits, (o, ng), dtype=torch.uint8, device=dev)
         s16 = (torch.rand(o, ng, device=dev) * 0.01 + 0.001).half()
-        for T in (1, 4, 8, 16):
+        for T in tokens:
             X = torch.randn(T, i, device=dev).to(torch.bfloat16)
             Y = torch.empty(T, o, dtype=torch.bfloat16, device=dev)
             d = eqat.make_desc(bits, group, o, i, T)
@@ -923,7 +925,7 @@ def run_decode_case(args):
     build_library()
     from paper_2407_11062_b200 import binding as eqat
     out = decode_leg(eqat, torch.device("cuda", 0), load_peaks(), args.case_iters, args.case_model, args.case_bits,
-                     args.case_group)
+                     args.case_group, args.decode_shape, tuple(int(t) for t in args.decode_tokens.split(",")))
     assert eqat.device_status() == (0, 0)
     print(json.dumps(out), flush=True)
 
@@ -933,6 +935,8 @@ def main():
     ap.add_argument("--kernel-case", action="store_true", help="run one linear shape a few times (for profilers)")
     ap.add_argument("--decode-case", action="store_true",
                     help="time the few-token packed forward on the linear shapes of --case-model (uses --case-iters)")
+    ap.add_argument("--decode-shape", default=None, help="decode case: only this linear of the block (e.g. gate_up)")
+    ap.add_argument("--decode-tokens", default="1,4,8,16", help="decode case: token counts, comma separated")
     ap.add_argument("--streaming-case", action="store_true", help="the cold streaming-kernel leg alone")
     ap.add_argument("--case-model", default="7b", choices=sorted(LINEARS))
     ap.add_argument("--case-shape", default="qkvo")

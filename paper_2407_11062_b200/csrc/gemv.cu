@@ -287,7 +287,7 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // avoid here; and with at most a few tokens there is nothing for a 128-row
 // accumulator to amortise.)
 //
-// Fragment construction, 2-bit codes (4-bit codes: expand_words4, one shift and
+// Fragment construction, 2-bit codes (4-bit codes: see expand_reg, one shift and
 // one logic operation per pair of codes, constant 128 throughout).  A 32-bit word
 // of the stream holds 16 consecutive codes of one row, code j at bits [2j, 2j + 2).  (w >> 2p) & 0x00030003 isolates codes
 // p and p + 8 in the two halves of a register; OR-ing 0x4300 into each half makes
@@ -415,26 +415,48 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// The eight registers (codes p and p + 8 as bf16 pairs, p = 0..7) of one 16-code word.
-__device__ __forceinline__ void expand_word2(uint32_t w, uint32_t (&P)[8]) {
-  const uint32_t t1 = w >> 6, t2 = w >> 12;
-  P[0] = and_or(w, 0x00030003u, 0x43004300u);
-  P[1] = and_or(w, 0x000C000Cu, 0x42004200u);
-  P[2] = and_or(w, 0x00300030u, 0x41004100u);
-  P[3] = and_or(t1, 0x00030003u, 0x43004300u);
-  P[4] = and_or(t1, 0x000C000Cu, 0x42004200u);
-  P[5] = and_or(t1, 0x00300030u, 0x41004100u);
-  P[6] = and_or(t2, 0x00030003u, 0x43004300u);
-  P[7] = and_or(t2, 0x000C000Cu, 0x42004200u);
+// The first instruction of a chain: D = A * B (the accumulator input is the constant zero, no register is cleared).
+__device__ __forceinline__ void mma_16816_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%10, %10, %10, %10};"
+               : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
 }
-// 4-bit codes: a word holds eight, code j at bits [4j, 4j + 4).  A lane's two words (16 consecutive columns)
-// give the registers (code p, code p + 4) of each word, all with the constant 128; the codes fill the low four
-// mantissa bits, so there is no room to skip a shift.
-__device__ __forceinline__ void expand_words4(uint32_t w0, uint32_t w1, uint32_t (&P)[8]) {
-#pragma unroll
-  for (int p = 0; p < 4; ++p) {
-    P[p] = and_or(w0 >> (4 * p), 0x000F000Fu, 0x43004300u);
-    P[4 + p] = and_or(w1 >> (4 * p), 0x000F000Fu, 0x43004300u);
+
+// (t & MASK) | magic with the mask as an immediate of the instruction and the magic in a register.  The logic
+// instruction takes one immediate; given two compile-time constants the compiler re-creates one of them with a
+// move in front of every use, which doubled the instruction count of the expansion.  The callers therefore pass
+// magics whose value the compiler cannot see (TcMagics).
+template <uint32_t MASK>
+__device__ __forceinline__ uint32_t and_imm_or(uint32_t t, uint32_t magic) {
+  uint32_t r;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(t), "n"(MASK), "r"(magic));
+  return r;
+}
+// The bf16 pairs (128, 128), (32, 32), (8, 8), built from a value that is zero at run time only.
+struct TcMagics {
+  uint32_t m128, m32, m8;
+  __device__ __forceinline__ explicit TcMagics(uint32_t zero)
+      : m128(0x43004300u | zero), m32(0x42004200u | zero), m8(0x41004100u | zero) {}
+};
+
+// Register r (0..7) of the expansion of a lane's 16 codes of one row.
+// 2-bit codes: one word, register r holds codes r and r + 8 as a bf16 pair.  Registers 0..2 come from the word
+// itself, 3..5 from the word shifted by 6, 6..7 from the word shifted by 12 (the compiler shares the shifts), each
+// with the mask and the constant of the position the code is left at (128, 32 or 8).
+// 4-bit codes: two words of eight codes, code j at bits [4j, 4j + 4); registers 0..3 hold codes (p, p + 4) of the
+// first word, 4..7 of the second, all with the constant 128 (the codes fill the low four mantissa bits, so there
+// is no room to skip a shift).
+template <int BITS>
+__device__ __forceinline__ uint32_t expand_reg(const uint32_t (&w)[BITS / 2], int r, const TcMagics& k) {
+  if constexpr (BITS == 2) {
+    const uint32_t t = r < 3 ? w[0] : (r < 6 ? w[0] >> 6 : w[0] >> 12);
+    const int pos = r % 3;
+    return pos == 0 ? and_imm_or<0x00030003u>(t, k.m128)
+                    : (pos == 1 ? and_imm_or<0x000C000Cu>(t, k.m32) : and_imm_or<0x00300030u>(t, k.m8));
+  } else {
+    return and_imm_or<0x000F000Fu>(w[BITS == 2 ? 0 : (r >> 2)] >> (4 * (r & 3)), k.m128);
   }
 }
 // Which of a lane's 16 columns sits in half `half` (0 = low) of register r (0..7) of the expansion.
@@ -701,7 +723,10 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
     // 2, 3 (-(128 + z) twice), lanes 2 and 3 zeros.  0xBF80 = -1, 0xC300 | z = -(128 + z) for z < 128.
     const uint32_t mask_a = q == 1 ? 0x007F007Fu : 0u, const_a = q == 0 ? 0xBF80BF80u : (q == 1 ? 0xC300C300u : 0u);
     const uint32_t mask_b = q == 0 ? 0x007F0000u : 0u, const_b = q == 0 ? 0xC300BF80u : 0u;
-    const uint2* xb_lane = xb + (size_t)q * T + g;                     // + chunk and item offsets
+    // + chunk and item offsets.  Lanes whose token column does not exist read the last token's entry instead of
+    // a zero: their accumulator columns are never stored.
+    const uint2* xb_lane = xb + (size_t)q * T + (g < T ? g : T - 1);
+    const TcMagics magics((uint32_t)stages >> 30);                     // stages is at most kTcMaxStages
     int slot = 0, buf = 0;
     uint32_t phase = 0, free_phase[2] = {0u, 0u};
     bool alive = true;
@@ -745,28 +770,22 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
 #pragma unroll
           for (int c = 0; c < kChunksPerWarp; ++c) {                   // independent chains, no branches
             const int cg = gbox * kChunksPerBox + chunk0 + c;
-            uint32_t PL[8], PH[8];
-            if constexpr (BITS == 2) {
-              expand_word2(w_lo[c][0], PL);
-              expand_word2(w_hi[c][0], PH);
-            } else {
-              expand_words4(w_lo[c][0], w_lo[c][1], PL);
-              expand_words4(w_hi[c][0], w_hi[c][1], PH);
-            }
             const uint2* item = xb_lane + (size_t)cg * (kTcItems * 4) * T;
-            float D[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            float D[4];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-              uint2 b = make_uint2(0u, 0u);
-              if (g < T) b = item[m * 4 * T];
-              mma_16816(D, PL[2 * m], PH[2 * m], PL[2 * m + 1], PH[2 * m + 1], b.x, b.y);
+            for (int m = 0; m < 4; ++m) {                              // the four registers of A right before their use
+              const uint2 b = item[m * 4 * T];
+              const uint32_t a0 = expand_reg<BITS>(w_lo[c], 2 * m, magics), a1 = expand_reg<BITS>(w_hi[c], 2 * m, magics);
+              const uint32_t a2 = expand_reg<BITS>(w_lo[c], 2 * m + 1, magics);
+              const uint32_t a3 = expand_reg<BITS>(w_hi[c], 2 * m + 1, magics);
+              if (m == 0) mma_16816_first(D, a0, a1, a2, a3, b.x, b.y);
+              else mma_16816(D, a0, a1, a2, a3, b.x, b.y);
             }
             {
               // correction: weights -1 and -(128 + z) against the split sums (see the header)
               const uint32_t zz_lo = ((sp.z_lo >> (8 * (c >> kSlotShift))) & 0xFFu) * 0x10001u;
               const uint32_t zz_hi = ((sp.z_hi >> (8 * (c >> kSlotShift))) & 0xFFu) * 0x10001u;
-              uint2 b = make_uint2(0u, 0u);
-              if (g < T) b = item[4 * 4 * T];
+              const uint2 b = item[4 * 4 * T];
               mma_16816(D, and_or(zz_lo, mask_a, const_a), and_or(zz_hi, mask_a, const_a), and_or(zz_lo, mask_b, const_b),
                         and_or(zz_hi, mask_b, const_b), b.x, b.y);
             }
