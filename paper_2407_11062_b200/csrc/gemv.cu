@@ -484,7 +484,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
   constexpr int kBoxesPerStage = tc_boxes_per_stage(BITS);
   constexpr int kStageBytes = tc_stage_bytes(BITS);
   const TcLayout L = tc_layout(T, in_features, stages, BITS);
-  uint2* xb = reinterpret_cast<uint2*>(ring + L.xb_off);           // [chunk][item][quad lane][token] -> 4 bf16
+  uint2* xb = reinterpret_cast<uint2*>(ring + L.xb_off);           // [chunk][quad lane][token][item] -> 4 bf16
   float* part = reinterpret_cast<float*>(ring + L.part_off);       // [2][warp][row][kTcMaxTokens]
   TcCtl* ctl = reinterpret_cast<TcCtl*>(ring + L.ctl_off);
   volatile int* abort_flag = &ctl->abort;
@@ -689,7 +689,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
           sx = (sx4[0] + sx4[1]) + (sx4[2] + sx4[3]);
 #pragma unroll
           for (int m = 0; m < 4; ++m)
-            xb[(((size_t)cg * kTcItems + m) * 4 + uq) * T + t] =
+            xb[(((size_t)cg * 4 + uq) * T + t) * kTcItems + m] =
                 make_uint2(h[tc_column<BITS>(2 * m, 0)] | (h[tc_column<BITS>(2 * m, 1)] << 16),
                            h[tc_column<BITS>(2 * m + 1, 0)] | (h[tc_column<BITS>(2 * m + 1, 1)] << 16));
         }
@@ -709,11 +709,11 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
               parts[i][pce] = hb;
               v[i] -= __uint_as_float(hb << 16);
             }
-          uint2* item = xb + ((size_t)cg * kTcItems + 4) * 4 * T + t;
-          item[0 * T] = make_uint2(parts[0][0] | (parts[0][1] << 16), parts[0][2] | (parts[1][0] << 16));
-          item[1 * T] = make_uint2(parts[1][1] | (parts[1][2] << 16), 0u);
-          item[2 * T] = make_uint2(0u, 0u);
-          item[3 * T] = make_uint2(0u, 0u);
+          uint2* item = xb + ((size_t)cg * 4 * T + t) * kTcItems + 4;    // + quad lane * T * kTcItems
+          item[0 * T * kTcItems] = make_uint2(parts[0][0] | (parts[0][1] << 16), parts[0][2] | (parts[1][0] << 16));
+          item[1 * T * kTcItems] = make_uint2(parts[1][1] | (parts[1][2] << 16), 0u);
+          item[2 * T * kTcItems] = make_uint2(0u, 0u);
+          item[3 * T * kTcItems] = make_uint2(0u, 0u);
         }
       }
       asm volatile("bar.sync 1, %0;" ::"n"(kTcWarps * 32) : "memory");
@@ -725,7 +725,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
     const uint32_t mask_b = q == 0 ? 0x007F0000u : 0u, const_b = q == 0 ? 0xC300BF80u : 0u;
     // + chunk and item offsets.  Lanes whose token column does not exist read the last token's entry instead of
     // a zero: their accumulator columns are never stored.
-    const uint2* xb_lane = xb + (size_t)q * T + (g < T ? g : T - 1);
+    const uint2* xb_lane = xb + ((size_t)q * T + (g < T ? g : T - 1)) * kTcItems;
     const TcMagics magics((uint32_t)stages >> 30);                     // stages is at most kTcMaxStages
     int slot = 0, buf = 0;
     uint32_t phase = 0, free_phase[2] = {0u, 0u};
@@ -770,11 +770,11 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
 #pragma unroll
           for (int c = 0; c < kChunksPerWarp; ++c) {                   // independent chains, no branches
             const int cg = gbox * kChunksPerBox + chunk0 + c;
-            const uint2* item = xb_lane + (size_t)cg * (kTcItems * 4) * T;
+            const uint2* item = xb_lane + (size_t)cg * (kTcItems * 4) * T;   // the lane's five entries of the chunk
             float D[4];
 #pragma unroll
             for (int m = 0; m < 4; ++m) {                              // the four registers of A right before their use
-              const uint2 b = item[m * 4 * T];
+              const uint2 b = item[m];
               const uint32_t a0 = expand_reg<BITS>(w_lo[c], 2 * m, magics), a1 = expand_reg<BITS>(w_hi[c], 2 * m, magics);
               const uint32_t a2 = expand_reg<BITS>(w_lo[c], 2 * m + 1, magics);
               const uint32_t a3 = expand_reg<BITS>(w_hi[c], 2 * m + 1, magics);
@@ -785,7 +785,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
               // correction: weights -1 and -(128 + z) against the split sums (see the header)
               const uint32_t zz_lo = ((sp.z_lo >> (8 * (c >> kSlotShift))) & 0xFFu) * 0x10001u;
               const uint32_t zz_hi = ((sp.z_hi >> (8 * (c >> kSlotShift))) & 0xFFu) * 0x10001u;
-              const uint2 b = item[4 * 4 * T];
+              const uint2 b = item[4];
               mma_16816(D, and_or(zz_lo, mask_a, const_a), and_or(zz_hi, mask_a, const_a), and_or(zz_lo, mask_b, const_b),
                         and_or(zz_hi, mask_b, const_b), b.x, b.y);
             }
