@@ -56,26 +56,33 @@ __device__ __forceinline__ float group_rcp(float s, float zr) {
 // from the exact one, immaterial for a gradient).
 __device__ __forceinline__ void quotient_round8(const float (&w)[8], float s, float rs, float (&r)[8],
                                                 float (&r_minus_t)[8]) {
-  float dmax = 0.0f;
+  float dq[2] = {0.0f, 0.0f};                       // largest |d| of elements 0..3 and 4..7
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const float r0 = fmaf(w[i], rs, 12582912.0f) - 12582912.0f;
     const float d = fmaf(w[i], rs, -r0);
     r[i] = r0;
     r_minus_t[i] = -d;
-    dmax = fmaxf(dmax, fabsf(d));
+    dq[i >> 2] = fmaxf(dq[i >> 2], fabsf(d));
   }
   // fmaxf drops NaNs, so a NaN reciprocal (group_rcp's way of asking for the exact path) is tested by itself; a NaN
   // weight makes r NaN on either path
-  if (!(dmax < 0.49999237060546875f) || rs != rs) {
-    // Some lane of nearly every warp lands here (bf16 weights over a min/max grid hit exact half-integer quotients
-    // in a few elements per thousand), so the whole warp walks this path: redo only the elements that need it.
+  const bool all_exact = rs != rs;
+  if (!(fmaxf(dq[0], dq[1]) < 0.49999237060546875f) || all_exact) {
+    // Some lane of every second warp lands here (bf16 weights over a min/max grid hit exact half-integer quotients
+    // in a few elements per thousand), and the whole warp walks what that lane walks.  So the walk goes by halves
+    // of the vector: a half with an element to redo is three times rarer than a vector with one.
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (!(fabsf(r_minus_t[i]) < 0.49999237060546875f)) {
-        const float q = __fdiv_rn(w[i], s);
-        r[i] = rintf(q);
-        r_minus_t[i] = r[i] - q;
+    for (int h = 0; h < 2; ++h) {
+      if (!(dq[h] < 0.49999237060546875f) || all_exact) {
+#pragma unroll
+        for (int i = 4 * h; i < 4 * h + 4; ++i) {
+          if (!(fabsf(r_minus_t[i]) < 0.49999237060546875f)) {
+            const float q = __fdiv_rn(w[i], s);
+            r[i] = rintf(q);
+            r_minus_t[i] = r[i] - q;
+          }
+        }
       }
     }
   }

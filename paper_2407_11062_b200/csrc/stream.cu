@@ -398,18 +398,24 @@ quantize_pack_stream_kernel(const __grid_constant__ CUtensorMap map_w, const flo
     for (int u = 0; u < 4; ++u) {
       float w[8], t[8];
       unpack8(raw[0][u], w);
-      uint32_t differ = exact_only ? 1u : 0u;
+      uint32_t differ[2] = {exact_only ? 1u : 0u, exact_only ? 1u : 0u};   // elements 0..3 and 4..7
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         t[i] = fmaf(w[i], rs_lo, cz);
-        differ |= __float_as_uint(t[i]) ^ __float_as_uint(fmaf(w[i], rs_hi, cz));
+        differ[i >> 2] |= __float_as_uint(t[i]) ^ __float_as_uint(fmaf(w[i], rs_hi, cz));
       }
-      if (differ != 0u) {
+      if ((differ[0] | differ[1]) != 0u) {
+        // the whole warp walks what one lane walks, so the walk goes by halves of the vector (see quotient_round8)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          if (exact_only || !(t[i] == fmaf(w[i], rs_hi, cz))) {
-            const float r = rintf(__fdiv_rn(w[i], sv));
-            t[i] = (r + zr) + kTwo23;
+        for (int h = 0; h < 2; ++h) {
+          if (differ[h] != 0u) {
+#pragma unroll
+            for (int i = 4 * h; i < 4 * h + 4; ++i) {
+              if (exact_only || !(t[i] == fmaf(w[i], rs_hi, cz))) {
+                const float r = rintf(__fdiv_rn(w[i], sv));
+                t[i] = (r + zr) + kTwo23;
+              }
+            }
           }
         }
       }
