@@ -626,9 +626,11 @@ def run_block_driver(eqat, device, steps=10):
             "per_linear_calls_tflops": f / (ms_layer * 1e-3) / 1e12}
 
 
-def time_rotation(calls, rounds):
+def time_rotation(calls, rounds, windows=1):
     """Device time per launch (us) of `calls` issued in order, `rounds` times over: one pass is captured in a CUDA
-    graph (so the host's launch cost is not in the figure) and replayed between a pair of events on its stream."""
+    graph (so the host's launch cost is not in the figure) and replayed between a pair of events on its stream.
+    With `windows` > 1 the measurement is repeated back to back and the median window is returned (a short window
+    of a few milliseconds can fall into a transient of the GPU's clocks)."""
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
@@ -641,14 +643,17 @@ def time_rotation(calls, rounds):
                 c()
         graph.replay()
         side.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(side)
-        for _ in range(rounds):
-            graph.replay()
-        e1.record(side)
-        side.synchronize()
+        times = []
+        for _ in range(windows):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side)
+            for _ in range(rounds):
+                graph.replay()
+            e1.record(side)
+            side.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e3 / (rounds * len(calls)))
     torch.cuda.current_stream().wait_stream(side)
-    return e0.elapsed_time(e1) * 1e3 / (rounds * len(calls))
+    return statistics.median(times)
 
 
 def run_streaming_leg(eqat, device, peaks, bits, group, shape=(11008, 4096), min_launches=56, min_bytes=640e6):
@@ -694,7 +699,7 @@ def run_streaming_leg(eqat, device, peaks, bits, group, shape=(11008, 4096), min
                     del S["W"]
             sets.append(S)
         rounds = int(np.ceil(min_launches / n))
-        us = time_rotation([S["call"] for S in sets], rounds)
+        us = time_rotation([S["call"] for S in sets], rounds, windows=3)
         launches = rounds * n
         r = hbm_roofline(nbytes / us / 1e3, peaks)
         r.update({"us_per_launch": us, "launches": launches, "distinct_buffer_sets": n,
@@ -708,7 +713,7 @@ def run_streaming_leg(eqat, device, peaks, bits, group, shape=(11008, 4096), min
     src = [torch.empty(out_f, in_f, dtype=bf, device=device).normal_(generator=g) for _ in range(n)]
     dst = [torch.empty_like(t) for t in src]
     rounds = int(np.ceil(min_launches / n))
-    us = time_rotation([lambda a=a, b=b: b.copy_(a) for a, b in zip(src, dst)], rounds)
+    us = time_rotation([lambda a=a, b=b: b.copy_(a) for a, b in zip(src, dst)], rounds, windows=3)
     yard = hbm_roofline(4 * n_elem / us / 1e3, peaks)
     yard.update({"us_per_launch": us, "launches": rounds * n, "distinct_buffer_sets": n, "bytes_per_launch": 4.0 * n_elem,
                  "what": "torch copy_ of one weight-sized bf16 tensor (not a kernel of this library)"})
@@ -718,7 +723,8 @@ def run_streaming_leg(eqat, device, peaks, bits, group, shape=(11008, 4096), min
     torch.cuda.empty_cache()
     return {"shape": f"{out_f} x {in_f}", "bits": bits, "group": group,
             "method": "distinct input/output sets per launch (combined > 4 x L2); the launches of one pass over the sets are "
-                      "captured in a CUDA graph and the graph is replayed back to back between one pair of CUDA events",
+                      "captured in a CUDA graph and the graph is replayed back to back between one pair of CUDA events; "
+                      "median of three such windows",
             "kernels": res, "copy_yardstick": yard}
 
 
@@ -834,6 +840,7 @@ def run_ours(args):
             out["configs"] = {name: run_extra_config(eqat, device, name, spec, peaks) for name, spec in EXTRA_CONFIGS.items()}
             out["block_ap_forms"] = run_block_ap_forms(eqat, device)
             out["few_tokens"] = decode_leg(eqat, device, peaks, 10)
+            out["few_tokens_w4g128"] = decode_leg(eqat, device, peaks, 10, bits=4, group=128, tokens=(1, 8))
             out["block_driver"] = run_block_driver(eqat, device)
             out["streaming"] = {"w2g64": run_streaming_leg(eqat, device, peaks, 2, 64),
                                 "w4g128": run_streaming_leg(eqat, device, peaks, 4, 128)}
