@@ -325,12 +325,15 @@ constexpr int kTcMaxTotalTokens = 32;                   // more go out as severa
 constexpr int kTcWarps = 16;
 constexpr int kTcThreads = (kTcWarps + 2) * 32;        // + producer warp + reducer warp
 constexpr int kTcRows = 16;                            // weight rows per task
-constexpr int kTcBoxBytes = 128;
+// Bytes of a row per box of the copy engine: 128 (512 columns of 2-bit codes, 256 of 4-bit codes) or, for 3-bit
+// codes, whose 64-column chunks are 24 bytes, 96 (256 columns).
+__host__ __device__ constexpr int tc_box_bytes(int bits) { return bits == 3 ? 96 : 128; }
+__host__ __device__ constexpr int tc_words_per_lane(int bits) { return bits == 2 ? 1 : 2; }   // per row and chunk
 // Boxes per stage: every consumer warp has four chunks of a stage, i.e. half a box of 2-bit codes (8 boxes,
 // 16 KB per stage) or a whole box of 4-bit codes (16 boxes, 32 KB per stage).
-__host__ __device__ constexpr int tc_boxes_per_stage(int bits) { return 4 * bits; }
-constexpr int kTcBoxSmem = kTcRows * kTcBoxBytes;      // 2 KB
-__host__ __device__ constexpr int tc_stage_bytes(int bits) { return tc_boxes_per_stage(bits) * kTcBoxSmem; }
+__host__ __device__ constexpr int tc_boxes_per_stage(int bits) { return bits == 2 ? 8 : 16; }
+__host__ __device__ constexpr int tc_box_smem(int bits) { return kTcRows * tc_box_bytes(bits); }   // 2 KB or 1.5 KB
+__host__ __device__ constexpr int tc_stage_bytes(int bits) { return tc_boxes_per_stage(bits) * tc_box_smem(bits); }
 constexpr int kTcAhead = 3;                            // stages of lead of the parameter loads
 constexpr int kTcItems = 5;                            // instructions per chunk: four on codes, one correction
 constexpr int kTcMaxStages = 8;
@@ -356,7 +359,7 @@ __host__ __device__ inline TcLayout tc_layout(int T, int in_features, int stages
   TcLayout L;
   // chunks of 64 columns, counted up to the end of the last (possibly partial) 128-byte box (512 columns of 2-bit
   // codes, 256 of 4-bit codes): the entries past in_features are zeros, so the compute loop needs no end-of-row case
-  const int box_cols = kTcBoxBytes * 8 / bits;
+  const int box_cols = tc_box_bytes(bits) * 8 / bits;
   const size_t chunks = (size_t)((in_features + box_cols - 1) / box_cols) * (box_cols / 64);
   L.stages = stages;
   L.xb_off = (size_t)stages * tc_stage_bytes(bits);
@@ -436,9 +439,9 @@ __device__ __forceinline__ uint32_t and_imm_or(uint32_t t, uint32_t magic) {
 }
 // The bf16 pairs (128, 128), (32, 32), (8, 8), built from a value that is zero at run time only.
 struct TcMagics {
-  uint32_t m128, m32, m8;
+  uint32_t m128, m32, m8, m32_128;                      // the last: 32 in the high half, 128 in the low half
   __device__ __forceinline__ explicit TcMagics(uint32_t zero)
-      : m128(0x43004300u | zero), m32(0x42004200u | zero), m8(0x41004100u | zero) {}
+      : m128(0x43004300u | zero), m32(0x42004200u | zero), m8(0x41004100u | zero), m32_128(0x42004300u | zero) {}
 };
 
 // Register r (0..7) of the expansion of a lane's 16 codes of one row.
@@ -448,25 +451,35 @@ struct TcMagics {
 // 4-bit codes: two words of eight codes, code j at bits [4j, 4j + 4); registers 0..3 hold codes (p, p + 4) of the
 // first word, 4..7 of the second, all with the constant 128 (the codes fill the low four mantissa bits, so there
 // is no room to skip a shift).
+// 3-bit codes: w[0] and w[1] hold the lane's 48 bits (code j at bits [3j, 3j + 3); bits 48 and up of w[1] belong to
+// the next lane).  Register r < 6 comes from the 32 bits starting at bit 3r: code r at the bottom of the low half
+// (constant 128) and code r + 6 at bits 2-4 of the high half (constant 32, whose last place is a quarter).
+// Registers 6 and 7 hold codes (12, 14) and (13, 15), moved to the bottom of their halves one at a time.
 template <int BITS>
-__device__ __forceinline__ uint32_t expand_reg(const uint32_t (&w)[BITS / 2], int r, const TcMagics& k) {
-  if constexpr (BITS == 2) {
+__device__ __forceinline__ uint32_t expand_reg(const uint32_t (&w)[tc_words_per_lane(BITS)], int r, const TcMagics& k) {
+  if constexpr (BITS == 3) {
+    if (r < 6) return and_imm_or<0x001C0007u>(r == 0 ? w[0] : __funnelshift_r(w[0], w[1], 3 * r), k.m32_128);
+    const uint32_t low = and_imm_or<0x00000007u>(w[1] >> (r == 6 ? 4 : 7), k.m128);
+    return and_imm_or<0x00070000u>(w[1] << (r == 6 ? 6 : 3), low);
+  } else if constexpr (BITS == 2) {
     const uint32_t t = r < 3 ? w[0] : (r < 6 ? w[0] >> 6 : w[0] >> 12);
     const int pos = r % 3;
     return pos == 0 ? and_imm_or<0x00030003u>(t, k.m128)
                     : (pos == 1 ? and_imm_or<0x000C000Cu>(t, k.m32) : and_imm_or<0x00300030u>(t, k.m8));
   } else {
-    return and_imm_or<0x000F000Fu>(w[BITS == 2 ? 0 : (r >> 2)] >> (4 * (r & 3)), k.m128);
+    return and_imm_or<0x000F000Fu>(w[BITS == 4 ? (r >> 2) : 0] >> (4 * (r & 3)), k.m128);
   }
 }
 // Which of a lane's 16 columns sits in half `half` (0 = low) of register r (0..7) of the expansion.
 template <int BITS>
 __host__ __device__ constexpr int tc_column(int r, int half) {
+  if (BITS == 3) return r < 6 ? r + 6 * half : r + 6 + 2 * half;
   return BITS == 2 ? r + 8 * half : (r < 4 ? r + 4 * half : r + 4 + 4 * half);
 }
 // Constant that the expansion adds to column j (0..15) of a lane.
 template <int BITS>
 __host__ __device__ constexpr float tc_bias(int j) {
+  if (BITS == 3) return (j >= 6 && j < 12) ? 32.0f : 128.0f;
   return BITS == 4 ? 128.0f : ((j & 7) % 3 == 0 ? 128.0f : ((j & 7) % 3 == 1 ? 32.0f : 8.0f));
 }
 
@@ -479,6 +492,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
   const uint32_t raw_addr = ptx::smem_addr(smem_raw);
   const uint32_t ring_addr = (raw_addr + 1023u) & ~1023u;          // boxes are 1024-byte aligned (swizzle period)
   uint8_t* ring = smem_raw + (ring_addr - raw_addr);
+  constexpr int kTcBoxBytes = tc_box_bytes(BITS), kTcBoxSmem = tc_box_smem(BITS);
   constexpr int kChunksPerBox = kTcBoxBytes * 8 / BITS / 64;        // 64-column chunks of a row per box: 8 or 4
   constexpr int kChunksPerWarp = 4;                                 // half a box (2-bit codes) or a box (4-bit codes)
   constexpr int kBoxesPerStage = tc_boxes_per_stage(BITS);
@@ -742,13 +756,26 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
         advance();
         const bool got = tc_wait(ptx::smem_addr(&ctl->full[slot]), phase, abort_flag, WAIT_STREAM_FULL, 0);
         if (!__all_sync(0xFFFFFFFFu, got)) { alive = false; break; }
-        uint32_t w_lo[kChunksPerWarp][BITS / 2], w_hi[kChunksPerWarp][BITS / 2];   // a lane's 16 codes per row and chunk
+        // a lane's 16 codes per row and chunk
+        uint32_t w_lo[kChunksPerWarp][tc_words_per_lane(BITS)], w_hi[kChunksPerWarp][tc_words_per_lane(BITS)];
         if (have) {
           // 16-byte piece c of row r sits at piece (c ^ (r & 7)); rows g and g + 8 share the pattern
           const uint32_t row = ring_addr + slot * kStageBytes + box * kTcBoxSmem + g * kTcBoxBytes;
 #pragma unroll
           for (int c = 0; c < kChunksPerWarp; ++c) {
-            if constexpr (BITS == 2) {                                 // word q of the chunk's one piece
+            if constexpr (BITS == 3) {
+              // no swizzle; the lane's 6 bytes start at byte 6q of the chunk's 24: the two words around them,
+              // shifted down by 0 or 16 bits
+              const uint32_t a = row + (uint32_t)(chunk0 + c) * 24u + (uint32_t)((6 * q) >> 2) * 4u;
+              uint32_t lo0, lo1, hi0, hi1;
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(lo0) : "r"(a) : "memory");
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(lo1) : "r"(a + 4) : "memory");
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(hi0) : "r"(a + 8 * kTcBoxBytes) : "memory");
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(hi1) : "r"(a + 8 * kTcBoxBytes + 4) : "memory");
+              const uint32_t sh = (q & 1) * 16u;
+              w_lo[c][0] = __funnelshift_r(lo0, lo1, sh); w_lo[c][1] = lo1 >> sh;
+              w_hi[c][0] = __funnelshift_r(hi0, hi1, sh); w_hi[c][1] = hi1 >> sh;
+            } else if constexpr (BITS == 2) {                          // word q of the chunk's one piece
               const uint32_t a = row + ((uint32_t)((chunk0 + c) ^ g) << 4) + q * 4;
               asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w_lo[c][0]) : "r"(a) : "memory");
               asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w_hi[c][0]) : "r"(a + 8 * kTcBoxBytes) : "memory");
@@ -834,13 +861,40 @@ __global__ void tc_wait_expiry_kernel(uint64_t limit_ns) {
   (void)tc_wait(ptx::smem_addr(&bar), 0u, &abort_word, WAIT_SELFTEST, 0, limit_ns);
 }
 
+// Tensor map of a byte matrix [outer, inner_bytes] row-major for copies of box_bytes x box_outer rows laid out in
+// shared memory as they are (no swizzle): the 96-byte boxes of 3-bit codes.
+bool make_tmap_u8_plain(CUtensorMap* tm, const void* base, uint64_t inner_bytes, uint64_t outer, uint32_t box_bytes,
+                        uint32_t box_outer) {
+  using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static const EncodeFn enc = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeFn>(p);
+  }();
+  if (enc == nullptr) return false;
+  const cuuint64_t dims[2] = {inner_bytes, outer};
+  const cuuint64_t strides[1] = {inner_bytes};
+  const cuuint32_t box[2] = {box_bytes, box_outer};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BITS, int PARAM_MODE>
 int launch_tc_mode(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
                    eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
   static SmemOptIn opt_in;
   if (!opt_in.ensure(packed_gemv_tc_kernel<BITS, PARAM_MODE>, (int)kTcSmemBudget)) return EQAT_ERR_CUDA;
   CUtensorMap mw;
-  if (!make_tmap_u8(&mw, Wq, (uint64_t)d.in_features * BITS / 8, (uint64_t)d.out_features, kTcBoxBytes, kTcRows))
+  const uint64_t row_bytes = (uint64_t)d.in_features * BITS / 8;
+  if (!(BITS == 3 ? make_tmap_u8_plain(&mw, Wq, row_bytes, (uint64_t)d.out_features, tc_box_bytes(BITS), kTcRows)
+                  : make_tmap_u8(&mw, Wq, row_bytes, (uint64_t)d.out_features, tc_box_bytes(BITS), kTcRows)))
     return EQAT_ERR_CUDA;
   const int sms = sm_count();
   if (sms <= 0) return EQAT_ERR_CUDA;
@@ -897,7 +951,8 @@ struct TcPlan {
 
 static TcPlan tc_plan(const eqat_desc& d) {
   const TcPlan none{0, 0};
-  if ((d.bits != 2 && d.bits != 4) || d.group < 64 || d.tokens < 1 || d.tokens > kTcMaxTotalTokens) return none;
+  if (d.bits < 2 || d.bits > 4 || d.group < 64 || d.tokens < 1 || d.tokens > kTcMaxTotalTokens) return none;
+  if (((int64_t)d.in_features * d.bits / 8) % 16 != 0) return none;    // the copy engine wants rows of 16-byte multiples
   if (d.zero_point_format != EQAT_ZP_U8) return none;
   const int T = (int)d.tokens;
   int fit = T < kTcMaxTokens ? T : kTcMaxTokens;
@@ -906,7 +961,8 @@ static TcPlan tc_plan(const eqat_desc& d) {
   const int launches = (T + fit - 1) / fit, slice = (T + launches - 1) / launches;
   if (launches > 1) {
     const double weight_mb = (double)d.out_features * d.in_features * d.bits / 8.0 / 1.0e6;
-    const double stream_tbs = d.bits == 2 ? 1.6 : 2.5, tiled_us = d.in_features / 64.0 * (d.bits == 2 ? 1.0 : 1.2);
+    const double stream_tbs = d.bits == 2 ? 1.6 : (d.bits == 3 ? 1.8 : 2.5);
+    const double tiled_us = d.in_features / 64.0 * (d.bits == 2 ? 1.0 : 1.2);
     const double few_us = launches * (4.0 + 0.5 * slice + weight_mb / stream_tbs);
     if (few_us >= 0.8 * tiled_us) return none;
   }
@@ -935,8 +991,9 @@ int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq
       const int stages = tc_stages_that_fit((int)part.tokens, d.in_features, d.bits);
       const eqat_bf16* Xs = X + (size_t)t0 * d.in_features;
       eqat_bf16* Ys = Y + (size_t)t0 * d.out_features;
-      const int rc = d.bits == 2 ? launch_tc<2>(part, Xs, Wq, s16, zq, Ys, group_shift, stages, st)
-                                 : launch_tc<4>(part, Xs, Wq, s16, zq, Ys, group_shift, stages, st);
+      const int rc = d.bits == 2   ? launch_tc<2>(part, Xs, Wq, s16, zq, Ys, group_shift, stages, st)
+                     : d.bits == 3 ? launch_tc<3>(part, Xs, Wq, s16, zq, Ys, group_shift, stages, st)
+                                   : launch_tc<4>(part, Xs, Wq, s16, zq, Ys, group_shift, stages, st);
       if (rc != EQAT_OK) return rc;
     }
     return EQAT_OK;

@@ -533,8 +533,8 @@ def test_e2e_small(eqat, bits, group, real_z):
 @pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("tokens", [1, 2, 3, 4, 5, 7, 8, 9])
 def test_e2e_few_tokens(eqat, bits, tokens):
-    """Decode-sized batches: up to four tokens (eight for 2-bit and 4-bit codes) take a matrix-vector forward kernel,
-    more the tiled one (rows this short are not worth several launches).
+    """Decode-sized batches: up to eight tokens take a matrix-vector forward kernel, more the tiled one (rows this
+    short are not worth several launches).
     640 = 10 units of 64 columns, fewer than the sixteen warps of a CTA (some get none); 1408 = 22 (one or two each)."""
     group = 64 if bits == 2 else 128
     cfg = small_cfg(f"gemv_{bits}_{tokens}", 448, 640 if group == 64 else 1408, bits, group, tokens, "student_t4", 0.02, 0.01)
@@ -558,7 +558,7 @@ def test_few_token_forward_agrees_with_tiled_forward(eqat):
     assert rel_err(torch_to_f64(Y4), torch_to_f64(r5["Y"][:4])) <= TOL
 
 
-@pytest.mark.parametrize("bits,group", [(2, 64), (4, 128), (4, 64)])
+@pytest.mark.parametrize("bits,group", [(2, 64), (3, 128), (3, 64), (4, 128), (4, 64)])
 def test_few_token_forward_is_deterministic(eqat, bits, group):
     """More row-blocks than SMs, several stages per row-block: the partial sums of the sixteen warps are added in
     a fixed order by one warp, so repeated launches must agree bit for bit (also while other work runs beside them)."""
@@ -597,7 +597,7 @@ def few_token_problem(out, in_f, tokens, seed, bits=2, group=64):
     return P, z8, s16, X
 
 
-@pytest.mark.parametrize("bits,group", [(2, 64), (4, 128)])
+@pytest.mark.parametrize("bits,group", [(2, 64), (3, 128), (4, 128)])
 def test_few_token_forward_does_not_depend_on_the_slicing(eqat, bits, group):
     """Thirteen tokens go out as two launches (seven and six tokens); every token's row must be bit for bit what the
     token gives alone, and what it gives in a batch of eight (one launch)."""
@@ -621,7 +621,7 @@ def test_few_token_forward_does_not_depend_on_the_slicing(eqat, bits, group):
     assert rel_err(torch_to_f64(Y), O.linear_fwd(torch_to_f64(X), What_o)) <= TOL
 
 
-@pytest.mark.parametrize("bits,group,tokens", [(2, 64, 1), (2, 64, 8), (2, 64, 12), (4, 128, 3), (4, 128, 12)])
+@pytest.mark.parametrize("bits,group,tokens", [(2, 64, 1), (2, 64, 8), (2, 64, 12), (3, 128, 5), (4, 128, 3), (4, 128, 12)])
 def test_few_token_forwards_back_to_back_keep_their_order(eqat, bits, group, tokens):
     """Twelve layers in a row, each reading what the one before wrote, issued without a pause (the launches may
     overlap their start-up with the tail of the launch before) and again with a synchronise after every call."""
@@ -653,7 +653,7 @@ def test_few_token_forwards_back_to_back_keep_their_order(eqat, bits, group, tok
     (1024, 256, 520, 2, 64),
     (64, 11008, 4, 2, 64),          # few-token kernel with more than 48 KB of staged activations
     (64, 28672, 2, 4, 128),         # the longest rows of the 70B block, 4-bit codes: two tokens fit one launch
-    (64, 28672, 3, 3, 128),         # activations too large to stage on the ordinary cores: the tiled kernel
+    (64, 28672, 3, 3, 128),         # 3-bit codes, the longest rows: slices of two tokens and one
     (448, 1408, 700, 3, 32),        # groups of 32, nothing a multiple of a tile
     (320, 1408, 1100, 2, 1408),     # one group per row with in_features not a power of two: 5.5 column tiles
     (192, 640, 3, 4, 640),          # one group per row through the few-token kernel
@@ -672,6 +672,10 @@ def test_few_token_forwards_back_to_back_keep_their_order(eqat, bits, group, tok
     (128, 4096, 13, 4, 64),         # 4-bit codes, groups of 64 (one group per chunk), slices of seven and six
     (80 * 16, 2304, 5, 4, 256),     # 4-bit codes, groups of 256, nine boxes per row, 80 row-blocks
     (64, 128, 2, 4, 64),            # rows of 64 bytes: half a box, two chunks, two groups
+    (128, 4096, 13, 3, 128),        # 3-bit codes: boxes of 96 bytes (256 columns), slices of seven and six
+    (80 * 16, 2304, 5, 3, 256),     # 3-bit codes, groups of 256, nine boxes per row, 80 row-blocks
+    (64, 11008, 8, 3, 64),          # 3-bit codes, groups of 64, 43 boxes per row, two launches of four tokens
+    (64, 128, 1, 3, 128),           # 3-bit rows of 48 bytes: half a box, one group
 ])
 def test_e2e_ragged(eqat, out, in_f, tokens, bits, group):
     cfg = small_cfg(f"e2er_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens)
