@@ -5,9 +5,9 @@
 // one pass over the packed weight, so the kernels are streams over its bytes.
 // Two kernels: the first (below) runs on the ordinary cores and takes every bit
 // width and zero-point format for up to four tokens; the second (further down)
-// builds weight fragments for warp-level matrix instructions and takes 2-bit
-// codes with byte zero points for up to eight tokens per launch (more tokens,
-// or rows too long for the staged activations, go out as several launches).
+// builds weight fragments for warp-level matrix instructions and takes codes
+// with byte zero points for up to eight tokens per launch (more tokens, or rows
+// too long for the staged activations, go out as several launches).
 //
 // First kernel.  Mapping: a CTA owns 32 consecutive weight rows, lane = row, and
 // its 16 warps split the row into contiguous runs of 64-code units.  All lanes
@@ -276,10 +276,10 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 }
 
 
-// ====================================================================== 2-bit and 4-bit codes on tensor-core tiles
+// ====================================================================== codes on tensor-core tiles
 // The kernel above spends three instructions per code and token on the ordinary
-// cores.  That is several times what the bytes allow, so 2-bit and 4-bit codes go
-// through warp-level matrix instructions instead (mma.sync m16n8k16, bf16 in,
+// cores.  That is several times what the bytes allow, so codes with byte zero
+// points go through warp-level matrix instructions instead (mma.sync m16n8k16, bf16 in,
 // fp32 out): 16 weight rows by 16 columns against up to 8 tokens per
 // instruction, with the weight fragment built in registers, one logic
 // operation per PAIR of codes.  (The paired-CTA tensor-memory path of gemm.cu
@@ -287,8 +287,7 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // avoid here; and with at most a few tokens there is nothing for a 128-row
 // accumulator to amortise.)
 //
-// Fragment construction, 2-bit codes (4-bit codes: see expand_reg, one shift and
-// one logic operation per pair of codes, constant 128 throughout).  A 32-bit word
+// Fragment construction, 2-bit codes (3-bit and 4-bit codes: see expand_reg).  A 32-bit word
 // of the stream holds 16 consecutive codes of one row, code j at bits [2j, 2j + 2).  (w >> 2p) & 0x00030003 isolates codes
 // p and p + 8 in the two halves of a register; OR-ing 0x4300 into each half makes
 // them the bf16 numbers 128 + q.  For p = 1, 2 (mod 3) the shift is skipped: a
@@ -307,9 +306,11 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // CTAs take tasks round-robin.  The producer thread copies the task's codes into
 // a shared-memory ring as [16 rows x 128 bytes] boxes (cp.async.bulk.tensor,
 // 128-byte swizzle, bytes past the end of a row arrive as zeros), eight boxes
-// per stage (sixteen for 4-bit codes).  Consumer warp w owns half of box w/2 of every stage: four chunks of
-// 16 bytes = 64 columns = the four words of the four lanes of a quad (4-bit
-// codes: two chunks of 32 bytes, two words per lane), so a
+// per stage.  Consumer warp w owns half of box w/2 of every stage: four chunks
+// of 16 bytes = 64 columns = the four words of the four lanes of a quad.  (4-bit
+// codes: sixteen boxes per stage, a warp owns a box = four chunks of 32 bytes,
+// two words per lane.  3-bit codes: sixteen unswizzled boxes of 96 bytes, a
+// warp owns a box = four chunks of 24 bytes, six bytes per lane.)  A
 // chunk lies in one quantisation group and its accumulator is scaled by one step
 // size per row.  Lane (g, q) of the warp holds rows g and g + 8 and, in
 // instruction m of a chunk, supplies codes 2m, 2m+8, 2m+1, 2m+9 of its word
@@ -938,12 +939,12 @@ int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const e
 
 }  // namespace
 
-// 2-bit and 4-bit codes with byte zero points go through the tensor-core kernel: in one launch when the
-// shared-memory plan fits all tokens, otherwise (long rows, or more than eight tokens) as several launches over
-// slices of the tokens, each of which streams the packed weight once more.  That is taken only while it is clearly
-// cheaper than the tiled kernel of gemm.cu.  Cost model (from timings on the Llama-2 7B and 70B shapes): a launch
-// of this kernel takes about 4 us + 0.5 us per token + the packed weight at 1.6 TB/s (2-bit codes) or 2.5 TB/s
-// (4-bit codes); the tiled kernel takes about 1 us (1.2 us) per 64 input columns for any token count below a full
+// Codes with byte zero points go through the tensor-core kernel: in one launch when the shared-memory plan fits all
+// tokens, otherwise (long rows, or more than eight tokens) as several launches over slices of the tokens, each of
+// which streams the packed weight once more.  That is taken only while it is clearly cheaper than the tiled kernel
+// of gemm.cu.  Cost model (from timings on the Llama-2 7B, 13B and 70B shapes): a launch of this kernel takes about
+// 4 us + 0.5 us per token + the packed weight at 2.25 / 2.6 / 3.5 TB/s (2 / 3 / 4-bit codes; 4 % more per further
+// token); the tiled kernel takes about 1 / 1.45 / 1.2 us per 64 input columns for any token count below a full
 // row-tile, because the K loop of a tile is serial.
 struct TcPlan {
   int launches, slice;                                   // slice = tokens per launch (the last one may have fewer)
@@ -961,9 +962,9 @@ static TcPlan tc_plan(const eqat_desc& d) {
   const int launches = (T + fit - 1) / fit, slice = (T + launches - 1) / launches;
   if (launches > 1) {
     const double weight_mb = (double)d.out_features * d.in_features * d.bits / 8.0 / 1.0e6;
-    const double stream_tbs = d.bits == 2 ? 1.6 : (d.bits == 3 ? 1.8 : 2.5);
-    const double tiled_us = d.in_features / 64.0 * (d.bits == 2 ? 1.0 : 1.2);
-    const double few_us = launches * (4.0 + 0.5 * slice + weight_mb / stream_tbs);
+    const double stream_tbs = d.bits == 2 ? 2.25 : (d.bits == 3 ? 2.6 : 3.5);
+    const double tiled_us = d.in_features / 64.0 * (d.bits == 2 ? 1.0 : (d.bits == 3 ? 1.45 : 1.2));
+    const double few_us = launches * (4.0 + 0.5 * slice + weight_mb / stream_tbs * (1.0 + 0.04 * (slice - 1)));
     if (few_us >= 0.8 * tiled_us) return none;
   }
   return TcPlan{launches, slice};
