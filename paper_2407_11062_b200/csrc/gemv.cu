@@ -279,22 +279,23 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // ====================================================================== codes on tensor-core tiles
 // The kernel above spends three instructions per code and token on the ordinary
 // cores.  That is several times what the bytes allow, so codes with byte zero
-// points go through warp-level matrix instructions instead (mma.sync m16n8k16, bf16 in,
-// fp32 out): 16 weight rows by 16 columns against up to 8 tokens per
+// points go through warp-level matrix instructions instead (mma.sync m16n8k16,
+// bf16 in, fp32 out): 16 weight rows by 16 columns against up to 8 tokens per
 // instruction, with the weight fragment built in registers, one logic
 // operation per PAIR of codes.  (The paired-CTA tensor-memory path of gemm.cu
 // wants its operands expanded into shared memory, which is exactly the cost to
 // avoid here; and with at most a few tokens there is nothing for a 128-row
 // accumulator to amortise.)
 //
-// Fragment construction, 2-bit codes (3-bit and 4-bit codes: see expand_reg).  A 32-bit word
-// of the stream holds 16 consecutive codes of one row, code j at bits [2j, 2j + 2).  (w >> 2p) & 0x00030003 isolates codes
-// p and p + 8 in the two halves of a register; OR-ing 0x4300 into each half makes
-// them the bf16 numbers 128 + q.  For p = 1, 2 (mod 3) the shift is skipped: a
-// code left at bits 2-3 (4-5) of a half with 0x4200 (0x4100) above it is the
-// bf16 number 32 + q (8 + q).  Eight registers from ten operations.  The added
-// constants and the zero point are taken out again by a fifth instruction per
-// chunk: with xb = sum of bias * x and xs = sum of x over the chunk's 64 columns,
+// Fragment construction, 2-bit codes (3-bit and 4-bit codes: see expand_reg).
+// A 32-bit word of the stream holds 16 consecutive codes of one row, code j at
+// bits [2j, 2j + 2).  (w >> 2p) & 0x00030003 isolates codes p and p + 8 in the
+// two halves of a register; OR-ing 0x4300 into each half makes them the bf16
+// numbers 128 + q.  For p = 1, 2 (mod 3) the shift is skipped: a code left at
+// bits 2-3 (4-5) of a half with 0x4200 (0x4100) above it is the bf16 number
+// 32 + q (8 + q).  Eight registers from ten operations.  The added constants
+// and the zero point are taken out again by a fifth instruction per chunk: with
+// xb = sum of bias * x and xs = sum of x over the chunk's 64 columns,
 //     sum (q - z) x = sum (bias + q) x - (xb - 128 xs) - (128 + z) xs,
 // and the fifth instruction multiplies weights -1 and -(128 + z) (the bf16
 // pattern 0xC300 | z) with xb - 128 xs and xs, each given as the sum of three
@@ -310,17 +311,16 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // of 16 bytes = 64 columns = the four words of the four lanes of a quad.  (4-bit
 // codes: sixteen boxes per stage, a warp owns a box = four chunks of 32 bytes,
 // two words per lane.  3-bit codes: sixteen unswizzled boxes of 96 bytes, a
-// warp owns a box = four chunks of 24 bytes, six bytes per lane.)  A
-// chunk lies in one quantisation group and its accumulator is scaled by one step
-// size per row.  Lane (g, q) of the warp holds rows g and g + 8 and, in
-// instruction m of a chunk, supplies codes 2m, 2m+8, 2m+1, 2m+9 of its word
-// (tc_column gives the order for either width);
-// the activations are staged once per CTA in exactly that order, so a lane
-// fetches its fragment of X with one 8-byte load.  Zero points are one byte
-// each here (the fp16 variant goes through the kernel above).  The 16 warps'
-// partial sums of a task go through a double-buffered shared array to a reducer
-// warp, which adds them in a fixed order and stores Y while the consumers are
-// on the next task.
+// warp owns a box = four chunks of 24 bytes, six bytes per lane.)  A chunk lies
+// in one quantisation group and its accumulator is scaled by one step size per
+// row.  Lane (g, q) of the warp holds rows g and g + 8 and, in instruction m of
+// a chunk, supplies four of its 16 codes (2m, 2m+8, 2m+1, 2m+9 for 2-bit codes;
+// tc_column gives the order for every width); the activations are staged once
+// per CTA in exactly that order, so a lane fetches its fragment of X for an
+// instruction with one 8-byte load.  Zero points are one byte each here (the
+// fp16 variant goes through the kernel above).  The 16 warps' partial sums of a
+// task go through a double-buffered shared array to a reducer warp, which adds
+// them in a fixed order and stores Y while the consumers are on the next task.
 constexpr int kTcMaxTokens = 8;                         // the instruction has eight token columns
 constexpr int kTcMaxTotalTokens = 32;                   // more go out as several launches over slices of the tokens
 constexpr int kTcWarps = 16;
@@ -331,14 +331,14 @@ constexpr int kTcRows = 16;                            // weight rows per task
 __host__ __device__ constexpr int tc_box_bytes(int bits) { return bits == 3 ? 96 : 128; }
 __host__ __device__ constexpr int tc_words_per_lane(int bits) { return bits == 2 ? 1 : 2; }   // per row and chunk
 // Boxes per stage: every consumer warp has four chunks of a stage, i.e. half a box of 2-bit codes (8 boxes,
-// 16 KB per stage) or a whole box of 4-bit codes (16 boxes, 32 KB per stage).
+// 16 KB per stage) or a whole box of 3-bit or 4-bit codes (16 boxes, 24 KB or 32 KB per stage).
 __host__ __device__ constexpr int tc_boxes_per_stage(int bits) { return bits == 2 ? 8 : 16; }
 __host__ __device__ constexpr int tc_box_smem(int bits) { return kTcRows * tc_box_bytes(bits); }   // 2 KB or 1.5 KB
 __host__ __device__ constexpr int tc_stage_bytes(int bits) { return tc_boxes_per_stage(bits) * tc_box_smem(bits); }
 constexpr int kTcAhead = 3;                            // stages of lead of the parameter loads
 constexpr int kTcItems = 5;                            // instructions per chunk: four on codes, one correction
 constexpr int kTcMaxStages = 8;
-__host__ __device__ constexpr int tc_min_stages(int bits) { return bits == 2 ? 3 : 2; }   // 48 KB / 64 KB in flight
+__host__ __device__ constexpr int tc_min_stages(int bits) { return bits == 2 ? 3 : 2; }   // at least 48 KB in flight
 constexpr uint64_t kTcWaitLimitNs = 2000000000ull;
 constexpr size_t kTcSmemBudget = 227 * 1024;             // the most a CTA can be given (eight tokens of 8192 columns need 225.2 KB)
 
