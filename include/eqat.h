@@ -231,7 +231,7 @@ int eqat_unpack_zeros(const eqat_desc* desc, const uint8_t* z_packed, uint8_t* z
  * packed weight instead and does not round (W_int - z) * s to bf16.  With byte
  * zero points (and, for 3-bit codes, packed rows that are multiples of 16
  * bytes) that kernel runs on matrix instructions and takes up to eight tokens
- * per launch, and up to 32 tokens go through it in slices (one pass over the
+ * per launch, and up to 64 tokens go through it in slices (one pass over the
  * packed weight per slice) while that is cheaper than the tiled kernel; a
  * token's result does not depend on how the tokens were sliced.
  *   X [T,in] bf16, Wq_packed, s16, z (in)   Y [T,out] bf16 (out) */

@@ -322,7 +322,7 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // task go through a double-buffered shared array to a reducer warp, which adds
 // them in a fixed order and stores Y while the consumers are on the next task.
 constexpr int kTcMaxTokens = 8;                         // the instruction has eight token columns
-constexpr int kTcMaxTotalTokens = 32;                   // more go out as several launches over slices of the tokens
+constexpr int kTcMaxTotalTokens = 64;                   // up to here, as several launches over slices of the tokens
 constexpr int kTcWarps = 16;
 constexpr int kTcThreads = (kTcWarps + 2) * 32;        // + producer warp + reducer warp
 constexpr int kTcRows = 16;                            // weight rows per task

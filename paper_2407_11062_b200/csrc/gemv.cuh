@@ -8,7 +8,7 @@ namespace eqat {
 constexpr int kGemvMaxTokens = 4;
 
 // True when a small-batch kernel handles this problem: groups of at least 64 elements and either byte zero points
-// (with packed rows that are multiples of 16 bytes) and at most 32 tokens (tensor-core kernel, at most eight tokens per launch; several launches only
+// (with packed rows that are multiples of 16 bytes) and at most 64 tokens (tensor-core kernel, at most eight tokens per launch; several launches only
 // while they are cheaper than the tiled kernel), or at most kGemvMaxTokens tokens and activations (as fp32) that fit
 // in the shared memory of one CTA.
 bool packed_gemv_applies(const eqat_desc& d);

@@ -676,6 +676,8 @@ def test_few_token_forwards_back_to_back_keep_their_order(eqat, bits, group, tok
     (80 * 16, 2304, 5, 3, 256),     # 3-bit codes, groups of 256, nine boxes per row, 80 row-blocks
     (64, 11008, 8, 3, 64),          # 3-bit codes, groups of 64, 43 boxes per row, two launches of four tokens
     (64, 128, 1, 3, 128),           # 3-bit rows of 48 bytes: half a box, one group
+    (128, 11008, 40, 2, 64),        # forty tokens over long rows: eight launches of five
+    (128, 11008, 64, 4, 128),       # the most tokens that go out in slices: thirteen launches (twelve of five, one of four)
 ])
 def test_e2e_ragged(eqat, out, in_f, tokens, bits, group):
     cfg = small_cfg(f"e2er_{out}_{in_f}_{tokens}", out, in_f, bits, group, tokens)
