@@ -226,13 +226,11 @@ int eqat_unpack_zeros(const eqat_desc* desc, const uint8_t* z_packed, uint8_t* z
  * desc->zero_point_format is EQAT_ZP_FP16. */
 
 /* Y = X * ((W_int - z) * s)^T, the packed codes expanded tile by tile in
- * shared memory inside the GEMM (Eq. 2; Sec. 3.3).  With one to four tokens
- * (decoding) and groups of at least 64 a matrix-vector kernel streams the
- * packed weight instead and does not round (W_int - z) * s to bf16.  With byte
- * zero points (and, for 3-bit codes, packed rows that are multiples of 16
- * bytes) that kernel runs on matrix instructions and takes up to eight tokens
- * per launch, and up to 64 tokens go through it in slices (one pass over the
- * packed weight per slice) while that is cheaper than the tiled kernel; a
+ * shared memory inside the GEMM (Eq. 2; Sec. 3.3).  With few tokens (decoding)
+ * and groups of at least 64 a matrix-vector kernel streams the packed weight
+ * instead and does not round (W_int - z) * s to bf16.  It takes up to eight
+ * tokens per launch, and up to 64 tokens go through it in slices (one pass over
+ * the packed weight per slice) while that is cheaper than the tiled kernel; a
  * token's result does not depend on how the tokens were sliced.
  *   X [T,in] bf16, Wq_packed, s16, z (in)   Y [T,out] bf16 (out) */
 int qlinear_packed_fwd(const eqat_desc* desc, const eqat_bf16* X, const uint8_t* Wq_packed,

@@ -2,25 +2,12 @@
 //     Y[T,out] = X[T,in] * dequant(Wq)^T,
 // the matrix-vector case of the E2E-QP forward (Eq. 2 on frozen codes).  The
 // 512-row tensor-memory tiles of gemm.cu would be almost empty here; the work is
-// one pass over the packed weight, so the kernels are streams over its bytes.
-// Two kernels: the first (below) runs on the ordinary cores and takes every bit
-// width and zero-point format for up to four tokens; the second (further down)
-// builds weight fragments for warp-level matrix instructions and takes codes
-// with byte zero points for up to eight tokens per launch (more tokens, or rows
-// too long for the staged activations, go out as several launches).
-//
-// First kernel.  Mapping: a CTA owns 32 consecutive weight rows, lane = row, and
-// its 16 warps split the row into contiguous runs of 64-code units.  All lanes
-// of a warp are on the same columns, so the activations are read from shared
-// memory as broadcasts (one wavefront per 16-byte load); each warp stages the
-// columns of its own units there as fp32, together with their sum over every
-// 64-column unit.
-//
-// Arithmetic: a code q is dropped into the top mantissa bits of the float 1.0,
-// giving 1 + q/2^N with two logic operations and no int-to-float conversion.
-// For a unit with step size s and zero point z
-//     sum_j (q_j - z) s x_j = s (2^N * sum_j (1 + q_j/2^N) x_j - (2^N + z) * sum_j x_j),
-// all in fp32, so the dequantised weight is never rounded to bf16 here.
+// one pass over the packed weight, so the kernel is a stream over its bytes that
+// builds weight fragments for warp-level matrix instructions in registers.  It
+// takes up to eight tokens per launch (more tokens, or rows too long for the
+// staged activations, go out as several launches).  The dequantised weight is
+// never rounded to bf16 here: the codes enter the matrix instructions as exact
+// small numbers and the step size scales fp32 accumulators.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -31,258 +18,13 @@
 namespace eqat {
 namespace {
 
-constexpr int kWarps = 16;
-constexpr int kThreads = kWarps * 32;
-constexpr int kRows = 32;                   // weight rows per CTA = lanes
-constexpr size_t kMaxSmem = 200 * 1024;
-
-__host__ __device__ inline size_t smem_floats(int T, int in_features) {
-  return (size_t)T * in_features + (size_t)T * (in_features >> 6) + (size_t)kWarps * T * 32;
-}
-
-// Code c (0..63) of a 64-code unit held in 2*BITS words, as the float 1 + q/2^BITS.
-template <int BITS>
-__device__ __forceinline__ float code_as_float(const uint32_t (&w)[2 * BITS], int c) {
-  const int bit = BITS * c, word = bit >> 5, off = bit & 31;
-  constexpr int pos = 23 - BITS;            // lowest mantissa bit the code occupies
-  uint32_t t;
-  if (off + BITS <= 32) {
-    t = off <= pos ? w[word] << (pos - off) : w[word] >> (off - pos);
-  } else {
-    t = __funnelshift_r(w[word], w[word + 1], off - pos);      // 3-bit codes that straddle two words
-  }
-  // (t & mask) | 1.0f as one three-input logic operation: both constants are passed in registers, which the
-  // compiler otherwise folds into two instructions with one immediate each.
-  uint32_t r;
-  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(t), "r"(((1u << BITS) - 1u) << pos), "r"(0x3F800000u));
-  return __uint_as_float(r);
-}
-
-template <int BITS>
-__device__ __forceinline__ void load_unit(const uint8_t* p, uint32_t (&w)[2 * BITS]) {
-  if constexpr (BITS == 3) {
-#pragma unroll
-    for (int i = 0; i < 3; ++i) {
-      const uint2 t = __ldg(reinterpret_cast<const uint2*>(p) + i);
-      w[2 * i] = t.x; w[2 * i + 1] = t.y;
-    }
-  } else {
-#pragma unroll
-    for (int i = 0; i < BITS / 2; ++i) {
-      const uint4 t = __ldg(reinterpret_cast<const uint4*>(p) + i);
-      w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
-    }
-  }
-}
-
-template <int BITS, int T>
-__global__ void __launch_bounds__(kThreads)
-packed_gemv_kernel(const eqat_bf16* __restrict__ X, const uint8_t* __restrict__ Wq, const eqat_fp16* __restrict__ s16,
-                   const void* __restrict__ zq, eqat_bf16* __restrict__ Y, int out_features, int in_features,
-                   int group_shift, int groups_per_row, int sectors, int z_fp16) {
-  extern __shared__ __align__(16) float smem_f[];
-  const int units = in_features >> 6;
-  float* xs = smem_f;                                   // [T][in]
-  float* xsum = xs + (size_t)T * in_features;           // [T][units]
-  float* part = xsum + (size_t)T * units;               // [warps][T][32]
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  const int row = blockIdx.x * kRows + lane;
-  const bool live = row < out_features;
-  const uint8_t* wrow = Wq + (size_t)(live ? row : 0) * ((size_t)in_features * BITS / 8);
-  const eqat_fp16* srow = s16 + (size_t)(live ? row : 0) * groups_per_row;
-  // zero points: one byte each, or (z_fp16) one fp16 value each; kept as 16 raw bits next to the step size
-  const size_t zrow = (size_t)(live ? row : 0) * groups_per_row;
-  const uint8_t* z8 = static_cast<const uint8_t*>(zq);
-  const eqat_fp16* z16 = static_cast<const eqat_fp16*>(zq);
-  // whole pairs of units per warp (in_features is a multiple of 128): a pair is 32-byte aligned for 2- and
-  // 4-bit codes, and lies in one group or in two consecutive ones
-  const int pairs = units >> 1;
-  const int u_begin = 2 * (int)((long)pairs * warp / kWarps), u_end = 2 * (int)((long)pairs * (warp + 1) / kWarps);
-  constexpr float kScale = (float)(1 << BITS);
-
-  float acc[T];
-#pragma unroll
-  for (int t = 0; t < T; ++t) acc[t] = 0.0f;
-  // Units are taken kBatch at a time and the next batch is requested before the current one is used, so every
-  // lane keeps 128 bytes of its row in flight: the rows of a warp are kilobytes apart, and with one unit per
-  // request the kernel waited on DRAM latency instead of streaming.
-  constexpr int kBatch = BITS == 2 ? 4 : 2;
-  uint32_t w_nxt[kBatch][2 * BITS];
-  uint32_t sz_nxt[kBatch];                              // fp16 step size | zero point << 16, fetched with the codes
-  auto fetch = [&](int u0) {
-#pragma unroll
-    for (int k = 0; k < kBatch; k += 2)
-      if (u0 + k < u_end) {
-        const uint8_t* src = wrow + (size_t)(u0 + k) * (8 * BITS);
-        // `sectors`: the packed matrix starts on a 32-byte boundary, so every pair of units does too and is
-        // fetched as whole 32-byte sectors; otherwise with 16-byte (3-bit: 8-byte) loads
-        bool fetched = false;
-        if constexpr (BITS == 2) {
-          if (sectors) {                                // both units: one 32-byte sector
-            ptx::ldg_256(src, reinterpret_cast<uint32_t(&)[8]>(w_nxt[k][0]));
-            fetched = true;
-          }
-        } else if constexpr (BITS == 4) {
-          if (sectors) {
-            ptx::ldg_256(src, w_nxt[k]);
-            ptx::ldg_256(src + 32, w_nxt[k + 1]);
-            fetched = true;
-          }
-        }
-        if (!fetched) {
-          load_unit<BITS>(src, w_nxt[k]);
-          load_unit<BITS>(src + 8 * BITS, w_nxt[k + 1]);
-        }
-        const int g = ((u0 + k) << 6) >> group_shift;
-        if (group_shift == 6) {
-          const uint32_t s2 = __ldg(reinterpret_cast<const uint32_t*>(srow + g));
-          if (z_fp16) {
-            const uint32_t z2 = __ldg(reinterpret_cast<const uint32_t*>(z16 + zrow + g));
-            sz_nxt[k] = (s2 & 0xFFFFu) | (z2 << 16);
-            sz_nxt[k + 1] = (s2 >> 16) | (z2 & 0xFFFF0000u);
-          } else {
-            const uint32_t z2 = __ldg(reinterpret_cast<const unsigned short*>(z8 + zrow + g));
-            sz_nxt[k] = (s2 & 0xFFFFu) | ((z2 & 0xFFu) << 16);
-            sz_nxt[k + 1] = (s2 >> 16) | ((z2 >> 8) << 16);
-          }
-        } else {
-          const uint32_t zraw = z_fp16 ? (uint32_t)__ldg(z16 + zrow + g) : (uint32_t)__ldg(z8 + zrow + g);
-          sz_nxt[k] = sz_nxt[k + 1] = (uint32_t)__ldg(srow + g) | (zraw << 16);
-        }
-      }
-  };
-  fetch(u_begin);                                       // in flight while this warp stages its activations
-
-  // A warp reads only the columns of its own units, so it stages just those (bf16 -> fp32) and their per-unit
-  // sums itself: no CTA-wide barrier before the main loop.
-  {
-    const int nu = u_end - u_begin;
-    for (int i = lane; i < T * nu * 8; i += 32) {       // one 16-byte piece (8 bf16) per iteration
-      const int t = i / (nu * 8), r8 = i - t * (nu * 8);
-      const size_t e0 = (size_t)t * in_features + (size_t)u_begin * 64 + (size_t)r8 * 8;
-      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(X + e0));
-      const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
-      float4 lo, hi;
-      lo.x = __uint_as_float(r[0] << 16); lo.y = __uint_as_float(r[0] & 0xFFFF0000u);
-      lo.z = __uint_as_float(r[1] << 16); lo.w = __uint_as_float(r[1] & 0xFFFF0000u);
-      hi.x = __uint_as_float(r[2] << 16); hi.y = __uint_as_float(r[2] & 0xFFFF0000u);
-      hi.z = __uint_as_float(r[3] << 16); hi.w = __uint_as_float(r[3] & 0xFFFF0000u);
-      reinterpret_cast<float4*>(xs + e0)[0] = lo;
-      reinterpret_cast<float4*>(xs + e0)[1] = hi;
-    }
-    __syncwarp();
-    for (int i = 0; i < T * nu; ++i) {                  // two elements per lane, fixed-order tree
-      const int t = i / nu, u = u_begin + (i - t * nu);
-      const float* xu = xs + (size_t)t * in_features + (size_t)u * 64;
-      float v = xu[lane] + xu[32 + lane];
-#pragma unroll
-      for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
-      if (lane == 0) xsum[t * units + u] = v;
-    }
-    __syncwarp();
-  }
-#pragma unroll 1
-  for (int u0 = u_begin; u0 < u_end; u0 += kBatch) {
-    uint32_t w[kBatch][2 * BITS], sz[kBatch];
-#pragma unroll
-    for (int k = 0; k < kBatch; ++k) {
-      sz[k] = sz_nxt[k];
-#pragma unroll
-      for (int i = 0; i < 2 * BITS; ++i) w[k][i] = w_nxt[k][i];
-    }
-    fetch(u0 + kBatch);
-#pragma unroll
-    for (int k = 0; k < kBatch; ++k) {
-      const int u = u0 + k;
-      if (u < u_end) {
-        const float s = __half2float(__ushort_as_half((unsigned short)(sz[k] & 0xFFFFu)));
-        const float z = z_fp16 ? __half2float(__ushort_as_half((unsigned short)(sz[k] >> 16))) : (float)(sz[k] >> 16);
-        // four independent partial sums per token and kAhead activation loads in flight: the loop is otherwise a
-        // single chain of dependent multiply-adds behind one shared-memory load
-        constexpr int kAhead = T == 1 ? 4 : (T == 2 ? 2 : 1);
-        float d4[T][4];
-#pragma unroll
-        for (int t = 0; t < T; ++t)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) d4[t][e] = 0.0f;
-#pragma unroll
-        for (int j = 0; j < 64; j += 4 * kAhead) {
-          float4 xv[kAhead][T];
-#pragma unroll
-          for (int a = 0; a < kAhead; ++a)
-#pragma unroll
-            for (int t = 0; t < T; ++t)
-              xv[a][t] = *reinterpret_cast<const float4*>(xs + (size_t)t * in_features + (size_t)u * 64 + j + 4 * a);
-#pragma unroll
-          for (int a = 0; a < kAhead; ++a) {
-            const int c = j + 4 * a;
-            const float q0 = code_as_float<BITS>(w[k], c), q1 = code_as_float<BITS>(w[k], c + 1),
-                        q2 = code_as_float<BITS>(w[k], c + 2), q3 = code_as_float<BITS>(w[k], c + 3);
-#pragma unroll
-            for (int t = 0; t < T; ++t) {
-              d4[t][0] = fmaf(q0, xv[a][t].x, d4[t][0]);
-              d4[t][1] = fmaf(q1, xv[a][t].y, d4[t][1]);
-              d4[t][2] = fmaf(q2, xv[a][t].z, d4[t][2]);
-              d4[t][3] = fmaf(q3, xv[a][t].w, d4[t][3]);
-            }
-          }
-        }
-        float dot[T];
-#pragma unroll
-        for (int t = 0; t < T; ++t) dot[t] = (d4[t][0] + d4[t][1]) + (d4[t][2] + d4[t][3]);
-#pragma unroll
-        for (int t = 0; t < T; ++t)
-          acc[t] = fmaf(s, fmaf(kScale, dot[t], -(kScale + z) * xsum[t * units + u]), acc[t]);
-      }
-    }
-  }
-#pragma unroll
-  for (int t = 0; t < T; ++t) part[(warp * T + t) * 32 + lane] = acc[t];
-  __syncthreads();
-  if (warp < T && live) {
-    float v = 0.0f;
-#pragma unroll
-    for (int wv = 0; wv < kWarps; ++wv) v += part[(wv * T + warp) * 32 + lane];      // fixed order: deterministic
-    Y[(size_t)warp * out_features + row] = (eqat_bf16)(pack_bf16x2(v, 0.0f) & 0xFFFFu);
-  }
-}
-
-template <int BITS, int T>
-int launch_one(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
-               eqat_bf16* Y, int group_shift, cudaStream_t st) {
-  auto kern = packed_gemv_kernel<BITS, T>;
-  const size_t smem = smem_floats(T, d.in_features) * sizeof(float);
-  if (smem > 48 * 1024) {
-    static SmemOptIn opt_in;        // raise the kernel's shared-memory limit once per device
-    if (!opt_in.ensure(kern, (int)kMaxSmem)) return EQAT_ERR_CUDA;
-  }
-  const int grid = (d.out_features + kRows - 1) / kRows;
-  const int sectors = (reinterpret_cast<uintptr_t>(Wq) & 31u) == 0 ? 1 : 0;
-  kern<<<grid, kThreads, smem, st>>>(X, Wq, s16, zq, Y, d.out_features, d.in_features, group_shift,
-                                     d.in_features / d.group, sectors, d.zero_point_format == EQAT_ZP_FP16 ? 1 : 0);
-  return launch_status();
-}
-
-template <int BITS>
-int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
-                eqat_bf16* Y, int group_shift, cudaStream_t st) {
-  switch ((int)d.tokens) {
-    case 1: return launch_one<BITS, 1>(d, X, Wq, s16, zq, Y, group_shift, st);
-    case 2: return launch_one<BITS, 2>(d, X, Wq, s16, zq, Y, group_shift, st);
-    case 3: return launch_one<BITS, 3>(d, X, Wq, s16, zq, Y, group_shift, st);
-    default: return launch_one<BITS, 4>(d, X, Wq, s16, zq, Y, group_shift, st);
-  }
-}
-
-
 // ====================================================================== codes on tensor-core tiles
-// The kernel above spends three instructions per code and token on the ordinary
-// cores.  That is several times what the bytes allow, so codes with byte zero
-// points go through warp-level matrix instructions instead (mma.sync m16n8k16,
-// bf16 in, fp32 out): 16 weight rows by 16 columns against up to 8 tokens per
-// instruction, with the weight fragment built in registers, one logic
-// operation per PAIR of codes.  (The paired-CTA tensor-memory path of gemm.cu
+// A loop on the ordinary cores spends three instructions per code and token.
+// That is several times what the bytes allow, so the codes go through
+// warp-level matrix instructions instead (mma.sync m16n8k16, bf16 in, fp32
+// out): 16 weight rows by 16 columns against up to 8 tokens per instruction,
+// with the weight fragment built in registers, one logic operation per PAIR of
+// codes.  (The paired-CTA tensor-memory path of gemm.cu
 // wants its operands expanded into shared memory, which is exactly the cost to
 // avoid here; and with at most a few tokens there is nothing for a 128-row
 // accumulator to amortise.)
@@ -317,8 +59,9 @@ int launch_bits(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const
 // a chunk, supplies four of its 16 codes (2m, 2m+8, 2m+1, 2m+9 for 2-bit codes;
 // tc_column gives the order for every width); the activations are staged once
 // per CTA in exactly that order, so a lane fetches its fragment of X for an
-// instruction with one 8-byte load.  Zero points are one byte each here (the
-// fp16 variant goes through the kernel above).  The 16 warps' partial sums of a
+// instruction with one 8-byte load.  Zero points are one byte each, or fp16
+// values (ZF16): then 128 + z is split into three bf16 numbers like the sums
+// and the fifth instruction holds all nine products.  The 16 warps' partial sums of a
 // task go through a double-buffered shared array to a reducer warp, which adds
 // them in a fixed order and stores Y while the consumers are on the next task.
 constexpr int kTcMaxTokens = 8;                         // the instruction has eight token columns
@@ -484,10 +227,10 @@ __host__ __device__ constexpr float tc_bias(int j) {
   return BITS == 4 ? 128.0f : ((j & 7) % 3 == 0 ? 128.0f : ((j & 7) % 3 == 1 ? 32.0f : 8.0f));
 }
 
-template <int BITS, int PARAM_MODE>
+template <int BITS, int PARAM_MODE, bool ZF16>
 __global__ void __launch_bounds__(kTcThreads, 1)
 packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16* __restrict__ X,
-                      const eqat_fp16* __restrict__ s16, const uint8_t* __restrict__ z8, eqat_bf16* __restrict__ Y,
+                      const eqat_fp16* __restrict__ s16, const void* __restrict__ zq, eqat_bf16* __restrict__ Y,
                       int out_features, int in_features, int group_shift, int groups_per_row, int T, int stages) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_addr(smem_raw);
@@ -552,46 +295,65 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
   // and kind where the rows of parameters keep the alignment for it; mode 0 fetches chunk by chunk.  Chunk c uses
   // slot c >> kSlotShift.  The loaded registers are not touched before the stage is computed (three stages later):
   // an instruction on them here would wait for the load.
-  struct StageParams { uint2 s_lo, s_hi; uint32_t z_lo, z_hi; };
+  // Zero points: one byte per slot in z_lo.x / z_hi.x, or (ZF16) one fp16 value per slot like the step sizes.
+  struct StageParams { uint2 s_lo, s_hi, z_lo, z_hi; };
   constexpr int kSlotShift = PARAM_MODE == 2 ? 1 : (PARAM_MODE == 3 ? 2 : 0);
+  const uint8_t* const z8 = static_cast<const uint8_t*>(zq);
+  const eqat_fp16* const z16 = static_cast<const eqat_fp16*>(zq);
   auto fetch = [&](int task, int k) {
     StageParams sp;
-    sp.s_lo = sp.s_hi = make_uint2(0u, 0u);
-    sp.z_lo = sp.z_hi = 0u;
+    sp.s_lo = sp.s_hi = sp.z_lo = sp.z_hi = make_uint2(0u, 0u);
     const int cg0 = (k * kBoxesPerStage + box) * kChunksPerBox + chunk0;
     if (task < n_tasks && cg0 < chunks) {
       const size_t p_lo = (size_t)(task * kTcRows + g) * groups_per_row, p_hi = p_lo + (size_t)8 * groups_per_row;
       if constexpr (PARAM_MODE == 1) {                    // the row has a multiple of four groups: all four exist
         sp.s_lo = __ldg(reinterpret_cast<const uint2*>(s16 + p_lo + cg0));
         sp.s_hi = __ldg(reinterpret_cast<const uint2*>(s16 + p_hi + cg0));
-        sp.z_lo = __ldg(reinterpret_cast<const uint32_t*>(z8 + p_lo + cg0));
-        sp.z_hi = __ldg(reinterpret_cast<const uint32_t*>(z8 + p_hi + cg0));
+        if constexpr (ZF16) {
+          sp.z_lo = __ldg(reinterpret_cast<const uint2*>(z16 + p_lo + cg0));
+          sp.z_hi = __ldg(reinterpret_cast<const uint2*>(z16 + p_hi + cg0));
+        } else {
+          sp.z_lo.x = __ldg(reinterpret_cast<const uint32_t*>(z8 + p_lo + cg0));
+          sp.z_hi.x = __ldg(reinterpret_cast<const uint32_t*>(z8 + p_hi + cg0));
+        }
       } else if constexpr (PARAM_MODE == 2) {             // an even number of groups per row: both exist
         const int g0 = cg0 >> 1;
         sp.s_lo.x = __ldg(reinterpret_cast<const uint32_t*>(s16 + p_lo + g0));
         sp.s_hi.x = __ldg(reinterpret_cast<const uint32_t*>(s16 + p_hi + g0));
-        sp.z_lo = __ldg(reinterpret_cast<const uint16_t*>(z8 + p_lo + g0));
-        sp.z_hi = __ldg(reinterpret_cast<const uint16_t*>(z8 + p_hi + g0));
+        if constexpr (ZF16) {
+          sp.z_lo.x = __ldg(reinterpret_cast<const uint32_t*>(z16 + p_lo + g0));
+          sp.z_hi.x = __ldg(reinterpret_cast<const uint32_t*>(z16 + p_hi + g0));
+        } else {
+          sp.z_lo.x = __ldg(reinterpret_cast<const uint16_t*>(z8 + p_lo + g0));
+          sp.z_hi.x = __ldg(reinterpret_cast<const uint16_t*>(z8 + p_hi + g0));
+        }
       } else if constexpr (PARAM_MODE == 3) {
         const int grp = (cg0 << 6) >> group_shift;
         sp.s_lo.x = __ldg(s16 + p_lo + grp);
         sp.s_hi.x = __ldg(s16 + p_hi + grp);
-        sp.z_lo = __ldg(z8 + p_lo + grp);
-        sp.z_hi = __ldg(z8 + p_hi + grp);
+        sp.z_lo.x = ZF16 ? (uint32_t)__ldg(z16 + p_lo + grp) : (uint32_t)__ldg(z8 + p_lo + grp);
+        sp.z_hi.x = ZF16 ? (uint32_t)__ldg(z16 + p_hi + grp) : (uint32_t)__ldg(z8 + p_hi + grp);
       } else {
-        uint32_t sl[4] = {0u, 0u, 0u, 0u}, sh[4] = {0u, 0u, 0u, 0u};
+        uint32_t sl[4] = {0u, 0u, 0u, 0u}, sh[4] = {0u, 0u, 0u, 0u}, zl[4] = {0u, 0u, 0u, 0u}, zh[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
         for (int c = 0; c < kChunksPerWarp; ++c) {
           if (cg0 + c < chunks) {
             const int grp = ((cg0 + c) << 6) >> group_shift;
             sl[c] = __ldg(s16 + p_lo + grp);
             sh[c] = __ldg(s16 + p_hi + grp);
-            sp.z_lo |= (uint32_t)__ldg(z8 + p_lo + grp) << (8 * c);
-            sp.z_hi |= (uint32_t)__ldg(z8 + p_hi + grp) << (8 * c);
+            zl[c] = ZF16 ? (uint32_t)__ldg(z16 + p_lo + grp) : (uint32_t)__ldg(z8 + p_lo + grp);
+            zh[c] = ZF16 ? (uint32_t)__ldg(z16 + p_hi + grp) : (uint32_t)__ldg(z8 + p_hi + grp);
           }
         }
         sp.s_lo = make_uint2(sl[0] | (sl[1] << 16), sl[2] | (sl[3] << 16));
         sp.s_hi = make_uint2(sh[0] | (sh[1] << 16), sh[2] | (sh[3] << 16));
+        if constexpr (ZF16) {
+          sp.z_lo = make_uint2(zl[0] | (zl[1] << 16), zl[2] | (zl[3] << 16));
+          sp.z_hi = make_uint2(zh[0] | (zh[1] << 16), zh[2] | (zh[3] << 16));
+        } else {
+          sp.z_lo.x = zl[0] | (zl[1] << 8) | (zl[2] << 16) | (zl[3] << 24);
+          sp.z_hi.x = zh[0] | (zh[1] << 8) | (zh[2] << 16) | (zh[3] << 24);
+        }
       }
     }
     return sp;
@@ -604,7 +366,7 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
   };
 #pragma unroll
   for (int i = 0; i < kTcAhead; ++i) {
-    nx[i] = StageParams{make_uint2(0u, 0u), make_uint2(0u, 0u), 0u, 0u};
+    nx[i] = StageParams{make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u)};
     if (warp < kTcWarps) { nx[i] = fetch(pf_task, pf_k); advance(); }
   }
 
@@ -726,8 +488,10 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
             }
           uint2* item = xb + ((size_t)cg * 4 * T + t) * kTcItems + 4;    // + quad lane * T * kTcItems
           item[0 * T * kTcItems] = make_uint2(parts[0][0] | (parts[0][1] << 16), parts[0][2] | (parts[1][0] << 16));
-          item[1 * T * kTcItems] = make_uint2(parts[1][1] | (parts[1][2] << 16), 0u);
-          item[2 * T * kTcItems] = make_uint2(0u, 0u);
+          // the three parts of xs once more per part of a three-part zero point (fp16 zero points; with byte zero
+          // points their weights are zero)
+          item[1 * T * kTcItems] = make_uint2(parts[1][1] | (parts[1][2] << 16), parts[1][0] | (parts[1][1] << 16));
+          item[2 * T * kTcItems] = make_uint2(parts[1][2] | (parts[1][0] << 16), parts[1][1] | (parts[1][2] << 16));
           item[3 * T * kTcItems] = make_uint2(0u, 0u);
         }
       }
@@ -809,15 +573,36 @@ packed_gemv_tc_kernel(const __grid_constant__ CUtensorMap map_w, const eqat_bf16
               if (m == 0) mma_16816_first(D, a0, a1, a2, a3, b.x, b.y);
               else mma_16816(D, a0, a1, a2, a3, b.x, b.y);
             }
-            {
+            const int slot = c >> kSlotShift;                          // a constant once the loop is unrolled
+            if constexpr (ZF16) {
+              // correction with a real zero point: 128 + z as three bf16 numbers (an fp32 value split without
+              // loss), each against the three parts of xs
+              const uint32_t z2_lo = slot < 2 ? sp.z_lo.x : sp.z_lo.y, z2_hi = slot < 2 ? sp.z_hi.x : sp.z_hi.y;
+              uint32_t a[2][2];
+#pragma unroll
+              for (int hrow = 0; hrow < 2; ++hrow) {
+                const uint32_t z2 = hrow == 0 ? z2_lo : z2_hi;
+                float t = 128.0f + __half2float(__ushort_as_half((unsigned short)((slot & 1) ? (z2 >> 16) : (z2 & 0xFFFFu))));
+                uint32_t n[3];                                         // the negated parts
+#pragma unroll
+                for (int pce = 0; pce < 3; ++pce) {
+                  const uint32_t hb = pack_bf16x2(t, 0.0f) & 0xFFFFu;
+                  t -= __uint_as_float(hb << 16);
+                  n[pce] = hb ^ 0x8000u;
+                }
+                a[hrow][0] = q == 0 ? 0xBF80BF80u : (q == 1 ? n[0] * 0x10001u : (q == 2 ? (n[1] | (n[2] << 16)) : 0u));
+                a[hrow][1] = q == 0 ? (0xBF80u | (n[0] << 16)) : (q == 1 ? n[1] * 0x10001u : (q == 2 ? n[2] * 0x10001u : 0u));
+              }
+              const uint2 b = item[4];
+              mma_16816(D, a[0][0], a[1][0], a[0][1], a[1][1], b.x, b.y);
+            } else {
               // correction: weights -1 and -(128 + z) against the split sums (see the header)
-              const uint32_t zz_lo = ((sp.z_lo >> (8 * (c >> kSlotShift))) & 0xFFu) * 0x10001u;
-              const uint32_t zz_hi = ((sp.z_hi >> (8 * (c >> kSlotShift))) & 0xFFu) * 0x10001u;
+              const uint32_t zz_lo = ((sp.z_lo.x >> (8 * slot)) & 0xFFu) * 0x10001u;
+              const uint32_t zz_hi = ((sp.z_hi.x >> (8 * slot)) & 0xFFu) * 0x10001u;
               const uint2 b = item[4];
               mma_16816(D, and_or(zz_lo, mask_a, const_a), and_or(zz_hi, mask_a, const_a), and_or(zz_lo, mask_b, const_b),
                         and_or(zz_hi, mask_b, const_b), b.x, b.y);
             }
-            const int slot = c >> kSlotShift;                          // a constant once the loop is unrolled
             const uint32_t s2_lo = slot < 2 ? sp.s_lo.x : sp.s_lo.y, s2_hi = slot < 2 ? sp.s_hi.x : sp.s_hi.y;
             const float s_lo = __half2float(__ushort_as_half((unsigned short)((slot & 1) ? (s2_lo >> 16) : (s2_lo & 0xFFFFu))));
             const float s_hi = __half2float(__ushort_as_half((unsigned short)((slot & 1) ? (s2_hi >> 16) : (s2_hi & 0xFFFFu))));
@@ -887,11 +672,11 @@ bool make_tmap_u8_plain(CUtensorMap* tm, const void* base, uint64_t inner_bytes,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BITS, int PARAM_MODE>
+template <int BITS, int PARAM_MODE, bool ZF16>
 int launch_tc_mode(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
                    eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
   static SmemOptIn opt_in;
-  if (!opt_in.ensure(packed_gemv_tc_kernel<BITS, PARAM_MODE>, (int)kTcSmemBudget)) return EQAT_ERR_CUDA;
+  if (!opt_in.ensure(packed_gemv_tc_kernel<BITS, PARAM_MODE, ZF16>, (int)kTcSmemBudget)) return EQAT_ERR_CUDA;
   CUtensorMap mw;
   const uint64_t row_bytes = (uint64_t)d.in_features * BITS / 8;
   if (!(BITS == 3 ? make_tmap_u8_plain(&mw, Wq, row_bytes, (uint64_t)d.out_features, tc_box_bytes(BITS), kTcRows)
@@ -914,7 +699,7 @@ int launch_tc_mode(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, co
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, packed_gemv_tc_kernel<BITS, PARAM_MODE>, mw, X, s16, static_cast<const uint8_t*>(zq), Y,
+  if (cudaLaunchKernelEx(&cfg, packed_gemv_tc_kernel<BITS, PARAM_MODE, ZF16>, mw, X, s16, zq, Y,
                          d.out_features, d.in_features, group_shift, ng, T, stages) != cudaSuccess) {
     (void)cudaGetLastError();
     return EQAT_ERR_CUDA;
@@ -922,19 +707,27 @@ int launch_tc_mode(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, co
   return launch_status();
 }
 
-template <int BITS>
-int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
-              eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
+template <int BITS, bool ZF16>
+int launch_tc_format(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
+                     eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
   // how a lane fetches the parameters of its 256 columns of a stage (see the kernel): one load per row and kind
   // where the rows of step sizes and zero points keep the alignment those loads need, chunk by chunk otherwise
   const uintptr_t s_addr = reinterpret_cast<uintptr_t>(s16), z_addr = reinterpret_cast<uintptr_t>(zq);
+  const uintptr_t z_unit = ZF16 ? 2 : 1;                 // bytes per zero point
   const int ng = d.in_features / d.group;
-  if (d.group == 64 && ng % 4 == 0 && (s_addr & 7u) == 0 && (z_addr & 3u) == 0)
-    return launch_tc_mode<BITS, 1>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
-  if (d.group == 128 && ng % 2 == 0 && (s_addr & 3u) == 0 && (z_addr & 1u) == 0)
-    return launch_tc_mode<BITS, 2>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
-  if (d.group >= 256) return launch_tc_mode<BITS, 3>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
-  return launch_tc_mode<BITS, 0>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
+  if (d.group == 64 && ng % 4 == 0 && (s_addr & 7u) == 0 && (z_addr & (4 * z_unit - 1)) == 0)
+    return launch_tc_mode<BITS, 1, ZF16>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
+  if (d.group == 128 && ng % 2 == 0 && (s_addr & 3u) == 0 && (z_addr & (2 * z_unit - 1)) == 0)
+    return launch_tc_mode<BITS, 2, ZF16>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
+  if (d.group >= 256) return launch_tc_mode<BITS, 3, ZF16>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
+  return launch_tc_mode<BITS, 0, ZF16>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
+}
+
+template <int BITS>
+int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16, const void* zq,
+              eqat_bf16* Y, int group_shift, int stages, cudaStream_t st) {
+  return d.zero_point_format == EQAT_ZP_FP16 ? launch_tc_format<BITS, true>(d, X, Wq, s16, zq, Y, group_shift, stages, st)
+                                             : launch_tc_format<BITS, false>(d, X, Wq, s16, zq, Y, group_shift, stages, st);
 }
 
 }  // namespace
@@ -954,7 +747,6 @@ static TcPlan tc_plan(const eqat_desc& d) {
   const TcPlan none{0, 0};
   if (d.bits < 2 || d.bits > 4 || d.group < 64 || d.tokens < 1 || d.tokens > kTcMaxTotalTokens) return none;
   if (((int64_t)d.in_features * d.bits / 8) % 16 != 0) return none;    // the copy engine wants rows of 16-byte multiples
-  if (d.zero_point_format != EQAT_ZP_U8) return none;
   const int T = (int)d.tokens;
   int fit = T < kTcMaxTokens ? T : kTcMaxTokens;
   while (fit >= 1 && tc_stages_that_fit(fit, d.in_features, d.bits) == 0) --fit;
@@ -971,10 +763,8 @@ static TcPlan tc_plan(const eqat_desc& d) {
 }
 
 bool packed_gemv_applies(const eqat_desc& d) {
-  // a 64-code unit must lie inside one group: groups of 32 go through the tiled kernel
-  if (d.tokens < 1 || d.group < 64) return false;
-  if (tc_plan(d).launches > 0) return true;
-  return d.tokens <= kGemvMaxTokens && smem_floats((int)d.tokens, d.in_features) * sizeof(float) <= kMaxSmem;
+  // a 64-column chunk must lie inside one group: groups of 32 go through the tiled kernel
+  return d.tokens >= 1 && d.group >= 64 && tc_plan(d).launches > 0;
 }
 
 int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,
@@ -999,11 +789,7 @@ int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq
     }
     return EQAT_OK;
   }
-  switch (d.bits) {
-    case 2: return launch_bits<2>(d, X, Wq, s16, zq, Y, group_shift, st);
-    case 3: return launch_bits<3>(d, X, Wq, s16, zq, Y, group_shift, st);
-    default: return launch_bits<4>(d, X, Wq, s16, zq, Y, group_shift, st);
-  }
+  return EQAT_ERR_UNSUPPORTED;                           // not reached for a problem packed_gemv_applies() accepted
 }
 
 int launch_wait_expiry_gemv(cudaStream_t st) {

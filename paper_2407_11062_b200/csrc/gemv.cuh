@@ -5,12 +5,9 @@
 
 namespace eqat {
 
-constexpr int kGemvMaxTokens = 4;
-
-// True when a small-batch kernel handles this problem: groups of at least 64 elements and either byte zero points
-// (with packed rows that are multiples of 16 bytes) and at most 64 tokens (tensor-core kernel, at most eight tokens per launch; several launches only
-// while they are cheaper than the tiled kernel), or at most kGemvMaxTokens tokens and activations (as fp32) that fit
-// in the shared memory of one CTA.
+// True when the few-token kernel handles this problem: groups of at least 64 elements, at most 64 tokens, staged
+// activations of at least one token that fit in the shared memory of a CTA, and, where the tokens need several
+// launches, a cost estimate below the tiled kernel's.
 bool packed_gemv_applies(const eqat_desc& d);
 // Y[T,out] = X[T,in] * dequant(Wq)^T for a problem packed_gemv_applies() accepted
 int launch_packed_gemv(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const eqat_fp16* s16,

@@ -541,6 +541,20 @@ def test_e2e_few_tokens(eqat, bits, tokens):
     check_e2e(run_e2e(eqat, cfg, cfg.linears[0], tokens), group)
 
 
+@pytest.mark.parametrize("bits,group,in_f,tokens", [
+    (2, 64, 1024, 1),       # four groups of 64 per 256 columns, vector loads of the parameters
+    (2, 64, 4096, 13),      # sliced: seven and six tokens
+    (3, 128, 2048, 5),      # two groups of 128 per 256 columns
+    (4, 128, 1408, 8),      # an odd number of groups per row: parameters fetched chunk by chunk
+    (2, 256, 1024, 3),      # one group per 256 columns
+    (4, 1152, 1152, 2),     # one group per row
+])
+def test_e2e_few_tokens_with_trained_zero_points(eqat, bits, group, in_f, tokens):
+    """The matrix-vector forward with fp16 zero points off the integers (the variant that trains z)."""
+    cfg = small_cfg(f"gemv_rz_{bits}_{group}_{tokens}", 320, in_f, bits, group, tokens, "student_t4", 0.02, 0.01)
+    check_e2e(run_e2e(eqat, cfg, cfg.linears[0], tokens, real_z=True), group)
+
+
 def test_few_token_forward_agrees_with_tiled_forward(eqat):
     """The same rows through both forward kernels (4 tokens alone, and as the first rows of a 9-token batch)."""
     cfg = small_cfg("gemv_vs_gemm", 512, 1024, 2, 64, 9)
