@@ -916,12 +916,13 @@ def run_streaming_case(args):
     print(json.dumps(r), flush=True)
 
 
-def decode_leg(eqat, dev, peaks, iters, model="7b", bits=BITS, group=GROUP, only_shape=None, tokens=(1, 4, 8, 16)):
+def decode_leg(eqat, dev, peaks, iters, model="7b", bits=BITS, group=GROUP, only_shape=None, tokens=(1, 4, 8, 16),
+               fp16_zero_points=False):
     """Few-token packed forward (the matrix-vector kernels) on the linear shapes of one block: device time per
     launch from a CUDA graph of launches over rotating weight copies (more than L2 in total), and the bandwidth that
     time means for the bytes one launch must read."""
     out = {"metric": "packed forward, few tokens", "unit": "us per call", "bits": bits, "group": group,
-           "model": model, "hbm_gbs_peak": peaks["hbm_gbs"],
+           "zero_points": "fp16" if fp16_zero_points else "uint8", "model": model, "hbm_gbs_peak": peaks["hbm_gbs"],
            "method": "CUDA graph of one call per weight copy (copies total > 2 x L2), replayed back to back; a call "
                      "is one kernel launch for up to 8 tokens where the staged activations fit, else one per token slice",
            "cases": {}}
@@ -933,14 +934,17 @@ def decode_leg(eqat, dev, peaks, iters, model="7b", bits=BITS, group=GROUP, only
         wbytes = o * i * bits // 8
         copies = max(4, int(320e6 // wbytes))
         Ps = [torch.randint(0, 256, (o, i * bits // 8), dtype=torch.uint8, device=dev) for _ in range(copies)]
-        z8 = torch.randint(0, 1 << bits, (o, ng), dtype=torch.uint8, device=dev)
+        if fp16_zero_points:
+            z8 = (torch.rand(o, ng, device=dev) * ((1 << bits) - 1)).half()
+        else:
+            z8 = torch.randint(0, 1 << bits, (o, ng), dtype=torch.uint8, device=dev)
         s16 = (torch.rand(o, ng, device=dev) * 0.01 + 0.001).half()
         for T in tokens:
             X = torch.randn(T, i, device=dev).to(torch.bfloat16)
             Y = torch.empty(T, o, dtype=torch.bfloat16, device=dev)
-            d = eqat.make_desc(bits, group, o, i, T)
+            d = eqat.make_desc(bits, group, o, i, T, 0, eqat.EQAT_ZP_FP16 if fp16_zero_points else eqat.EQAT_ZP_U8)
             us = time_rotation([lambda P=P: eqat.qlinear_packed_fwd(d, X, P, s16, z8, Y) for P in Ps], iters)
-            nbytes = wbytes + o * ng * 3 + T * (i + o) * 2
+            nbytes = wbytes + o * ng * (4 if fp16_zero_points else 3) + T * (i + o) * 2
             out["cases"][f"{lin.name}/T{T}"] = {"us": us, "bytes": nbytes, "gbs": nbytes / us / 1e3,
                                                  "frac_of_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
         del Ps
@@ -955,7 +959,8 @@ def run_decode_case(args):
     build_library()
     from paper_2407_11062_b200 import binding as eqat
     out = decode_leg(eqat, torch.device("cuda", 0), load_peaks(), args.case_iters, args.case_model, args.case_bits,
-                     args.case_group, args.decode_shape, tuple(int(t) for t in args.decode_tokens.split(",")))
+                     args.case_group, args.decode_shape, tuple(int(t) for t in args.decode_tokens.split(",")),
+                     args.decode_fp16_zero_points)
     assert eqat.device_status() == (0, 0)
     print(json.dumps(out), flush=True)
 
@@ -967,6 +972,7 @@ def main():
                     help="time the few-token packed forward on the linear shapes of --case-model (uses --case-iters)")
     ap.add_argument("--decode-shape", default=None, help="decode case: only this linear of the block (e.g. gate_up)")
     ap.add_argument("--decode-tokens", default="1,4,8,16", help="decode case: token counts, comma separated")
+    ap.add_argument("--decode-fp16-zero-points", action="store_true", help="decode case: zero points as fp16 values")
     ap.add_argument("--streaming-case", action="store_true", help="the cold streaming-kernel leg alone")
     ap.add_argument("--case-model", default="7b", choices=sorted(LINEARS))
     ap.add_argument("--case-shape", default="qkvo")
