@@ -732,7 +732,7 @@ int launch_tc(const eqat_desc& d, const eqat_bf16* X, const uint8_t* Wq, const e
 
 }  // namespace
 
-// Codes with byte zero points go through the tensor-core kernel: in one launch when the shared-memory plan fits all
+// How the tokens go through the kernel: in one launch when the shared-memory plan fits all
 // tokens, otherwise (long rows, or more than eight tokens) as several launches over slices of the tokens, each of
 // which streams the packed weight once more.  That is taken only while it is clearly cheaper than the tiled kernel
 // of gemm.cu.  Cost model (from timings on the Llama-2 7B, 13B and 70B shapes): a launch of this kernel takes about
